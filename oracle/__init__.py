@@ -1,0 +1,23 @@
+"""CPU oracle of the XNOR-Net forward block (test infrastructure only).
+
+Thin numpy/ctypes binding over ``xnor_oracle.c``; all arithmetic lives in the
+C file.  Nothing in the CUDA package imports this module, and this module
+imports nothing from it.
+"""
+from .binding import (  # noqa: F401
+    build,
+    lib_path,
+    num_threads,
+    set_num_threads,
+    bn_affine,
+    sign,
+    channel_abs_mean,
+    box_filter,
+    binarize_weights,
+    binconv_acc,
+    scale_output,
+    xnor_block,
+    shortcut_conv1x1,
+    speedup_model,
+    out_extent,
+)

@@ -1,0 +1,216 @@
+/*
+ * CPU oracle for the XNOR-Net binary-convolution forward block
+ * (BatchNorm affine -> BinActiv -> BinConv), arxiv 1603.05279.
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is the slow, plain, nested-loop
+ * statement of what the block computes, written from the paper's equations in
+ * +/-1 arithmetic: no bit packing, no popcount, no tiling, no fusion.  Only the
+ * test-suite, the smoke check and the CPU-baseline leg of the benchmark may
+ * call it; the CUDA library never does, and the two share no code.
+ *
+ * Conventions (one reading of each point the paper leaves open):
+ *   - tensors are dense row-major: x[N][C][H][W], w[Co][C][kh][kw],
+ *     out[N][Co][Ho][Wo], Ho = (H + 2*pad - kh)/stride + 1 (same for Wo);
+ *   - sign(v) = +1 when v >= 0 (so +0 and -0 give +1), else -1
+ *     (Section 3.1, the assignment below Eq. 4; used for inputs too);
+ *   - the BN affine is ONE fused multiply-add in fp32, y = fmaf(scale,x,shift);
+ *   - zero padding: a tap that falls outside the image contributes 0 to the
+ *     binary convolution and 0 to the box filter that makes K; the box filter
+ *     always divides by kh*kw (K = A * k with k_ij = 1/(w h), Section 3.2);
+ *   - real-valued sums (alpha, A, K, out) are accumulated in double and
+ *     rounded to float once; the +/-1 convolution is exact int32.
+ *
+ * The only parallelism is an OpenMP "parallel for" over independent outer
+ * indices (images, filters); loop bodies are unchanged by it.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+static int out_extent(int in, int k, int stride, int pad) {
+  return (in + 2 * pad - k) / stride + 1;
+}
+
+/* Block order B-A-C-P, Section 3.2 "Training XNOR-Networks": the input is
+ * normalised before it is binarised.  At inference BatchNorm is a per-channel
+ * affine map; scale and shift are inputs (folded by the caller).
+ * scale == NULL means identity (y = x). */
+void oracle_bn_affine(const float *x, const float *scale, const float *shift,
+                      int N, int C, int H, int W, float *y) {
+  const size_t hw = (size_t)H * W;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int c = 0; c < C; ++c) {
+      const float *xp = x + ((size_t)n * C + c) * hw;
+      float *yp = y + ((size_t)n * C + c) * hw;
+      for (size_t i = 0; i < hw; ++i)
+        yp[i] = scale ? fmaf(scale[c], xp[i], shift[c]) : xp[i];
+    }
+}
+
+/* sign() of Eq. 4 / Eq. 9: +1 for v >= 0, -1 otherwise, as int8. */
+void oracle_sign(const float *v, size_t count, int8_t *s) {
+#pragma omp parallel for schedule(static)
+  for (size_t i = 0; i < count; ++i) s[i] = (v[i] >= 0.0f) ? 1 : -1;
+}
+
+/* Section 3.2 "Binary Convolution": A = (sum over channels of |I|) / c,
+ * one value per spatial position of each image. */
+void oracle_channel_abs_mean(const float *y, int N, int C, int H, int W,
+                             float *A) {
+  const size_t hw = (size_t)H * W;
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (size_t i = 0; i < hw; ++i) {
+      double s = 0.0;
+      for (int c = 0; c < C; ++c) s += fabs((double)y[((size_t)n * C + c) * hw + i]);
+      A[(size_t)n * hw + i] = (float)(s / (double)C);
+    }
+}
+
+/* Section 3.2: K = A * k, k a kh x kw filter whose entries are all
+ * 1/(kh*kw); evaluated at the convolution's own output positions (same
+ * stride and zero padding), so K[n][oy][ox] is the scale beta of the input
+ * window that output (oy,ox) sees. */
+void oracle_box_filter(const float *A, int N, int H, int W, int kh, int kw,
+                       int stride, int pad, float *K) {
+  const int Ho = out_extent(H, kh, stride, pad), Wo = out_extent(W, kw, stride, pad);
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int oy = 0; oy < Ho; ++oy)
+      for (int ox = 0; ox < Wo; ++ox) {
+        double s = 0.0;
+        for (int ky = 0; ky < kh; ++ky)
+          for (int kx = 0; kx < kw; ++kx) {
+            const int iy = oy * stride + ky - pad, ix = ox * stride + kx - pad;
+            if (iy < 0 || iy >= H || ix < 0 || ix >= W) continue; /* pad adds 0 */
+            s += (double)A[((size_t)n * H + iy) * W + ix];
+          }
+        K[((size_t)n * Ho + oy) * Wo + ox] = (float)(s / (double)(kh * kw));
+      }
+}
+
+/* Eq. 4 and Eq. 6 (also Algorithm 1, the two assignments inside the filter
+ * loop): per filter, B = sign(W) and alpha = ||W||_1 / n, n = c*kh*kw. */
+void oracle_binarize_weights(const float *w, int Co, int C, int kh, int kw,
+                             int8_t *B, float *alpha) {
+  const size_t n = (size_t)C * kh * kw;
+#pragma omp parallel for schedule(static)
+  for (int co = 0; co < Co; ++co) {
+    double l1 = 0.0;
+    for (size_t i = 0; i < n; ++i) {
+      const float v = w[(size_t)co * n + i];
+      B[(size_t)co * n + i] = (v >= 0.0f) ? 1 : -1;
+      l1 += fabs((double)v);
+    }
+    alpha[co] = (float)(l1 / (double)n);
+  }
+}
+
+/* The binary convolution sign(I) (*) sign(W) of Eq. 11, written as the sum of
+ * products of +/-1 values that XNOR + bitcount evaluates (Section 3.2, first
+ * paragraph).  Taps outside the image add nothing. */
+void oracle_binconv_acc(const int8_t *Hs, const int8_t *B, int N, int C, int H,
+                        int W, int Co, int kh, int kw, int stride, int pad,
+                        int32_t *acc) {
+  const int Ho = out_extent(H, kh, stride, pad), Wo = out_extent(W, kw, stride, pad);
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < Co; ++co)
+      for (int oy = 0; oy < Ho; ++oy)
+        for (int ox = 0; ox < Wo; ++ox) {
+          int32_t s = 0;
+          for (int c = 0; c < C; ++c)
+            for (int ky = 0; ky < kh; ++ky)
+              for (int kx = 0; kx < kw; ++kx) {
+                const int iy = oy * stride + ky - pad, ix = ox * stride + kx - pad;
+                if (iy < 0 || iy >= H || ix < 0 || ix >= W) continue;
+                s += (int32_t)Hs[(((size_t)n * C + c) * H + iy) * W + ix] *
+                     (int32_t)B[(((size_t)co * C + c) * kh + ky) * kw + kx];
+              }
+          acc[(((size_t)n * Co + co) * Ho + oy) * Wo + ox] = s;
+        }
+}
+
+/* The "(.) K alpha" of Eq. 11: K is per image and position, shared by all
+ * filters; alpha is per filter.  residual (nullable) is added afterwards
+ * (ResNet shortcut). */
+void oracle_scale_output(const int32_t *acc, const float *K, const float *alpha,
+                         const float *residual, int N, int Co, int Ho, int Wo,
+                         float *out) {
+  const size_t hw = (size_t)Ho * Wo;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < Co; ++co)
+      for (size_t i = 0; i < hw; ++i) {
+        const size_t o = ((size_t)n * Co + co) * hw + i;
+        double v = (double)acc[o] * (double)K[(size_t)n * hw + i] * (double)alpha[co];
+        if (residual) v += (double)residual[o];
+        out[o] = (float)v;
+      }
+}
+
+/* Whole block in the paper's order: BN -> BinActiv (sign, A, K) -> BinConv.
+ * Every intermediate is returned so each can be compared on its own.
+ * Buffers (caller-allocated): y[N*C*H*W] float, Hs[N*C*H*W] int8,
+ * A[N*H*W], K[N*Ho*Wo], B[Co*C*kh*kw] int8, alpha[Co],
+ * acc[N*Co*Ho*Wo] int32, out[N*Co*Ho*Wo]. */
+void oracle_xnor_block(const float *x, const float *bn_scale, const float *bn_shift,
+                       const float *w, const float *residual, int N, int C, int H,
+                       int W, int Co, int kh, int kw, int stride, int pad,
+                       float *y, int8_t *Hs, float *A, float *K, int8_t *B,
+                       float *alpha, int32_t *acc, float *out) {
+  const int Ho = out_extent(H, kh, stride, pad), Wo = out_extent(W, kw, stride, pad);
+  oracle_bn_affine(x, bn_scale, bn_shift, N, C, H, W, y);
+  oracle_sign(y, (size_t)N * C * H * W, Hs);
+  oracle_channel_abs_mean(y, N, C, H, W, A);
+  oracle_box_filter(A, N, H, W, kh, kw, stride, pad, K);
+  oracle_binarize_weights(w, Co, C, kh, kw, B, alpha);
+  oracle_binconv_acc(Hs, B, N, C, H, W, Co, kh, kw, stride, pad, acc);
+  oracle_scale_output(acc, K, alpha, residual, N, Co, Ho, Wo, out);
+}
+
+/* Full-precision 1x1 strided convolution without bias: the projection
+ * shortcut ("type B") of the ResNet-18 variant in Section 4.2.  Plain
+ * definition, double accumulation. */
+void oracle_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H,
+                             int W, int Co, int stride, float *out) {
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < Co; ++co)
+      for (int oy = 0; oy < Ho; ++oy)
+        for (int ox = 0; ox < Wo; ++ox) {
+          double s = 0.0;
+          for (int c = 0; c < C; ++c)
+            s += (double)x[(((size_t)n * C + c) * H + (size_t)oy * stride) * W + (size_t)ox * stride] *
+                 (double)w[(size_t)co * C + c];
+          out[(((size_t)n * Co + co) * Ho + oy) * Wo + ox] = (float)s;
+        }
+}
+
+/* Section 4.1: with 64 binary operations per clock, the ratio of the cost of
+ * a standard convolution (c*N_W*N_I operations) to the binary one
+ * (c*N_W*N_I/64 + N_I) is S = 64 c N_W / (c N_W + 64). */
+double oracle_speedup_model(double c, double n_w) {
+  return 64.0 * c * n_w / (c * n_w + 64.0);
+}
