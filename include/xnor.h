@@ -1,0 +1,163 @@
+/*
+ * libxnor -- forward path of the XNOR-Net binary convolution block
+ * (BatchNorm affine -> BinActiv -> BinConv, arxiv 1603.05279) on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - Every data pointer is a DEVICE pointer owned by the caller; the library
+ *    allocates nothing and frees nothing.  Descriptor structs are read on the
+ *    host during the call and need not outlive it.
+ *  - Every pointer must be 16-byte aligned.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*,
+ *    NULL = the legacy default stream) and return without synchronising.
+ *    Outputs are fully overwritten.
+ *  - Errors are returned as xnor_status; nothing is printed, thrown or
+ *    aborted.  On any status other than XNOR_OK nothing was launched.
+ *  - Tensors are dense, row-major, fp32 unless stated:
+ *      activations  x  [N][C_in][H][W]               ("NCHW")
+ *      filters      w  [C_out][C_in][k_h][k_w]       (no bias; the paper
+ *                                                     assumes bias-free filters,
+ *                                                     footnote in Section 3)
+ *      output      out [N][C_out][H_out][W_out],
+ *      H_out = (H + 2*pad - k_h)/stride + 1, likewise W_out.
+ *  - sign(v) = +1 when v >= 0 (+0 and -0 included), -1 otherwise (the
+ *    assignment under Eq. 4, used for weights and inputs alike).  A set bit
+ *    means +1.
+ *  - Bit packing is along channels in 32-bit words: channel c is bit (c % 32)
+ *    of word (c / 32); Cw = ceil(C_in / 32) words per pixel or filter tap;
+ *    unused high bits of the last word are 0 in both operands.
+ *  - Zero padding: a filter tap that falls outside the image contributes 0 to
+ *    the binary convolution and 0 to the box filter that makes K.
+ */
+#ifndef XNOR_H_
+#define XNOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  XNOR_OK = 0,
+  XNOR_ERR_INVALID_ARG = 1, /* null/misaligned pointer, non-positive size, k > H + 2 pad ... */
+  XNOR_ERR_UNSUPPORTED = 2, /* a shape the kernels were not built for (see each call)       */
+  XNOR_ERR_CUDA = 3,        /* the launch failed; the CUDA error was read and cleared        */
+  XNOR_ERR_TIMEOUT = 4      /* a bounded device-side wait gave up (see xnor_device_status)   */
+} xnor_status;
+
+/* Geometry of one convolution layer.  Square or rectangular filters, one
+ * stride and one zero-padding amount for both axes, no groups, no dilation. */
+typedef struct {
+  int N, C_in, H, W;
+  int C_out, k_h, k_w;
+  int stride, pad;
+} xnor_conv_desc;
+
+/* Library version: major*10000 + minor*100 + patch. */
+int xnor_version(void);
+
+/* Static, human-readable name of a status code. */
+const char *xnor_status_string(xnor_status s);
+
+/* ceil(C_in / 32): 32-bit words per packed pixel or filter tap. */
+size_t xnor_words_per_pixel(int C_in);
+
+/* Output extent (in + 2*pad - k)/stride + 1, or 0 when the filter does not fit. */
+int xnor_out_extent(int in, int k, int stride, int pad);
+
+/*
+ * Weight binarisation -- Section 3.1, Eq. 4 and Eq. 6 (the two assignments in
+ * the filter loop of Algorithm 1): per filter, B = sign(W) and
+ * alpha = ||W||_1 / n with n = C_in*k_h*k_w.  Done once per layer at
+ * inference; the real-valued weights are not needed afterwards.
+ *
+ *   w         in   fp32 [C_out][C_in][k_h][k_w]
+ *   w_packed  out  u32  [C_out][k_h][k_w][Cw]   sign bits, channel-innermost
+ *   alpha     out  fp32 [C_out]
+ *
+ * INVALID_ARG: null or misaligned pointer, non-positive size.
+ * UNSUPPORTED: k_h*k_w*Cw > 12288 words per filter (does not fit the staging buffer).
+ */
+xnor_status xnor_binarize_weights(const float *w, int C_out, int C_in, int k_h, int k_w,
+                                  uint32_t *w_packed, float *alpha, void *cuda_stream);
+
+/*
+ * BatchNorm affine + BinActiv -- Section 3.2, "Binary Convolution" and the
+ * B-A-C-P block order of "Training XNOR-Networks": the input is normalised,
+ * then BinActiv produces sign(I) and the scaling map K = A * k, where
+ * A = (sum over channels of |I|)/c and k is the k_h x k_w filter with all
+ * entries 1/(k_h*k_w).
+ *
+ *   x         in   fp32 [N][C_in][H][W]
+ *   bn_scale  in   fp32 [C_in]  or NULL     y = fmaf(bn_scale[c], x, bn_shift[c]),
+ *   bn_shift  in   fp32 [C_in]  or NULL     one fused rounding; both NULL = identity
+ *   d         in   host pointer; C_out is ignored
+ *   x_packed  out  u32  [N][H][W][Cw]       bit = (y >= 0)
+ *   A         out  fp32 [N][H][W]           channel mean of |y|; also the scratch the
+ *                                           K kernel reads, so it must not be NULL
+ *   K         out  fp32 [N][H_out][W_out]   box filter of zero-padded A at the
+ *                                           convolution's own output positions, divisor
+ *                                           always k_h*k_w
+ *
+ * INVALID_ARG: null/misaligned pointer (bn_* may both be NULL, not just one),
+ * non-positive size, stride < 1, pad < 0, filter larger than the padded image.
+ */
+xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn_shift,
+                          const xnor_conv_desc *d, uint32_t *x_packed, float *A, float *K,
+                          void *cuda_stream);
+
+/*
+ * BinConv -- Eq. 11: out = (sign(I) (*) sign(W)) (.) K alpha, where (*) is the
+ * convolution evaluated with XNOR and bit-count (Section 3.2).  K is shared
+ * by all filters of the layer and differs per image; alpha is per filter.
+ *
+ *   x_packed  in   u32  [N][H][W][Cw]            from xnor_binactiv
+ *   w_packed  in   u32  [C_out][k_h][k_w][Cw]    from xnor_binarize_weights
+ *   alpha     in   fp32 [C_out]
+ *   K         in   fp32 [N][H_out][W_out]
+ *   residual  in   fp32 [N][C_out][H_out][W_out] or NULL; added after the scaling
+ *                  (ResNet shortcut); may be the same buffer as out
+ *   out       out  fp32 [N][C_out][H_out][W_out]
+ *   acc_out   out  i32  [N][C_out][H_out][W_out] or NULL; the exact integer result of
+ *                  sign(I) (*) sign(W) (sum over in-image taps of +-1 products), for
+ *                  verification
+ *
+ * INVALID_ARG as above.  UNSUPPORTED: k_h or k_w > 11, C_in*k_h*k_w >= 2^24
+ * (the integer result must be exact in fp32).
+ */
+xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_packed,
+                                const float *alpha, const float *K, const float *residual,
+                                const xnor_conv_desc *d, float *out, int32_t *acc_out,
+                                void *cuda_stream);
+
+/*
+ * Full-precision 1x1 strided convolution without bias: the projection
+ * shortcut ("type B") of the ResNet-18 variant the paper binarises
+ * (Section 4.2).  Its result is the `residual` of a block's second BinConv.
+ *
+ *   x    in   fp32 [N][C_in][H][W]
+ *   w    in   fp32 [C_out][C_in]
+ *   out  out  fp32 [N][C_out][(H-1)/stride+1][(W-1)/stride+1]
+ */
+xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,
+                                  int C_out, int stride, float *out, void *cuda_stream);
+
+/*
+ * Which BinConv engine xnor_conv2d_forward uses.  XNOR_ENGINE_AUTO (default)
+ * picks by shape.  Process-wide; meant for tests and measurements.
+ *   XNOR_ENGINE_POPC  CUDA-core XOR + population count, any supported shape
+ *   XNOR_ENGINE_UMMA  5th-generation tensor cores (+-1/0 int8 operands, exact
+ *                     int32 accumulation); UNSUPPORTED is returned by
+ *                     xnor_conv2d_forward for shapes this engine does not cover
+ */
+typedef enum { XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2 } xnor_engine;
+xnor_status xnor_set_engine(xnor_engine e);
+xnor_engine xnor_get_engine(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XNOR_H_ */

@@ -1,0 +1,185 @@
+"""ctypes binding of libxnor.so: argument marshalling only.
+
+Each function has the name and argument order of the C entry point it
+forwards to (see include/xnor.h) and takes torch CUDA tensors where the C call
+takes device pointers.  Nothing here computes: a missing or unloadable library
+raises, there is no fallback.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libxnor.so")
+
+XNOR_OK = 0
+XNOR_ERR_INVALID_ARG = 1
+XNOR_ERR_UNSUPPORTED = 2
+XNOR_ERR_CUDA = 3
+XNOR_ERR_TIMEOUT = 4
+
+XNOR_ENGINE_AUTO = 0
+XNOR_ENGINE_POPC = 1
+XNOR_ENGINE_UMMA = 2
+
+EXPORTS = [
+    "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
+    "xnor_binarize_weights", "xnor_binactiv", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
+    "xnor_set_engine", "xnor_get_engine",
+]
+
+
+class xnor_conv_desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("N", "C_in", "H", "W", "C_out", "k_h", "k_w", "stride", "pad")]
+
+
+class XnorError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__("%s returned %s" % (where, status_string(status)))
+
+
+_lib = None
+
+
+def load():
+    """Load libxnor.so (built in-tree by paper_1603_05279_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libxnor.so is not built: run `python -m paper_1603_05279_b200.build` "
+                          "(needs nvcc); there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    lib.xnor_version.restype = ci
+    lib.xnor_status_string.restype = ctypes.c_char_p
+    lib.xnor_status_string.argtypes = [ci]
+    lib.xnor_words_per_pixel.restype = ctypes.c_size_t
+    lib.xnor_words_per_pixel.argtypes = [ci]
+    lib.xnor_out_extent.restype = ci
+    lib.xnor_out_extent.argtypes = [ci] * 4
+    lib.xnor_binarize_weights.restype = ci
+    lib.xnor_binarize_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
+    lib.xnor_binactiv.restype = ci
+    lib.xnor_binactiv.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp, vp, vp]
+    lib.xnor_conv2d_forward.restype = ci
+    lib.xnor_conv2d_forward.argtypes = [vp, vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc),
+                                        vp, vp, vp]
+    lib.xnor_shortcut_conv1x1.restype = ci
+    lib.xnor_shortcut_conv1x1.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, vp, vp]
+    lib.xnor_set_engine.restype = ci
+    lib.xnor_set_engine.argtypes = [ci]
+    lib.xnor_get_engine.restype = ci
+    _lib = lib
+    return lib
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("libxnor takes device pointers: tensor is on %s" % t.device)
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("expected %s, got %s" % (dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(status, where):
+    if status != XNOR_OK:
+        raise XnorError(status, where)
+
+
+def make_desc(N, C_in, H, W, C_out, k_h, k_w, stride, pad):
+    return xnor_conv_desc(N, C_in, H, W, C_out, k_h, k_w, stride, pad)
+
+
+def desc_of(s):
+    """xnor_conv_desc of a workloads.ConvShape."""
+    return xnor_conv_desc(s.N, s.C_in, s.H, s.W, s.C_out, s.k, s.k, s.stride, s.pad)
+
+
+def xnor_version():
+    return int(load().xnor_version())
+
+
+def status_string(status):
+    return load().xnor_status_string(int(status)).decode()
+
+
+def xnor_words_per_pixel(C_in):
+    return int(load().xnor_words_per_pixel(int(C_in)))
+
+
+def xnor_out_extent(n, k, stride, pad):
+    return int(load().xnor_out_extent(int(n), int(k), int(stride), int(pad)))
+
+
+def xnor_set_engine(engine):
+    _check(load().xnor_set_engine(int(engine)), "xnor_set_engine")
+
+
+def xnor_get_engine():
+    return int(load().xnor_get_engine())
+
+
+def xnor_binarize_weights(w, w_packed, alpha, stream=None):
+    C_out, C_in, k_h, k_w = w.shape
+    _check(load().xnor_binarize_weights(_ptr(w, torch.float32), C_out, C_in, k_h, k_w,
+                                        _ptr(w_packed, torch.int32), _ptr(alpha, torch.float32),
+                                        _stream(stream)), "xnor_binarize_weights")
+
+
+def xnor_binactiv(x, bn_scale, bn_shift, d, x_packed, A, K, stream=None):
+    _check(load().xnor_binactiv(_ptr(x, torch.float32), _ptr(bn_scale, torch.float32),
+                                _ptr(bn_shift, torch.float32), ctypes.byref(d),
+                                _ptr(x_packed, torch.int32), _ptr(A, torch.float32),
+                                _ptr(K, torch.float32), _stream(stream)), "xnor_binactiv")
+
+
+def xnor_conv2d_forward(x_packed, w_packed, alpha, K, residual, d, out, acc_out=None, stream=None):
+    _check(load().xnor_conv2d_forward(_ptr(x_packed, torch.int32), _ptr(w_packed, torch.int32),
+                                      _ptr(alpha, torch.float32), _ptr(K, torch.float32),
+                                      _ptr(residual, torch.float32), ctypes.byref(d),
+                                      _ptr(out, torch.float32), _ptr(acc_out, torch.int32),
+                                      _stream(stream)), "xnor_conv2d_forward")
+
+
+def xnor_shortcut_conv1x1(x, w, stride, out, stream=None):
+    N, C_in, H, W = x.shape
+    C_out = w.shape[0]
+    _check(load().xnor_shortcut_conv1x1(_ptr(x, torch.float32), _ptr(w, torch.float32), N, C_in,
+                                        H, W, C_out, int(stride), _ptr(out, torch.float32),
+                                        _stream(stream)), "xnor_shortcut_conv1x1")
+
+
+# ---- buffer helpers (allocation only; torch owns the memory) -------------------------------
+def alloc_weights(C_out, C_in, k_h, k_w, device="cuda"):
+    Cw = (C_in + 31) // 32
+    return (torch.empty((C_out, k_h, k_w, Cw), dtype=torch.int32, device=device),
+            torch.empty((C_out,), dtype=torch.float32, device=device))
+
+
+def alloc_binactiv(d, device="cuda"):
+    Cw = (d.C_in + 31) // 32
+    Ho = (d.H + 2 * d.pad - d.k_h) // d.stride + 1
+    Wo = (d.W + 2 * d.pad - d.k_w) // d.stride + 1
+    return (torch.empty((d.N, d.H, d.W, Cw), dtype=torch.int32, device=device),
+            torch.empty((d.N, d.H, d.W), dtype=torch.float32, device=device),
+            torch.empty((d.N, Ho, Wo), dtype=torch.float32, device=device))
+
+
+def alloc_out(d, dtype=torch.float32, device="cuda"):
+    Ho = (d.H + 2 * d.pad - d.k_h) // d.stride + 1
+    Wo = (d.W + 2 * d.pad - d.k_w) // d.stride + 1
+    return torch.empty((d.N, d.C_out, Ho, Wo), dtype=dtype, device=device)

@@ -1,0 +1,105 @@
+// C-ABI entry points of libxnor: argument checks and dispatch.  No kernel code.
+#include "common.cuh"
+
+namespace {
+
+xnor_engine g_engine = XNOR_ENGINE_AUTO;
+
+inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+inline bool bad_ptr(const void *p) { return p == nullptr || misaligned(p); }
+
+xnor_status check_desc(const xnor_conv_desc *d, bool need_cout) {
+  if (!d) return XNOR_ERR_INVALID_ARG;
+  if (d->N <= 0 || d->C_in <= 0 || d->H <= 0 || d->W <= 0 || d->k_h <= 0 || d->k_w <= 0)
+    return XNOR_ERR_INVALID_ARG;
+  if (need_cout && d->C_out <= 0) return XNOR_ERR_INVALID_ARG;
+  if (d->stride < 1 || d->pad < 0) return XNOR_ERR_INVALID_ARG;
+  if (d->k_h > d->H + 2 * d->pad || d->k_w > d->W + 2 * d->pad) return XNOR_ERR_INVALID_ARG;
+  return XNOR_OK;
+}
+
+xnor_status from_cuda(cudaError_t e) { return e == cudaSuccess ? XNOR_OK : XNOR_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int xnor_version(void) { return 100; }
+
+const char *xnor_status_string(xnor_status s) {
+  switch (s) {
+    case XNOR_OK: return "XNOR_OK";
+    case XNOR_ERR_INVALID_ARG: return "XNOR_ERR_INVALID_ARG";
+    case XNOR_ERR_UNSUPPORTED: return "XNOR_ERR_UNSUPPORTED";
+    case XNOR_ERR_CUDA: return "XNOR_ERR_CUDA";
+    case XNOR_ERR_TIMEOUT: return "XNOR_ERR_TIMEOUT";
+  }
+  return "XNOR_ERR_UNKNOWN";
+}
+
+size_t xnor_words_per_pixel(int C_in) { return C_in > 0 ? (size_t)(C_in + 31) / 32 : 0; }
+
+int xnor_out_extent(int in, int k, int stride, int pad) {
+  if (in <= 0 || k <= 0 || stride < 1 || pad < 0 || k > in + 2 * pad) return 0;
+  return (in + 2 * pad - k) / stride + 1;
+}
+
+xnor_status xnor_set_engine(xnor_engine e) {
+  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC && e != XNOR_ENGINE_UMMA)
+    return XNOR_ERR_INVALID_ARG;
+  g_engine = e;
+  return XNOR_OK;
+}
+
+xnor_engine xnor_get_engine(void) { return g_engine; }
+
+xnor_status xnor_binarize_weights(const float *w, int C_out, int C_in, int k_h, int k_w,
+                                  uint32_t *w_packed, float *alpha, void *cuda_stream) {
+  if (bad_ptr(w) || bad_ptr(w_packed) || bad_ptr(alpha)) return XNOR_ERR_INVALID_ARG;
+  if (C_out <= 0 || C_in <= 0 || k_h <= 0 || k_w <= 0) return XNOR_ERR_INVALID_ARG;
+  if ((long long)k_h * k_w * ((C_in + 31) / 32) > 12288) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_binarize_weights(w, C_out, C_in, k_h, k_w, w_packed, alpha,
+                                                 (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn_shift,
+                          const xnor_conv_desc *d, uint32_t *x_packed, float *A, float *K,
+                          void *cuda_stream) {
+  xnor_status s = check_desc(d, false);
+  if (s != XNOR_OK) return s;
+  if (bad_ptr(x) || bad_ptr(x_packed) || bad_ptr(A) || bad_ptr(K)) return XNOR_ERR_INVALID_ARG;
+  if ((bn_scale == nullptr) != (bn_shift == nullptr)) return XNOR_ERR_INVALID_ARG;
+  if (bn_scale && (misaligned(bn_scale) || misaligned(bn_shift))) return XNOR_ERR_INVALID_ARG;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  return from_cuda(xnor::launch_binactiv(x, bn_scale, bn_shift, g, x_packed, A, K,
+                                         (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_packed,
+                                const float *alpha, const float *K, const float *residual,
+                                const xnor_conv_desc *d, float *out, int32_t *acc_out,
+                                void *cuda_stream) {
+  xnor_status s = check_desc(d, true);
+  if (s != XNOR_OK) return s;
+  if (bad_ptr(x_packed) || bad_ptr(w_packed) || bad_ptr(alpha) || bad_ptr(K) || bad_ptr(out))
+    return XNOR_ERR_INVALID_ARG;
+  if ((residual && misaligned(residual)) || (acc_out && misaligned(acc_out)))
+    return XNOR_ERR_INVALID_ARG;
+  if (d->k_h > 11 || d->k_w > 11) return XNOR_ERR_UNSUPPORTED;
+  if ((long long)d->C_in * d->k_h * d->k_w >= (1LL << 24)) return XNOR_ERR_UNSUPPORTED;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  if (g_engine == XNOR_ENGINE_UMMA) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, out,
+                                             acc_out, (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,
+                                  int C_out, int stride, float *out, void *cuda_stream) {
+  if (bad_ptr(x) || bad_ptr(w) || bad_ptr(out)) return XNOR_ERR_INVALID_ARG;
+  if (N <= 0 || C_in <= 0 || H <= 0 || W <= 0 || C_out <= 0 || stride < 1)
+    return XNOR_ERR_INVALID_ARG;
+  return from_cuda(xnor::launch_shortcut_conv1x1(x, w, N, C_in, H, W, C_out, stride, out,
+                                                 (cudaStream_t)cuda_stream));
+}
+
+}  // extern "C"

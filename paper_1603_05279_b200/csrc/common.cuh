@@ -1,0 +1,36 @@
+// Shared declarations of the CUDA translation units of libxnor (internal).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "xnor.h"
+
+namespace xnor {
+
+struct ConvGeom {
+  int N, C, H, W, Co, kh, kw, stride, pad, Ho, Wo, Cw;
+};
+
+inline ConvGeom make_geom(const xnor_conv_desc &d) {
+  ConvGeom g;
+  g.N = d.N; g.C = d.C_in; g.H = d.H; g.W = d.W; g.Co = d.C_out;
+  g.kh = d.k_h; g.kw = d.k_w; g.stride = d.stride; g.pad = d.pad;
+  g.Ho = (d.H + 2 * d.pad - d.k_h) / d.stride + 1;
+  g.Wo = (d.W + 2 * d.pad - d.k_w) / d.stride + 1;
+  g.Cw = (d.C_in + 31) / 32;
+  return g;
+}
+
+// Launchers: return the cudaError_t of the launch (cudaGetLastError, cleared).
+cudaError_t launch_binarize_weights(const float *w, int Co, int C, int kh, int kw,
+                                    uint32_t *w_packed, float *alpha, cudaStream_t st);
+cudaError_t launch_binactiv(const float *x, const float *scale, const float *shift,
+                            const ConvGeom &g, uint32_t *x_packed, float *A, float *K,
+                            cudaStream_t st);
+cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                                const float *K, const float *residual, const ConvGeom &g,
+                                float *out, int32_t *acc_out, cudaStream_t st);
+cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,
+                                    int Co, int stride, float *out, cudaStream_t st);
+
+}  // namespace xnor

@@ -1,0 +1,42 @@
+"""Helpers shared by the GPU parity tests (no arithmetic of the method)."""
+import numpy as np
+import torch
+
+REL_TOL = 1e-5   # fp32 outputs: max |gpu - oracle| <= REL_TOL * max |oracle|
+
+
+def unpack_bits(words, C):
+    """u32/i32 words [..., Cw] -> +-1 int8 [..., C]; also checks the tail bits are 0."""
+    w = np.ascontiguousarray(words).view(np.uint32)
+    Cw = w.shape[-1]
+    bits = ((w[..., :, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(*w.shape[:-1], Cw * 32)
+    assert not bits[..., C:].any(), "tail bits of the last word must be 0"
+    return np.where(bits[..., :C] == 1, 1, -1).astype(np.int8)
+
+
+def unpack_activations(x_packed, C):
+    """[N][H][W][Cw] words -> +-1 [N][C][H][W]."""
+    return np.ascontiguousarray(unpack_bits(x_packed, C).transpose(0, 3, 1, 2))
+
+
+def unpack_weights(w_packed, C):
+    """[Co][kh][kw][Cw] words -> +-1 [Co][C][kh][kw]."""
+    return np.ascontiguousarray(unpack_bits(w_packed, C).transpose(0, 3, 1, 2))
+
+
+def assert_close(gpu, ref, what, rel=REL_TOL):
+    gpu = np.asarray(gpu, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert gpu.shape == ref.shape, (what, gpu.shape, ref.shape)
+    scale = np.abs(ref).max() if ref.size else 0.0
+    err = np.abs(gpu - ref).max() if ref.size else 0.0
+    assert err <= rel * scale + 1e-30, "%s: max abs err %.3e > %.1e * max|ref| (%.3e)" % (
+        what, err, rel, scale)
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def host(t):
+    return t.detach().cpu().numpy()
