@@ -45,7 +45,7 @@ typedef enum {
   XNOR_ERR_INVALID_ARG = 1, /* null/misaligned pointer, non-positive size, k > H + 2 pad ... */
   XNOR_ERR_UNSUPPORTED = 2, /* a shape the kernels were not built for (see each call)       */
   XNOR_ERR_CUDA = 3,        /* the launch failed; the CUDA error was read and cleared        */
-  XNOR_ERR_TIMEOUT = 4      /* a bounded device-side wait gave up (see xnor_device_status)   */
+  XNOR_ERR_TIMEOUT = 4      /* a bounded device-side wait gave up (see xnor_check_device)    */
 } xnor_status;
 
 /* Geometry of one convolution layer.  Square or rectangular filters, one
@@ -156,6 +156,16 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
 typedef enum { XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2 } xnor_engine;
 xnor_status xnor_set_engine(xnor_engine e);
 xnor_engine xnor_get_engine(void);
+
+/*
+ * The one call that synchronises: waits for `cuda_stream`, then reads the
+ * device-side status word.  Every wait inside the tensor-core kernel (on a
+ * shared-memory barrier) is bounded; a wait that expires records
+ * XNOR_ERR_TIMEOUT there, the kernel stops issuing work, releases its tensor
+ * memory and returns, and the outputs of that launch are undefined.  Returns
+ * XNOR_OK, XNOR_ERR_TIMEOUT (the word is then cleared) or XNOR_ERR_CUDA.
+ */
+xnor_status xnor_check_device(void *cuda_stream);
 
 #ifdef __cplusplus
 }

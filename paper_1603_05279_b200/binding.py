@@ -26,7 +26,7 @@ XNOR_ENGINE_UMMA = 2
 EXPORTS = [
     "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
     "xnor_binarize_weights", "xnor_binactiv", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
-    "xnor_set_engine", "xnor_get_engine",
+    "xnor_set_engine", "xnor_get_engine", "xnor_check_device",
 ]
 
 
@@ -73,6 +73,8 @@ def load():
     lib.xnor_set_engine.restype = ci
     lib.xnor_set_engine.argtypes = [ci]
     lib.xnor_get_engine.restype = ci
+    lib.xnor_check_device.restype = ci
+    lib.xnor_check_device.argtypes = [vp]
     _lib = lib
     return lib
 
@@ -131,6 +133,11 @@ def xnor_set_engine(engine):
 
 def xnor_get_engine():
     return int(load().xnor_get_engine())
+
+
+def xnor_check_device(stream=None):
+    """Synchronises the stream and raises XnorError if a device-side wait expired."""
+    _check(load().xnor_check_device(_stream(stream)), "xnor_check_device")
 
 
 def xnor_binarize_weights(w, w_packed, alpha, stream=None):

@@ -88,9 +88,22 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
   if (d->k_h > 11 || d->k_w > 11) return XNOR_ERR_UNSUPPORTED;
   if ((long long)d->C_in * d->k_h * d->k_w >= (1LL << 24)) return XNOR_ERR_UNSUPPORTED;
   const xnor::ConvGeom g = xnor::make_geom(*d);
-  if (g_engine == XNOR_ENGINE_UMMA) return XNOR_ERR_UNSUPPORTED;
+  const bool umma_ok = xnor::umma_supported(g);
+  if (g_engine == XNOR_ENGINE_UMMA && !umma_ok) return XNOR_ERR_UNSUPPORTED;
+  if (g_engine != XNOR_ENGINE_POPC && umma_ok)
+    return from_cuda(xnor::launch_binconv_umma(x_packed, w_packed, alpha, K, residual, g, out,
+                                               acc_out, (cudaStream_t)cuda_stream));
   return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, out,
                                              acc_out, (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_check_device(void *cuda_stream) {
+  int st = 0;
+  if (xnor::read_device_status(&st, (cudaStream_t)cuda_stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return XNOR_ERR_CUDA;
+  }
+  return st == 0 ? XNOR_OK : XNOR_ERR_TIMEOUT;
 }
 
 xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,

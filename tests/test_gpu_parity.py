@@ -12,7 +12,7 @@ from util import REL_TOL, assert_close, dev, host, unpack_activations, unpack_we
 
 pytestmark = pytest.mark.gpu
 
-ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_AUTO]
+ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_AUTO]
 
 
 def rng(seed):
@@ -44,6 +44,7 @@ def gpu_block(x, w, stride, pad, scale=None, shift=None, residual=None, engine=B
         X.xnor_conv2d_forward(xp, wp, alpha, K, res, d, out, acc)
     finally:
         X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
+    X.xnor_check_device()
     torch.cuda.synchronize()
     return dict(wp=host(wp), alpha=host(alpha), xp=host(xp), A=host(A), K=host(K),
                 out=host(out), acc=host(acc))
@@ -90,6 +91,11 @@ def test_block_parity(oracle, shape, engine):
     g = rng(sum(shape))
     x = g.standard_normal((N, C, H, W)).astype(np.float32)
     w = g.standard_normal((Co, C, kh, kw)).astype(np.float32)
+    if engine == B.XNOR_ENGINE_UMMA and s != 1:
+        with pytest.raises(X.XnorError) as e:       # the tensor-core engine covers stride 1
+            gpu_block(x, w, s, p, engine=engine)
+        assert e.value.status == B.XNOR_ERR_UNSUPPORTED
+        return
     check_block(oracle, x, w, s, p, engine=engine)
 
 
@@ -169,6 +175,7 @@ def _run_layer_full(s, seed, engine=B.XNOR_ENGINE_AUTO):
         X.xnor_conv2d_forward(xp, wp, alpha, K, None, d, out, acc)
     finally:
         X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
+    X.xnor_check_device()
     torch.cuda.synchronize()
     return x, w, out, acc, K
 
