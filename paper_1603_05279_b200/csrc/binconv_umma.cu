@@ -30,6 +30,12 @@
 namespace xnor {
 
 __device__ int g_device_status = 0;
+#ifdef XNOR_TRACE
+__device__ long long g_trace[64];
+#define TRACE(i) do { if (blockIdx.x == gridDim.x / 2 && blockIdx.y == 0) g_trace[i] = clock64(); } while (0)
+#else
+#define TRACE(i) do {} while (0)
+#endif
 
 namespace {
 
@@ -38,7 +44,11 @@ constexpr int kProducers = 32 * kProducerWarps;
 constexpr int kThreads = 32 + kProducers;
 constexpr int kTileM = 128;
 constexpr int kMaxStages = 6;
+constexpr int kMaxWps = 4;       // channel words per weight stage (one MMA of K = 32 each)
+constexpr int kPrefetch = 4;     // weight stages whose packed words are in flight
+constexpr int kMaxChunkWords = 16;  // channel words of the patch resident at a time, upper bound
 constexpr long long kWaitCycles = 1ll << 31;   // about a second
+constexpr size_t kCtrlBytes = 256;
 
 struct UmmaParams {
   const uint32_t *xp, *wp;
@@ -129,14 +139,32 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                ::"r"(bar) : "memory");
 }
 
-// 32 sign bits -> 32 bytes of +1 (0x01) / -1 (0xFF).  Register j holds the
-// channels j, j+8, j+16, j+24 of the word (the K order is the same for both
-// operands, so any fixed permutation is fine).
-__device__ __forceinline__ void expand_word(uint32_t w, uint32_t v[8]) {
+// Operand encodings.  Bit j of every byte of a packed word (channels j, j+8,
+// j+16, j+24) lands in register j of the 32 expanded bytes; both operands use
+// the same order, so the K order is consistent.
+//
+// Weights take ONE logic op per register: byte = beta * 2^j (beta = sign bit,
+// 0 or 1) for j = 0..6 is just `w & (0x01010101 << j)`; bit 7 is moved down to
+// beta * 64.  Activations carry the compensating power of two and the sign:
+// byte = a * 2^(6-j) (a = +-1; 0 for padding and for the channel tail), and
+// a * 1 for j = 7.  Every product is 64 * a * beta, so the tensor core returns
+// D = 64 * sum(a * beta).  With sign(W) = 2 beta - 1 the wanted sum is
+//   sum(a * sign(W)) = D / 32 - S,   S = sum of a over the window,
+// and S is a box sum of per-pixel values (2 popcount - channels) that the
+// activation expansion leaves in shared memory.  All of it is exact integer
+// arithmetic (|D| <= 64 * C_in * k_h * k_w < 2^31).
+__device__ __forceinline__ void expand_weights(uint32_t w, uint32_t v[8]) {
+#pragma unroll
+  for (int j = 0; j < 7; ++j) v[j] = w & (0x01010101u << j);
+  v[7] = (w >> 1) & 0x40404040u;
+}
+
+__device__ __forceinline__ void expand_activations(uint32_t w, uint32_t v[8]) {
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const uint32_t t = (w >> j) & 0x01010101u;
-    v[j] = 0xFFFFFFFFu - 0xFEu * t;
+    const uint32_t sc = j < 7 ? (64u >> j) : 1u;                // |byte value|
+    const uint32_t t = (w >> j) & 0x01010101u;                  // sign bit per byte
+    v[j] = (256u - sc) * 0x01010101u - t * (256u - 2u * sc);    // bit ? +sc : -sc, no borrows
   }
 }
 
@@ -146,6 +174,8 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
                "r"(d) : "memory");
 }
 
+// Asynchronous load of 16 accumulator columns (one value per lane and column);
+// the registers are valid only after tmem_wait16 on the same array.
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t r[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -154,15 +184,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t r[16]) {
         "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
         "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Waits for every tcgen05.ld of this thread; the array is an in/out operand so
+// that no use of it can be scheduled above the wait.
+__device__ __forceinline__ void tmem_wait16(int32_t r[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]),
+                 "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]),
+                 "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
+
+// NT_CT: filters per CTA when known at compile time (0 = read P.NT); WPS: channel
+// words per weight stage.  Both only remove address arithmetic and predicates.
+template <int NT_CT, int WPS>
 __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int taps = P.kh * P.kw;
+  const int NT = NT_CT ? NT_CT : P.NT;
   const uint32_t patch_bytes = (uint32_t)(2 * P.cwc) * P.ppix * 16u;
-  const uint32_t stage_bytes = (uint32_t)(2 * P.wps) * P.NT * 16u;
+  const uint32_t stage_bytes = (uint32_t)(2 * WPS) * NT * 16u;
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t patch_addr = smem_base;
   const uint32_t stage_addr = patch_addr + patch_bytes;
@@ -171,18 +214,20 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
   // bars: [0,S) full, [S,2S) empty, 2S patch_full, 2S+1 patch_free, 2S+2 accum_full
   const uint32_t bar0 = smem_u32(bars);
   const int S = P.stages;
-  auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
   const uint32_t patch_full = bar0 + 8u * (2 * S), patch_free = patch_full + 8u,
                  accum_full = patch_full + 16u;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kMaxStages + 4);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  int *pix_sum = reinterpret_cast<int *>(ctrl + kCtrlBytes);   // [ppix] sum over channels of a
+  float *alpha_sm = reinterpret_cast<float *>(pix_sum + P.ppix);  // [NT], 16-byte aligned
 
+  if (tid == 0) TRACE(0);
+  for (int q = tid; q < P.ppix; q += kThreads) pix_sum[q] = 0;
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < S; ++s) {
-        mbar_init(full_bar(s), kProducerWarps);
-        mbar_init(empty_bar(s), 1);
+        mbar_init(bar0 + 8u * s, kProducerWarps);
+        mbar_init(bar0 + 8u * (S + s), 1);
       }
       mbar_init(patch_full, kProducerWarps);
       mbar_init(patch_free, 1);
@@ -199,54 +244,63 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (tid == 0) TRACE(1);
 
-  const long long m0 = (long long)blockIdx.x * kTileM;
-  const int co0 = blockIdx.y * P.NT;
+  const uint32_t m0 = blockIdx.x * (uint32_t)kTileM;
+  const int co0 = blockIdx.y * NT;
   const int nchunks = (P.Cw + P.cwc - 1) / P.cwc;
+  const uint32_t a_lbo = (uint32_t)P.ppix * 16u, b_lbo = (uint32_t)NT * 16u;
 
   if (warp == 0) {
     // ------------------------------------------------------------ MMA issuer
-    uint32_t it = 0, accumulate = 0;
+    uint32_t accumulate = 0, ph = 0;
+    int s = 0;
     bool ok = true;
     for (int cc = 0; cc < nchunks && ok; ++cc) {
       const int cwn = min(P.cwc, P.Cw - cc * P.cwc);
       ok = mbar_wait(patch_full, cc & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
+      if (lane == 0) TRACE(2);
+      int kx = 0;
+      uint32_t a_tap = patch_addr;                       // + (ky*Wp + kx) * 16
       for (int tap = 0; tap < taps && ok; ++tap) {
-        const int ky = tap / P.kw, kx = tap - ky * P.kw;
-        const uint32_t a_tap = patch_addr + (uint32_t)(ky * P.Wp + kx) * 16u;
-        for (int wb = 0; wb < cwn; wb += P.wps, ++it) {
-          const int nw = min(P.wps, cwn - wb);
-          const int s = it % S;
-          ok = mbar_wait(full_bar(s), (it / S) & 1, abort_flag);
+        for (int wb = 0; wb < cwn; wb += WPS) {
+          const int nw = min(WPS, cwn - wb);
+          ok = mbar_wait(bar0 + 8u * s, ph, abort_flag);
           if (!ok) break;
           tc_fence_after();
           if (lane == 0) {
+            uint32_t a_addr = a_tap + (uint32_t)(2 * wb) * a_lbo;
+            uint32_t b_addr = stage_addr + s * stage_bytes;
             for (int wi = 0; wi < nw; ++wi) {
-              const uint64_t ad = make_desc(a_tap + (uint32_t)(2 * (wb + wi)) * P.ppix * 16u,
-                                            (uint32_t)P.ppix * 16u, 128u);
-              const uint64_t bd = make_desc(stage_addr + s * stage_bytes +
-                                                (uint32_t)(2 * wi) * P.NT * 16u,
-                                            (uint32_t)P.NT * 16u, 128u);
-              umma_i8(tmem_base, ad, bd, P.idesc, accumulate);
+              umma_i8(tmem_base, make_desc(a_addr, a_lbo, 128u), make_desc(b_addr, b_lbo, 128u),
+                      P.idesc, accumulate);
               accumulate = 1;
+              a_addr += 2u * a_lbo;
+              b_addr += 2u * b_lbo;
             }
-            umma_commit(empty_bar(s));
+            umma_commit(bar0 + 8u * (S + s));
           }
           __syncwarp();
+          if (++s == S) { s = 0; ph ^= 1u; }
         }
+        if (++kx == P.kw) { kx = 0; a_tap += (uint32_t)(P.Wp - P.kw + 1) * 16u; }
+        else a_tap += 16u;
       }
       if (ok && lane == 0) umma_commit(patch_free);
       __syncwarp();
     }
     if (ok && lane == 0) umma_commit(accum_full);
+    if (lane == 0) TRACE(3);
     __syncwarp();
   } else {
     // ------------------------------------------------------------ producers
     const int pt = tid - 32;
-    uint32_t it = 0;
+    uint32_t ph = 1;          // parity to wait for on the empty barriers
+    int s = 0;
     bool ok = true;
+    const int crem = P.C - 32 * (P.Cw - 1);
     for (int cc = 0; cc < nchunks && ok; ++cc) {
       const int cw0 = cc * P.cwc;
       const int cwn = min(P.cwc, P.Cw - cw0);
@@ -254,129 +308,267 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
         ok = mbar_wait(patch_free, (cc - 1) & 1, abort_flag);
         if (!ok) break;
       }
-      // expand the activation patch: item = (word wl, stream pixel q), q fastest
-      for (int item = pt; item < P.ppix * cwn; item += kProducers) {
-        const int wl = item / P.ppix, q = item - wl * P.ppix;
-        const long long sq = m0 + q;
-        uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-        if (sq < P.L) {
-          const long long r = sq / P.Wp;
-          const int c = (int)(sq - r * P.Wp);
-          const long long n = r / P.Hp;
-          const int ry = (int)(r - n * P.Hp);
-          if (c >= P.pad && ry >= P.pad) {
-            const int cw = cw0 + wl;
-            const uint32_t w = __ldg(P.xp + (((size_t)n * P.H + (ry - P.pad)) * P.W + (c - P.pad)) *
-                                                P.Cw + cw);
-            expand_word(w, v);
-            if (cw == P.Cw - 1 && P.tail_mask != 0xFFFFFFFFu) {
+      // expand the activation patch: one thread per stream pixel, all channel words of
+      // the chunk; every global load is issued before the first expansion
+      if (cc == 0)
+        for (int i = pt; i < NT; i += kProducers)
+          alpha_sm[i] = co0 + i < P.Co ? __ldg(P.alpha + co0 + i) : 0.0f;
+      for (int q = pt; q < P.ppix; q += kProducers) {
+        const uint32_t sq = m0 + (uint32_t)q;
+        const uint32_t *src = nullptr;
+        if (sq < (uint32_t)P.L) {
+          const uint32_t r = sq / (uint32_t)P.Wp;
+          const int c = (int)(sq - r * (uint32_t)P.Wp);
+          const uint32_t n = r / (uint32_t)P.Hp;
+          const int ry = (int)(r - n * (uint32_t)P.Hp);
+          if (c >= P.pad && ry >= P.pad)
+            src = P.xp + (((size_t)n * P.H + (ry - P.pad)) * P.W + (c - P.pad)) * P.Cw + cw0;
+        }
+        uint32_t pw[kMaxChunkWords];
 #pragma unroll
-              for (int j = 0; j < 8; ++j) v[j] &= ((P.tail_mask >> j) & 0x01010101u) * 0xFFu;
+        for (int wl = 0; wl < kMaxChunkWords; ++wl)
+          pw[wl] = (src != nullptr && wl < cwn) ? __ldg(src + wl) : 0u;
+        int psum = 0;
+        uint32_t a = patch_addr + (uint32_t)q * 16u;
+#pragma unroll
+        for (int wl = 0; wl < kMaxChunkWords; ++wl) {
+          if (wl < cwn) {
+            uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+            if (src != nullptr) {
+              expand_activations(pw[wl], v);
+              int nreal = 32;
+              if (cw0 + wl == P.Cw - 1 && crem != 32) {
+                nreal = crem;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] &= ((P.tail_mask >> j) & 0x01010101u) * 0xFFu;
+              }
+              psum += 2 * __popc(pw[wl]) - nreal;
             }
+            sts128(a, v[0], v[1], v[2], v[3]);
+            sts128(a + a_lbo, v[4], v[5], v[6], v[7]);
+            a += 2u * a_lbo;
           }
         }
-        const uint32_t a = patch_addr + (uint32_t)(2 * wl) * P.ppix * 16u + (uint32_t)q * 16u;
-        sts128(a, v[0], v[1], v[2], v[3]);
-        sts128(a + (uint32_t)P.ppix * 16u, v[4], v[5], v[6], v[7]);
+        pix_sum[q] += psum;
       }
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(patch_full);
+      if (pt == 0) TRACE(8);
 
-      for (int tap = 0; tap < taps && ok; ++tap) {
-        for (int wb = 0; wb < cwn; wb += P.wps, ++it) {
-          const int nw = min(P.wps, cwn - wb);
-          const int s = it % S;
-          ok = mbar_wait(empty_bar(s), ((it / S) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          if (pt < P.NT) {
-            const int co = co0 + pt;
-            const uint32_t *src = P.wp + ((size_t)co * taps + tap) * P.Cw + cw0 + wb;
-            const uint32_t dst = stage_addr + s * stage_bytes + (uint32_t)pt * 16u;
-            for (int wi = 0; wi < nw; ++wi) {
-              uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-              if (co < P.Co) expand_word(__ldg(src + wi), v);
-              const uint32_t a = dst + (uint32_t)(2 * wi) * P.NT * 16u;
-              sts128(a, v[0], v[1], v[2], v[3]);
-              sts128(a + (uint32_t)P.NT * 16u, v[4], v[5], v[6], v[7]);
+      // weight stages of this chunk in the issuer's order (tap outer, words inner).
+      // kPrefetch register sets hold the packed words of the next stages; a set is
+      // refilled right after it is expanded, so a load has kPrefetch stages to land.
+      const int co = co0 + pt;
+      const bool row_live = pt < NT && co < P.Co;
+      const uint32_t *f_ptr = P.wp + (size_t)(row_live ? co : 0) * taps * P.Cw + cw0;
+      int f_wb = 0, f_tap = row_live ? 0 : taps;     // dead rows never fetch
+      uint32_t pf[kPrefetch][WPS];
+      auto fetch = [&](uint32_t dst[WPS]) {
+        if (f_tap < taps) {
+#pragma unroll
+          for (int wi = 0; wi < WPS; ++wi) dst[wi] = f_wb + wi < cwn ? __ldg(f_ptr + f_wb + wi) : 0u;
+          f_wb += WPS;
+          if (f_wb >= cwn) { f_wb = 0; ++f_tap; f_ptr += P.Cw; }
+        } else {
+#pragma unroll
+          for (int wi = 0; wi < WPS; ++wi) dst[wi] = 0u;
+        }
+      };
+#pragma unroll
+      for (int d = 0; d < kPrefetch; ++d) fetch(pf[d]);
+      const uint32_t row_addr = stage_addr + (uint32_t)pt * 16u;
+      int tap = 0, wb = 0;
+      while (tap < taps && ok) {
+#pragma unroll
+        for (int d = 0; d < kPrefetch; ++d) {
+          if (tap < taps && ok) {
+            ok = mbar_wait(bar0 + 8u * (S + s), ph, abort_flag);
+            if (ok) {
+              if (pt < NT) {
+                const uint32_t a = row_addr + s * stage_bytes;
+                const int nw = cwn - wb;           // >= WPS except in a ragged last stage
+#pragma unroll
+                for (int wi = 0; wi < WPS; ++wi) {
+                  if (wi == 0 || wi < nw) {
+                    uint32_t v[8];
+                    expand_weights(pf[d][wi], v);      // 0 for rows beyond C_out
+                    sts128(a + (uint32_t)(2 * wi) * b_lbo, v[0], v[1], v[2], v[3]);
+                    sts128(a + (uint32_t)(2 * wi + 1) * b_lbo, v[4], v[5], v[6], v[7]);
+                  }
+                }
+              }
+              fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar0 + 8u * s);
+              if (++s == S) { s = 0; ph ^= 1u; }
+              wb += WPS;
+              if (wb >= cwn) { wb = 0; ++tap; }
+              fetch(pf[d]);
             }
           }
-          fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(full_bar(s));
         }
       }
     }
     // ------------------------------------------------------------ epilogue
+    if (pt == 0) TRACE(9);
     if (ok) ok = mbar_wait(accum_full, 0, abort_flag);
+    if (pt == 0) TRACE(10);
     if (ok) {
       tc_fence_after();
       const int quarter = warp & 3;              // TMEM lanes 32*quarter .. +31
       const int half = (warp - 1) >> 2;          // which half of the column blocks
-      const int nblk = P.NT / 16;
+      const int nblk = NT / 16;
       const int b_begin = half == 0 ? 0 : (nblk + 1) / 2;
       const int b_end = half == 0 ? (nblk + 1) / 2 : nblk;
-      const long long m = m0 + quarter * 32 + lane;
-      bool valid = m < P.L;
-      long long n = 0;
+      const int lm = quarter * 32 + lane;
+      const uint32_t m = m0 + (uint32_t)lm;
+      bool valid = m < (uint32_t)P.L;
+      uint32_t n = 0;
       int oy = 0, ox = 0;
       if (valid) {
-        const long long r = m / P.Wp;
-        ox = (int)(m - r * P.Wp);
-        n = r / P.Hp;
-        oy = (int)(r - n * P.Hp);
+        const uint32_t r = m / (uint32_t)P.Wp;
+        ox = (int)(m - r * (uint32_t)P.Wp);
+        n = r / (uint32_t)P.Hp;
+        oy = (int)(r - n * (uint32_t)P.Hp);
         valid = ox < P.Wo && oy < P.Ho;
+      }
+      int wsum = 0;                               // S: sum of a over the window of pixel m
+      if (valid) {
+        for (int ky = 0; ky < P.kh; ++ky)
+          for (int kx = 0; kx < P.kw; ++kx) wsum += pix_sum[lm + ky * P.Wp + kx];
       }
       const size_t HoWo = (size_t)P.Ho * P.Wo;
       const size_t pix = (size_t)oy * P.Wo + ox;
-      const float kv = valid ? __ldg(P.K + (size_t)n * HoWo + pix) : 0.0f;
-      for (int b = b_begin; b < b_end; ++b) {
-        int32_t r[16];
-        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 16), r);
+      // out = (D/32 - S) * K * alpha, evaluated as float(D - 32 S) * (K/32) * alpha: the
+      // power-of-two factors move exactly, and |D - 32 S| < 2^24 so the conversion is exact
+      const float kvs = valid ? __ldg(P.K + (size_t)n * HoWo + pix) * 0.03125f : 0.0f;
+      const int wsum32 = wsum * 32;
+      const size_t o0 = ((size_t)n * P.Co + co0 + b_begin * 16) * HoWo + pix;
+      float *optr = P.out + o0;
+      const bool plain = P.residual == nullptr && P.acc_out == nullptr;
+      const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      auto emit = [&](int b, const int32_t r[16]) {
         if (valid) {
+          if (plain && co0 + b * 16 + 16 <= P.Co) {
+            float *p = optr;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int co = co0 + b * 16 + j;
-            if (co < P.Co) {
-              const size_t o = ((size_t)n * P.Co + co) * HoWo + pix;
-              float v = __fmul_rn(__fmul_rn((float)r[j], kv), __ldg(P.alpha + co));
-              if (P.residual) v += P.residual[o];
-              P.out[o] = v;
-              if (P.acc_out) P.acc_out[o] = r[j];
+            for (int j4 = 0; j4 < 4; ++j4) {
+              const float4 al = *reinterpret_cast<const float4 *>(alpha_sm + b * 16 + j4 * 4);
+              const float a4[4] = {al.x, al.y, al.z, al.w};
+#pragma unroll
+              for (int jj = 0; jj < 4; ++jj) {
+                *p = __fmul_rn(__fmul_rn((float)(r[j4 * 4 + jj] - wsum32), kvs), a4[jj]);
+                p += HoWo;
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int co = co0 + b * 16 + j;
+              if (co < P.Co) {
+                const size_t o = (size_t)(optr - P.out) + (size_t)j * HoWo;
+                float v = __fmul_rn(__fmul_rn((float)(r[j] - wsum32), kvs), alpha_sm[b * 16 + j]);
+                if (P.residual) v += P.residual[o];
+                P.out[o] = v;
+                if (P.acc_out) P.acc_out[o] = (r[j] - wsum32) >> 5;
+              }
             }
           }
+          optr += 16 * HoWo;
+        }
+      };
+      // two register sets: the load of the next 16 columns is in flight while the
+      // current 16 are scaled and stored
+      int32_t ra[16], rb[16];
+      if (b_begin < b_end) {
+        tmem_ld16(t_lane + (uint32_t)(b_begin * 16), ra);
+        tmem_wait16(ra);
+      }
+      for (int b = b_begin; b < b_end; b += 2) {
+        if (b + 1 < b_end) tmem_ld16(t_lane + (uint32_t)((b + 1) * 16), rb);
+        emit(b, ra);
+        if (b + 1 < b_end) {
+          tmem_wait16(rb);
+          if (b + 2 < b_end) tmem_ld16(t_lane + (uint32_t)((b + 2) * 16), ra);
+          emit(b + 1, rb);
+          if (b + 2 < b_end) tmem_wait16(ra);
         }
       }
     }
   }
+  if (tid == 32) TRACE(11);
   tc_fence_before();
   __syncthreads();
+  if (tid == 0) TRACE(4);
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                  ::"r"(tmem_base), "r"((uint32_t)P.tmem_cols) : "memory");
   }
 }
 
-constexpr size_t kSmemBudget = 110 * 1024;   // two CTAs per SM
-constexpr size_t kCtrlBytes = 256;
+constexpr size_t kSmemBudget = 115000;   // two CTAs per SM
+
+struct Plan {
+  int ppix, NT, ntiles, tmem_cols, cwc, wps, stages;
+  size_t smem;
+  bool ok;
+};
+
+Plan make_plan(const ConvGeom &g) {
+  Plan p{};
+  p.ok = false;
+  if (g.stride != 1) return p;
+  const int Wp = g.W + g.pad, Hp = g.H + g.pad;
+  if ((long long)g.N * Hp * Wp >= (1ll << 31) - kTileM) return p;
+  const int halo = (g.kh - 1) * Wp + g.kw - 1;
+  p.ppix = (kTileM + halo + 7) / 8 * 8;
+  if ((size_t)p.ppix * 16 >= (1u << 18)) return p;
+  p.ntiles = (g.Co + 255) / 256;
+  p.NT = (((g.Co + p.ntiles - 1) / p.ntiles) + 15) / 16 * 16;
+  p.tmem_cols = 32;
+  while (p.tmem_cols < p.NT) p.tmem_cols *= 2;
+  const size_t fixed = kCtrlBytes + (size_t)p.ppix * sizeof(int) + (size_t)p.NT * sizeof(float);
+  const size_t word_bytes = (size_t)p.ppix * 32;            // patch bytes per channel word
+  const size_t max_patch_words = kMaxChunkWords;
+  // whole channel range resident: pick the stage width that needs the fewest stage steps
+  long best_steps = -1;
+  if ((size_t)g.Cw <= max_patch_words) {
+    for (int wps = kMaxWps; wps >= 1; --wps) {
+      const size_t stage_bytes = (size_t)2 * wps * p.NT * 16;
+      if (fixed + word_bytes * g.Cw + 3 * stage_bytes > kSmemBudget) continue;
+      int stages = (int)((kSmemBudget - fixed - word_bytes * g.Cw) / stage_bytes);
+      if (stages > kMaxStages) stages = kMaxStages;
+      // stage steps per tap, with a small penalty per barrier round trip
+      const long steps = (g.Cw + wps - 1) / wps * (long)(wps * 4 + 1);
+      if (best_steps < 0 || steps < best_steps) {
+        best_steps = steps; p.wps = wps; p.stages = stages; p.cwc = g.Cw;
+      }
+    }
+  }
+  if (best_steps < 0) {   // chunk the channels: 3 stages of 2 words, the rest for the patch
+    p.wps = 2; p.stages = 3;
+    const size_t stage_bytes = (size_t)2 * p.wps * p.NT * 16;
+    if (fixed + 3 * stage_bytes + word_bytes > kSmemBudget) return p;
+    size_t cwc = (kSmemBudget - fixed - 3 * stage_bytes) / word_bytes;
+    if (cwc > max_patch_words) cwc = max_patch_words;
+    if (cwc > (size_t)g.Cw) cwc = g.Cw;
+    p.cwc = (int)cwc;
+  }
+  p.smem = (size_t)p.cwc * word_bytes + (size_t)p.stages * 2 * p.wps * p.NT * 16 + fixed;
+  p.ok = true;
+  return p;
+}
 
 }  // namespace
 
-bool umma_supported(const ConvGeom &g) {
-  if (g.stride != 1) return false;
-  const int Wp = g.W + g.pad;
-  const int halo = (g.kh - 1) * Wp + g.kw - 1;
-  const int ppix = (kTileM + halo + 7) / 8 * 8;
-  // one channel word of patch plus two minimal weight stages must fit
-  const size_t need = (size_t)ppix * 32 + 2 * (size_t)256 * 32 + kCtrlBytes;
-  if (need > kSmemBudget) return false;
-  if ((size_t)ppix * 16 >= (1u << 18)) return false;
-  return true;
-}
+bool umma_supported(const ConvGeom &g) { return make_plan(g).ok; }
 
 cudaError_t launch_binconv_umma(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st) {
+  const Plan pl = make_plan(g);
+  if (!pl.ok) return cudaErrorInvalidValue;
   UmmaParams P;
   P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
   P.out = out; P.acc_out = acc_out;
@@ -384,47 +576,42 @@ cudaError_t launch_binconv_umma(const uint32_t *xp, const uint32_t *wp, const fl
   P.pad = g.pad; P.Ho = g.Ho; P.Wo = g.Wo; P.Cw = g.Cw;
   P.Hp = g.H + g.pad; P.Wp = g.W + g.pad;
   P.L = (long long)g.N * P.Hp * P.Wp;
-  const int halo = (g.kh - 1) * P.Wp + g.kw - 1;
-  P.ppix = (kTileM + halo + 7) / 8 * 8;
-  const int ntiles = (g.Co + 255) / 256;
-  P.NT = (((g.Co + ntiles - 1) / ntiles) + 15) / 16 * 16;
-  P.tmem_cols = 32;
-  while (P.tmem_cols < P.NT) P.tmem_cols *= 2;
-  P.wps = 2;
-  const size_t stage_bytes = (size_t)2 * P.wps * P.NT * 16;
-  const size_t word_bytes = (size_t)P.ppix * 32;   // patch bytes per channel word
-  int stages = 4, cwc = 0;
-  for (; stages >= 2; --stages) {
-    const size_t left = kSmemBudget - kCtrlBytes - stages * stage_bytes;
-    cwc = (int)(left / word_bytes);
-    if (cwc >= g.Cw) break;
-  }
-  if (stages < 2) {   // the whole channel range does not fit: chunk it, keep 3 stages
-    stages = 3;
-    cwc = (int)((kSmemBudget - kCtrlBytes - stages * stage_bytes) / word_bytes);
-  }
-  if (cwc > g.Cw) cwc = g.Cw;
-  if (cwc < 1) return cudaErrorInvalidValue;
-  P.cwc = cwc;
-  P.stages = stages;
+  P.ppix = pl.ppix; P.NT = pl.NT; P.tmem_cols = pl.tmem_cols;
+  P.cwc = pl.cwc; P.wps = pl.wps; P.stages = pl.stages;
   P.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.NT >> 3) << 17) |
             ((uint32_t)(kTileM >> 4) << 24);
   const int crem = g.C - 32 * (g.Cw - 1);
   P.tail_mask = crem == 32 ? 0xFFFFFFFFu : ((1u << crem) - 1u);
-  const size_t smem = (size_t)2 * cwc * P.ppix * 16 + stages * stage_bytes + kCtrlBytes;
+  using KernelFn = void (*)(const UmmaParams);
+  static const KernelFn table[5][kMaxWps] = {
+#define XNOR_ROW(NT) {binconv_umma_kernel<NT, 1>, binconv_umma_kernel<NT, 2>, \
+                      binconv_umma_kernel<NT, 3>, binconv_umma_kernel<NT, 4>}
+      XNOR_ROW(0), XNOR_ROW(64), XNOR_ROW(128), XNOR_ROW(192), XNOR_ROW(256)
+#undef XNOR_ROW
+  };
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(binconv_umma_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmemBudget);
-    if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
+    for (int i = 0; i < 5; ++i)
+      for (int j = 0; j < kMaxWps; ++j) {
+        cudaError_t e = cudaFuncSetAttribute(table[i][j],
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemBudget);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
+      }
     attr_set = true;
   }
+  const int row = (P.NT % 64 == 0) ? P.NT / 64 : 0;
   const long long mtiles = (P.L + kTileM - 1) / kTileM;
-  const dim3 grid((unsigned)mtiles, (unsigned)ntiles);
-  binconv_umma_kernel<<<grid, kThreads, smem, st>>>(P);
+  const dim3 grid((unsigned)mtiles, (unsigned)pl.ntiles);
+  table[row][P.wps - 1]<<<grid, kThreads, pl.smem, st>>>(P);
   return cudaGetLastError();
 }
+
+#ifdef XNOR_TRACE
+extern "C" int xnor_debug_trace(long long *host64) {
+  return (int)cudaMemcpyFromSymbol(host64, g_trace, sizeof(long long) * 64);
+}
+#endif
 
 cudaError_t read_device_status(int *status, cudaStream_t st) {
   cudaError_t e = cudaStreamSynchronize(st);
