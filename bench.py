@@ -195,7 +195,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     X.load()
-    X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2}[args.engine])
+    X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2, "umma_i8": 3}[args.engine])
     stream = torch.cuda.current_stream()
 
     # ---- synthetic inputs: every rank has its own batch of 256 (weak scaling, no exchange)
@@ -377,7 +377,7 @@ def main():
     ap.add_argument("--ref-images", type=int, default=8,
                     help="images per layer per step of the reference (oracle) arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_i8"])
     ap.add_argument("--layers", default="0,1,2,3",
                     help="subset of the four layers (profiling runs only; the bench line is the "
                          "default: all four)")

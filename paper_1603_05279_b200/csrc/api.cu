@@ -45,7 +45,8 @@ int xnor_out_extent(int in, int k, int stride, int pad) {
 }
 
 xnor_status xnor_set_engine(xnor_engine e) {
-  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC && e != XNOR_ENGINE_UMMA)
+  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC && e != XNOR_ENGINE_UMMA &&
+      e != XNOR_ENGINE_UMMA_I8)
     return XNOR_ERR_INVALID_ARG;
   g_engine = e;
   return XNOR_OK;
@@ -88,22 +89,29 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
   if (d->k_h > 11 || d->k_w > 11) return XNOR_ERR_UNSUPPORTED;
   if ((long long)d->C_in * d->k_h * d->k_w >= (1LL << 24)) return XNOR_ERR_UNSUPPORTED;
   const xnor::ConvGeom g = xnor::make_geom(*d);
-  const bool umma_ok = xnor::umma_supported(g);
-  if (g_engine == XNOR_ENGINE_UMMA && !umma_ok) return XNOR_ERR_UNSUPPORTED;
-  if (g_engine != XNOR_ENGINE_POPC && umma_ok)
-    return from_cuda(xnor::launch_binconv_umma(x_packed, w_packed, alpha, K, residual, g, out,
-                                               acc_out, (cudaStream_t)cuda_stream));
+  const cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (g_engine == XNOR_ENGINE_UMMA_I8) {
+    if (!xnor::umma_i8_supported(g)) return XNOR_ERR_UNSUPPORTED;
+    return from_cuda(xnor::launch_binconv_i8(x_packed, w_packed, alpha, K, residual, g, out,
+                                             acc_out, st));
+  }
+  const bool fp4_ok = xnor::umma_fp4_supported(g);
+  if (g_engine == XNOR_ENGINE_UMMA && !fp4_ok) return XNOR_ERR_UNSUPPORTED;
+  if (g_engine != XNOR_ENGINE_POPC && fp4_ok)
+    return from_cuda(xnor::launch_binconv_fp4(x_packed, w_packed, alpha, K, residual, g, out,
+                                              acc_out, st));
   return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, out,
                                              acc_out, (cudaStream_t)cuda_stream));
 }
 
 xnor_status xnor_check_device(void *cuda_stream) {
-  int st = 0;
-  if (xnor::read_device_status(&st, (cudaStream_t)cuda_stream) != cudaSuccess) {
+  int s4 = 0, s8 = 0;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess ||
+      xnor::read_status_fp4(&s4) != cudaSuccess || xnor::read_status_i8(&s8) != cudaSuccess) {
     (void)cudaGetLastError();
     return XNOR_ERR_CUDA;
   }
-  return st == 0 ? XNOR_OK : XNOR_ERR_TIMEOUT;
+  return (s4 == 0 && s8 == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
 }
 
 xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,

@@ -1,4 +1,6 @@
-// BinConv on the 5th-generation tensor cores (Eq. 11).
+// BinConv on the 5th-generation tensor cores with int8 operands (Eq. 11).
+// Kept beside the fp4 kernel as the measured alternative: same structure, half
+// the tensor-core rate and twice the shared-memory bytes per 1-bit MAC.
 //
 // sign(I) (*) sign(W) is an exact integer contraction, so it runs as an
 // implicit GEMM with +-1/0 int8 operands and int32 accumulators in tensor
@@ -26,18 +28,15 @@
 // Every wait is bounded: on expiry the CTA records XNOR_ERR_TIMEOUT in a
 // device status word, stops issuing work, frees its tensor memory and exits.
 #include "common.cuh"
+#include "umma_common.cuh"
 
 namespace xnor {
 
-__device__ int g_device_status = 0;
-#ifdef XNOR_TRACE
-__device__ long long g_trace[64];
-#define TRACE(i) do { if (blockIdx.x == gridDim.x / 2 && blockIdx.y == 0) g_trace[i] = clock64(); } while (0)
-#else
-#define TRACE(i) do {} while (0)
-#endif
+__device__ int g_status_i8 = 0;
 
 namespace {
+
+using namespace umma;
 
 constexpr int kProducerWarps = 8;
 constexpr int kProducers = 32 * kProducerWarps;
@@ -47,7 +46,6 @@ constexpr int kMaxStages = 6;
 constexpr int kMaxWps = 4;       // channel words per weight stage (one MMA of K = 32 each)
 constexpr int kPrefetch = 4;     // weight stages whose packed words are in flight
 constexpr int kMaxChunkWords = 16;  // channel words of the patch resident at a time, upper bound
-constexpr long long kWaitCycles = 1ll << 31;   // about a second
 constexpr size_t kCtrlBytes = 256;
 
 struct UmmaParams {
@@ -67,64 +65,6 @@ struct UmmaParams {
   uint32_t tail_mask;  // bits of real channels in the last word (all ones if C % 32 == 0)
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false when the wait expired or another thread of the
-// CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 64; ++i)
-      if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
-      *abort_flag = 1;
-      atomicExch(&g_device_status, (int)XNOR_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-
-__device__ __forceinline__ void fence_proxy_async() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_before() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_after() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor, no swizzle, K-major: 8-row x 16-byte core
-// matrices; lbo = byte distance between the two core matrices along K, sbo =
-// byte distance between 8-row groups.
-__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) |
-         ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
-}
-
 __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
                                         uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -132,11 +72,6 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-               ::"r"(bar) : "memory");
 }
 
 // Operand encodings.  Bit j of every byte of a packed word (channels j, j+8,
@@ -168,38 +103,10 @@ __device__ __forceinline__ void expand_activations(uint32_t w, uint32_t v[8]) {
   }
 }
 
-__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c,
-                                       uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c),
-               "r"(d) : "memory");
-}
-
-// Asynchronous load of 16 accumulator columns (one value per lane and column);
-// the registers are valid only after tmem_wait16 on the same array.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t r[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-}
-
-// Waits for every tcgen05.ld of this thread; the array is an in/out operand so
-// that no use of it can be scheduled above the wait.
-__device__ __forceinline__ void tmem_wait16(int32_t r[16]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]),
-                 "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]),
-                 "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :: "memory");
-}
-
 // NT_CT: filters per CTA when known at compile time (0 = read P.NT); WPS: channel
 // words per weight stage.  Both only remove address arithmetic and predicates.
 template <int NT_CT, int WPS>
-__global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaParams P) {
+__global__ void __launch_bounds__(kThreads, 2) binconv_i8_kernel(const UmmaParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int taps = P.kh * P.kw;
@@ -221,7 +128,6 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
   int *pix_sum = reinterpret_cast<int *>(ctrl + kCtrlBytes);   // [ppix] sum over channels of a
   float *alpha_sm = reinterpret_cast<float *>(pix_sum + P.ppix);  // [NT], 16-byte aligned
 
-  if (tid == 0) TRACE(0);
   for (int q = tid; q < P.ppix; q += kThreads) pix_sum[q] = 0;
   if (warp == 0) {
     if (lane == 0) {
@@ -244,7 +150,6 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (tid == 0) TRACE(1);
 
   const uint32_t m0 = blockIdx.x * (uint32_t)kTileM;
   const int co0 = blockIdx.y * NT;
@@ -258,16 +163,15 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
     bool ok = true;
     for (int cc = 0; cc < nchunks && ok; ++cc) {
       const int cwn = min(P.cwc, P.Cw - cc * P.cwc);
-      ok = mbar_wait(patch_full, cc & 1, abort_flag);
+      ok = mbar_wait(patch_full, cc & 1, abort_flag, &g_status_i8);
       if (!ok) break;
       tc_fence_after();
-      if (lane == 0) TRACE(2);
       int kx = 0;
       uint32_t a_tap = patch_addr;                       // + (ky*Wp + kx) * 16
       for (int tap = 0; tap < taps && ok; ++tap) {
         for (int wb = 0; wb < cwn; wb += WPS) {
           const int nw = min(WPS, cwn - wb);
-          ok = mbar_wait(bar0 + 8u * s, ph, abort_flag);
+          ok = mbar_wait(bar0 + 8u * s, ph, abort_flag, &g_status_i8);
           if (!ok) break;
           tc_fence_after();
           if (lane == 0) {
@@ -292,7 +196,6 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
       __syncwarp();
     }
     if (ok && lane == 0) umma_commit(accum_full);
-    if (lane == 0) TRACE(3);
     __syncwarp();
   } else {
     // ------------------------------------------------------------ producers
@@ -305,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
       const int cw0 = cc * P.cwc;
       const int cwn = min(P.cwc, P.Cw - cw0);
       if (cc > 0) {
-        ok = mbar_wait(patch_free, (cc - 1) & 1, abort_flag);
+        ok = mbar_wait(patch_free, (cc - 1) & 1, abort_flag, &g_status_i8);
         if (!ok) break;
       }
       // expand the activation patch: one thread per stream pixel, all channel words of
@@ -354,7 +257,6 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
       fence_proxy_async();
       __syncwarp();
       if (lane == 0) mbar_arrive(patch_full);
-      if (pt == 0) TRACE(8);
 
       // weight stages of this chunk in the issuer's order (tap outer, words inner).
       // kPrefetch register sets hold the packed words of the next stages; a set is
@@ -383,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
 #pragma unroll
         for (int d = 0; d < kPrefetch; ++d) {
           if (tap < taps && ok) {
-            ok = mbar_wait(bar0 + 8u * (S + s), ph, abort_flag);
+            ok = mbar_wait(bar0 + 8u * (S + s), ph, abort_flag, &g_status_i8);
             if (ok) {
               if (pt < NT) {
                 const uint32_t a = row_addr + s * stage_bytes;
@@ -411,9 +313,7 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
       }
     }
     // ------------------------------------------------------------ epilogue
-    if (pt == 0) TRACE(9);
-    if (ok) ok = mbar_wait(accum_full, 0, abort_flag);
-    if (pt == 0) TRACE(10);
+    if (ok) ok = mbar_wait(accum_full, 0, abort_flag, &g_status_i8);
     if (ok) {
       tc_fence_after();
       const int quarter = warp & 3;              // TMEM lanes 32*quarter .. +31
@@ -497,10 +397,8 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_umma_kernel(const UmmaPar
       }
     }
   }
-  if (tid == 32) TRACE(11);
   tc_fence_before();
   __syncthreads();
-  if (tid == 0) TRACE(4);
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                  ::"r"(tmem_base), "r"((uint32_t)P.tmem_cols) : "memory");
@@ -562,9 +460,9 @@ Plan make_plan(const ConvGeom &g) {
 
 }  // namespace
 
-bool umma_supported(const ConvGeom &g) { return make_plan(g).ok; }
+bool umma_i8_supported(const ConvGeom &g) { return make_plan(g).ok; }
 
-cudaError_t launch_binconv_umma(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+cudaError_t launch_binconv_i8(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st) {
   const Plan pl = make_plan(g);
@@ -584,8 +482,8 @@ cudaError_t launch_binconv_umma(const uint32_t *xp, const uint32_t *wp, const fl
   P.tail_mask = crem == 32 ? 0xFFFFFFFFu : ((1u << crem) - 1u);
   using KernelFn = void (*)(const UmmaParams);
   static const KernelFn table[5][kMaxWps] = {
-#define XNOR_ROW(NT) {binconv_umma_kernel<NT, 1>, binconv_umma_kernel<NT, 2>, \
-                      binconv_umma_kernel<NT, 3>, binconv_umma_kernel<NT, 4>}
+#define XNOR_ROW(NT) {binconv_i8_kernel<NT, 1>, binconv_i8_kernel<NT, 2>, \
+                      binconv_i8_kernel<NT, 3>, binconv_i8_kernel<NT, 4>}
       XNOR_ROW(0), XNOR_ROW(64), XNOR_ROW(128), XNOR_ROW(192), XNOR_ROW(256)
 #undef XNOR_ROW
   };
@@ -607,20 +505,11 @@ cudaError_t launch_binconv_umma(const uint32_t *xp, const uint32_t *wp, const fl
   return cudaGetLastError();
 }
 
-#ifdef XNOR_TRACE
-extern "C" int xnor_debug_trace(long long *host64) {
-  return (int)cudaMemcpyFromSymbol(host64, g_trace, sizeof(long long) * 64);
-}
-#endif
-
-cudaError_t read_device_status(int *status, cudaStream_t st) {
-  cudaError_t e = cudaStreamSynchronize(st);
-  if (e != cudaSuccess) return e;
-  e = cudaMemcpyFromSymbol(status, g_device_status, sizeof(int));
-  if (e != cudaSuccess) return e;
-  if (*status != 0) {
+cudaError_t read_status_i8(int *status) {
+  cudaError_t e = cudaMemcpyFromSymbol(status, g_status_i8, sizeof(int));
+  if (e == cudaSuccess && *status != 0) {
     const int zero = 0;
-    e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+    e = cudaMemcpyToSymbol(g_status_i8, &zero, sizeof(int));
   }
   return e;
 }

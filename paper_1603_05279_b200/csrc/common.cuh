@@ -30,12 +30,18 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st);
-bool umma_supported(const ConvGeom &g);
-cudaError_t launch_binconv_umma(const uint32_t *xp, const uint32_t *wp, const float *alpha,
-                                const float *K, const float *residual, const ConvGeom &g,
-                                float *out, int32_t *acc_out, cudaStream_t st);
-// Synchronises st, then reads (and clears if set) the device status word.
-cudaError_t read_device_status(int *status, cudaStream_t st);
+// Tensor-core engines (stride 1): 4-bit operands (default) and int8 operands.
+bool umma_fp4_supported(const ConvGeom &g);
+cudaError_t launch_binconv_fp4(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                               const float *K, const float *residual, const ConvGeom &g,
+                               float *out, int32_t *acc_out, cudaStream_t st);
+bool umma_i8_supported(const ConvGeom &g);
+cudaError_t launch_binconv_i8(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                              const float *K, const float *residual, const ConvGeom &g,
+                              float *out, int32_t *acc_out, cudaStream_t st);
+// Read (and clear if set) the device status word of each tensor-core kernel.
+cudaError_t read_status_fp4(int *status);
+cudaError_t read_status_i8(int *status);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,
                                     int Co, int stride, float *out, cudaStream_t st);
 
