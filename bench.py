@@ -311,19 +311,22 @@ def run_ours(args):
     if engine == "auto":
         engine = "umma" if all(s.stride == 1 for s in shapes) else "mixed"
     if engine != "popc":
-        # int8 tensor-core peak = measured bf16 peak x 2 (nominal int8 : bf16 ratio); the
-        # sustained figure, because the kernel is timed inside a long step
-        roofline = {"kernel": "binconv_umma_kernel (4 launches per step)", "bound": "tensor",
+        # tensor-core peak for the operand type in use = measured bf16 peak x the nominal
+        # ratio of that type to bf16 (e2m1: 9 / 2.25 = 4, int8: 2); the sustained figure,
+        # because the kernel is timed inside a long step.  2 flops per 1-bit MAC.
+        ratio, kind = (2, "int8") if engine == "umma_i8" else (4, "e2m1 (fp4)")
+        roofline = {"kernel": "BinConv tensor-core kernel (one launch per layer, %d per step)"
+                              % len(layers), "bound": "tensor",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12,
-                    "peak": 2 * peaks["bf16_sustained"], "unit": "TOP/s (2 ops per 1-bit MAC)",
-                    "peak_source": "2 x %s sustained bf16 TFLOP/s (int8:bf16 nominal ratio 2)"
-                                   % peaks["source"], "traffic": None}
+                    "peak": ratio * peaks["bf16_sustained"], "unit": "TFLOP/s",
+                    "peak_source": "%d x %s sustained bf16 TFLOP/s (nominal %s : bf16 ratio)"
+                                   % (ratio, peaks["source"], kind), "traffic": None}
     else:
         clk = (clocks["sm_mhz"] or 1965.0) * 1e6
         peak = POPC_PER_CLK_PER_SM * 32 * props.multi_processor_count * clk * 2 / 1e12
         roofline = {"kernel": "binconv_popc_kernel (4 launches per step)", "bound": "alu",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12, "peak": peak,
-                    "unit": "TOP/s (2 ops per 1-bit MAC)",
+                    "unit": "TFLOP/s",
                     "peak_source": "derived: 16 popc/clk/SM x 32 bits x %d SMs x median SM clock "
                                    "during the run" % props.multi_processor_count,
                     "traffic": None}
@@ -344,7 +347,10 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": ("u32 bit words (XOR+popcount), int32 sums, fp32 scaling" if engine == "popc"
-                  else "int8 +-1/0 tensor-core operands from 1-bit words, int32 sums, fp32 scaling"),
+                  else "int8 +-1/0 tensor-core operands from 1-bit words, int32 sums, fp32 scaling"
+                  if engine == "umma_i8"
+                  else "e2m1 (fp4) tensor-core operands from 1-bit words, exact integer sums in "
+                       "fp32, fp32 scaling"),
         "data": "synthetic",
         "config": {"workload": WORKLOAD if full else "subset of " + WORKLOAD,
                    "layers": [s.name for s in shapes],
