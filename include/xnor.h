@@ -110,6 +110,39 @@ xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn
                           void *cuda_stream);
 
 /*
+ * xnor_binactiv without a caller-supplied A buffer.  (The paper has no
+ * counterpart; this exists for callers that cannot allocate.)
+ *
+ * xnor_binactiv needs N*H*W floats of device memory for the A plane, which the
+ * box filter reads back to make K.  Some callers have no way to provide it:
+ * code that runs where cudaMalloc is not permitted (inside a real-time or
+ * pre-planned memory budget, in a plug-in that is handed its input and output
+ * buffers and nothing else), or that only needs x_packed and K and has no use
+ * for A.  For them this entry point keeps A in a fixed array inside the library:
+ * XNOR_BINACTIV_STATIC_MAX_PIXELS floats (4 MiB) of device memory, held by
+ * every GPU that has loaded the library until the process exits.  The call
+ * allocates nothing and frees nothing, directly or through any other library.
+ *
+ *   x, bn_scale, bn_shift, d, x_packed, K   exactly as for xnor_binactiv; the
+ *                                           results are bit-identical to it
+ *
+ * UNSUPPORTED: N*H*W > XNOR_BINACTIV_STATIC_MAX_PIXELS (nothing is launched;
+ * split the batch or use xnor_binactiv).  INVALID_ARG as for xnor_binactiv.
+ *
+ * The first call on each device looks up the array's device address (with
+ * that device current); make that first call outside any stream capture.
+ * All calls on one device share the one array: two calls whose kernels can
+ * overlap on the GPU (different streams without an ordering between them)
+ * race on it and must be serialised by the caller.  The array keeps whatever
+ * the last call left; nothing has to be cleared, because each call writes
+ * every element it later reads.
+ */
+#define XNOR_BINACTIV_STATIC_MAX_PIXELS (1u << 20)
+xnor_status xnor_binactiv_static(const float *x, const float *bn_scale, const float *bn_shift,
+                                 const xnor_conv_desc *d, uint32_t *x_packed, float *K,
+                                 void *cuda_stream);
+
+/*
  * BinConv -- Eq. 11: out = (sign(I) (*) sign(W)) (.) K alpha, where (*) is the
  * convolution evaluated with XNOR and bit-count (Section 3.2).  K is shared
  * by all filters of the layer and differs per image; alpha is per filter.

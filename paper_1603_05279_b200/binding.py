@@ -26,7 +26,7 @@ XNOR_ENGINE_UMMA_I8 = 3
 
 EXPORTS = [
     "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
-    "xnor_binarize_weights", "xnor_binactiv", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
+    "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device",
 ]
 
@@ -66,6 +66,8 @@ def load():
     lib.xnor_binarize_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
     lib.xnor_binactiv.restype = ci
     lib.xnor_binactiv.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp, vp, vp]
+    lib.xnor_binactiv_static.restype = ci
+    lib.xnor_binactiv_static.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp, vp]
     lib.xnor_conv2d_forward.restype = ci
     lib.xnor_conv2d_forward.argtypes = [vp, vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc),
                                         vp, vp, vp]
@@ -153,6 +155,18 @@ def xnor_binactiv(x, bn_scale, bn_shift, d, x_packed, A, K, stream=None):
                                 _ptr(bn_shift, torch.float32), ctypes.byref(d),
                                 _ptr(x_packed, torch.int32), _ptr(A, torch.float32),
                                 _ptr(K, torch.float32), _stream(stream)), "xnor_binactiv")
+
+
+BINACTIV_STATIC_MAX_PIXELS = 1 << 20
+
+
+def xnor_binactiv_static(x, bn_scale, bn_shift, d, x_packed, K, stream=None):
+    """xnor_binactiv for callers that cannot supply the A buffer: A lives in a fixed
+    4 MiB array inside the library (at most BINACTIV_STATIC_MAX_PIXELS pixels per call)."""
+    _check(load().xnor_binactiv_static(_ptr(x, torch.float32), _ptr(bn_scale, torch.float32),
+                                       _ptr(bn_shift, torch.float32), ctypes.byref(d),
+                                       _ptr(x_packed, torch.int32), _ptr(K, torch.float32),
+                                       _stream(stream)), "xnor_binactiv_static")
 
 
 def xnor_conv2d_forward(x_packed, w_packed, alpha, K, residual, d, out, acc_out=None, stream=None):

@@ -76,6 +76,21 @@ xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn
                                          (cudaStream_t)cuda_stream));
 }
 
+xnor_status xnor_binactiv_static(const float *x, const float *bn_scale, const float *bn_shift,
+                                 const xnor_conv_desc *d, uint32_t *x_packed, float *K,
+                                 void *cuda_stream) {
+  xnor_status s = check_desc(d, false);
+  if (s != XNOR_OK) return s;
+  if (bad_ptr(x) || bad_ptr(x_packed) || bad_ptr(K)) return XNOR_ERR_INVALID_ARG;
+  if ((bn_scale == nullptr) != (bn_shift == nullptr)) return XNOR_ERR_INVALID_ARG;
+  if (bn_scale && (misaligned(bn_scale) || misaligned(bn_shift))) return XNOR_ERR_INVALID_ARG;
+  if ((unsigned long long)d->N * d->H * d->W > XNOR_BINACTIV_STATIC_MAX_PIXELS)
+    return XNOR_ERR_UNSUPPORTED;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  return from_cuda(xnor::launch_binactiv_static(x, bn_scale, bn_shift, g, x_packed, K,
+                                                (cudaStream_t)cuda_stream));
+}
+
 xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_packed,
                                 const float *alpha, const float *K, const float *residual,
                                 const xnor_conv_desc *d, float *out, int32_t *acc_out,

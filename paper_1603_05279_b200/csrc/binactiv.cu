@@ -112,4 +112,50 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   return cudaGetLastError();
 }
 
+
+// ---------------------------------------------------------------------------
+// xnor_binactiv_static: the same two kernels, with the A plane kept in a
+// fixed array of this library instead of a caller buffer.
+namespace {
+
+constexpr size_t kStaticPixels = XNOR_BINACTIV_STATIC_MAX_PIXELS;
+constexpr int kMaxDevices = 64;
+
+// Lives in the device memory of every GPU that loads the library, until exit.
+static __device__ __align__(256) float g_static_A[kStaticPixels];
+
+// In host code `g_static_A` is only a handle for the runtime; the device
+// address has to be asked for, per device, with that device current.
+float *g_static_A_ptr[kMaxDevices] = {};
+
+cudaError_t static_A_address(float **ptr) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (g_static_A_ptr[dev] == nullptr) {
+    void *p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_A);
+    if (e != cudaSuccess) return e;
+    g_static_A_ptr[dev] = static_cast<float *>(p);
+  }
+  *ptr = g_static_A_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+size_t binactiv_static_max_pixels() { return kStaticPixels; }
+
+cudaError_t launch_binactiv_static(const float *x, const float *scale, const float *shift,
+                                   const ConvGeom &g, uint32_t *x_packed, float *K,
+                                   cudaStream_t st) {
+  float *A = nullptr;
+  cudaError_t e = static_A_address(&A);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
+  // every A value the box filter reads is written by the pack kernel of this call first,
+  // so nothing left by an earlier call is ever used and nothing needs clearing
+  return launch_binactiv(x, scale, shift, g, x_packed, A, K, st);
+}
+
 }  // namespace xnor

@@ -27,6 +27,11 @@ cudaError_t launch_binarize_weights(const float *w, int Co, int C, int kh, int k
 cudaError_t launch_binactiv(const float *x, const float *scale, const float *shift,
                             const ConvGeom &g, uint32_t *x_packed, float *A, float *K,
                             cudaStream_t st);
+// Same, with A in the library's own fixed array (N*H*W <= binactiv_static_max_pixels()).
+size_t binactiv_static_max_pixels();
+cudaError_t launch_binactiv_static(const float *x, const float *scale, const float *shift,
+                                   const ConvGeom &g, uint32_t *x_packed, float *K,
+                                   cudaStream_t st);
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st);
