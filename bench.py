@@ -1,10 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the XNOR-Net forward block on B200.
 
-One step = one pass of the whole hot path over one batch: for each of the four
-AlexNet-shaped binary convolution layers (batch 256 per GPU, synthetic seeded
-inputs) weight binarisation, BN affine + BinActiv (sign-pack, A, K) and BinConv.
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+One step = one pass of the whole hot path over one batch.  Default workload:
+the four AlexNet-shaped binary convolution layers at batch 256 per GPU
+(synthetic seeded inputs); per layer: weight binarisation, BN affine + BinActiv
+(sign-pack, A, K) and BinConv.  `--workload` selects the other shape sets
+(resnet18, sweep, single, chain = the 16-layer ResNet-18 chain with residual
+adds); the bench line proper is the default.  Prints ONE JSON line (rank 0).
+`--impl reference` times the CPU oracle instead.
 """
 import argparse
 import json
@@ -21,11 +24,14 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+from paper_1603_05279_b200 import dist_util as du  # noqa: E402
 from paper_1603_05279_b200 import workloads as wl  # noqa: E402
 
 METRIC = "binary conv TOPS (1-bit MACs/s)"
 UNIT = "T 1-bit MAC/s"
-WORKLOAD = "alexnet_conv2-5_batch256"
+WORKLOAD_NAMES = {"alexnet": "alexnet_conv2-5_batch256", "resnet18": "resnet18_3x3_layers_batch256",
+                  "sweep": "efficiency_sweep_batch64", "single": "single_layer_batch1",
+                  "chain": "xnor_resnet18_chain_16_layers_batch256"}
 HBM_FALLBACK_GBS = 6650.0
 BF16_FALLBACK_TFLOPS = 1590.0
 # popc engine: population count issues 16 results per clock per SM (CUDA C programming
@@ -55,14 +61,54 @@ def host_cores():
         return os.cpu_count() or 1
 
 
+def workload_shapes(name, batch):
+    if name == "chain":
+        return wl.chain_shapes(batch)
+    return [wl.scaled(s, batch) if batch else s for s in wl.CONFIGS[name]]
+
+
+def default_batch(name):
+    return {"alexnet": 256, "resnet18": 256, "sweep": 64, "single": 1, "chain": 256}[name]
+
+
 # ------------------------------------------------------------------ CPU oracle timing
-def oracle_pass(n_images, seeds_rank=0):
-    """Times the oracle, as it stands, on the first n_images of each layer's batch.
+def oracle_pass(name, layer_ids, n_images, rank=0):
+    """Times the oracle, as it stands, on the first n_images of the workload's batch.
     Returns (seconds, macs)."""
     import oracle
     total_t, total_macs = 0.0, 0
-    for li, s in enumerate(wl.ALEXNET):
-        seed = wl.layer_seed("alexnet", li) + 100000 * seeds_rank
+    if name == "chain":
+        shapes = wl.chain_shapes(n_images)
+        seed0 = du.rank_seed(wl.layer_seed("chain", 0), rank)
+        x = wl.normal((n_images, shapes[0].C_in, shapes[0].H, shapes[0].W), seed0)
+        block_in = x
+        for i, s in enumerate(shapes):
+            w = wl.make_weights(s, seed0 + i)
+            t0 = time.perf_counter()
+            mean = x.mean(axis=(0, 2, 3), dtype=np.float64)
+            var = x.var(axis=(0, 2, 3), dtype=np.float64)
+            scale = (1.0 / np.sqrt(var + 1e-5))
+            shift = (-mean * scale).astype(np.float32)
+            scale = scale.astype(np.float32)
+            res = None
+            if i % 2 == 1:
+                s0 = shapes[i - 1]
+                if s0.stride != 1 or s0.C_in != s0.C_out:
+                    pw = wl.normal((s0.C_out, s0.C_in, 1, 1), seed0 + 700 + i - 1, 0.05)
+                    res = oracle.shortcut_conv1x1(block_in, pw, s0.stride)
+                else:
+                    res = block_in
+            r = oracle.xnor_block(x, w, s.stride, s.pad, scale, shift, res)
+            total_t += time.perf_counter() - t0
+            total_macs += wl.macs(s)
+            x = r.out
+            if i % 2 == 1:
+                block_in = x
+        return total_t, total_macs
+    shapes = wl.CONFIGS[name]
+    for li in layer_ids:
+        s = shapes[li]
+        seed = du.rank_seed(wl.layer_seed(name, li), rank)
         x = wl.make_input(s, seed, n_images=n_images)
         w = wl.make_weights(s, seed)
         scale = np.ones((s.C_in,), np.float32)
@@ -74,38 +120,38 @@ def oracle_pass(n_images, seeds_rank=0):
     return total_t, total_macs
 
 
-def cpu_baseline(budget_s=12.0):
+def cpu_baseline(name, layer_ids, batch, budget_s=12.0):
     import oracle
     oracle.build()
     cores = host_cores()
     oracle.set_num_threads(cores)
-    n = 2
-    t, m = oracle_pass(n)
-    want = int(min(256, max(2, n * budget_s / max(t, 1e-3))))
+    n = min(2, batch)
+    t, m = oracle_pass(name, layer_ids, n)
+    want = int(min(batch, max(n, n * budget_s / max(t, 1e-3))))
     if want > n:
         n = want
-        t, m = oracle_pass(n)
+        t, m = oracle_pass(name, layer_ids, n)
     return dict(value=m / t / 1e12, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
-                sample="first %d of 256 images of each of the 4 layers, whole block "
-                       "(BN, BinActiv, weight binarisation, BinConv); %.1f s" % (n, t),
+                sample="first %d of %d images of each layer, whole block (BN, BinActiv, weight "
+                       "binarisation, BinConv); %.1f s" % (n, batch, t),
                 images_per_s=n / t)
 
 
 def run_reference(args):
     """The reference arm: the CPU oracle on a bounded sample per step."""
-    rank = int(os.environ.get("RANK", "0"))
+    world, rank, _ = du.env_world()
     if rank != 0:
         return
     import oracle
     oracle.build()
     cores = host_cores()
     oracle.set_num_threads(cores)
-    n = args.ref_images
-    for _ in range(args.warmup):
-        oracle_pass(n)
+    n = min(args.ref_images, args.batch)
+    for _ in range(min(args.warmup, 1)):
+        oracle_pass(args.workload, args.layer_ids, n)
     t_total, m_total = 0.0, 0
     for _ in range(args.steps):
-        t, m = oracle_pass(n)
+        t, m = oracle_pass(args.workload, args.layer_ids, n)
         t_total += t
         m_total += m
     value = m_total / t_total / 1e12
@@ -114,11 +160,12 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * t_total / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8 (+-1 products, int32 sums)", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample_images_per_step": n},
+        "config": {"workload": WORKLOAD_NAMES[args.workload], "sample_images_per_step": n},
         "images_per_s": n * args.steps / t_total,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
                          "kind": "oracle",
-                         "sample": "each step = first %d of 256 images of each layer" % n},
+                         "sample": "each step = first %d of %d images of each layer"
+                                   % (n, args.batch)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -140,7 +187,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_id), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -179,47 +226,147 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(inside)}
 
 
-# ------------------------------------------------------------------ the CUDA arm
+# ------------------------------------------------------------------ workloads on the GPU
+class LayersJob:
+    """Independent layers: per layer binarize_weights -> binactiv -> conv."""
+
+    def __init__(self, name, layer_ids, batch, rank):
+        import torch
+        from paper_1603_05279_b200.runner import LAUNCHES_PER_LAYER, LayerBuffers
+        self.torch = torch
+        shapes = [wl.scaled(wl.CONFIGS[name][i], batch) for i in layer_ids]
+        self.shapes = shapes
+        self.layers = [LayerBuffers(s) for s in shapes]
+        self.host_x, self.host_w, self.host_out = [], [], []
+        for li, L in zip(layer_ids, self.layers):
+            seed = du.rank_seed(wl.layer_seed(name, li), rank)
+            self.host_x.append(torch.from_numpy(wl.make_input(L.shape, seed)).pin_memory())
+            self.host_w.append(torch.from_numpy(wl.make_weights(L.shape, seed)).pin_memory())
+            self.host_out.append(torch.empty(L.out.shape, dtype=torch.float32).pin_memory())
+            L.x.copy_(self.host_x[-1])
+            L.w.copy_(self.host_w[-1])
+        self.launches = LAUNCHES_PER_LAYER * len(self.layers)
+        self.macs = sum(wl.macs(s) for s in shapes)
+        self.conv_macs = [wl.macs(s) for s in shapes]
+        self.images = batch
+        self.h2d = sum(t.numel() * 4 for t in self.host_x + self.host_w)
+        self.d2h = sum(t.numel() * 4 for t in self.host_out)
+        self.act_bytes = sum(L.binactiv_bytes() for L in self.layers)
+        self.part_names = ("binarize_weights", "binactiv", "conv")
+
+    def step(self, stream):
+        for L in self.layers:
+            L.forward(stream)
+
+    def e2e_step(self, stream):
+        for li, L in enumerate(self.layers):
+            L.x.copy_(self.host_x[li], non_blocking=True)
+            L.w.copy_(self.host_w[li], non_blocking=True)
+            L.forward(stream)
+            self.host_out[li].copy_(L.out, non_blocking=True)
+
+    def parts(self, stream):
+        for li, L in enumerate(self.layers):
+            yield "binarize_weights", li, lambda L=L: L.binarize_weights(stream)
+            yield "binactiv", li, lambda L=L: L.binactiv(stream)
+            yield "conv", li, lambda L=L: L.conv(stream)
+
+
+class ChainJob:
+    """The 16-layer chain: weight binarisation, then 8 residual blocks."""
+
+    def __init__(self, batch, rank):
+        import torch
+        from paper_1603_05279_b200 import binding as B
+        from paper_1603_05279_b200.runner import ChainRunner
+        self.torch, self.B = torch, B
+        ch = ChainRunner(batch)
+        self.ch = ch
+        self.shapes = ch.shapes
+        seed0 = du.rank_seed(wl.layer_seed("chain", 0), rank)
+        self.host_x = torch.from_numpy(wl.normal(tuple(ch.x0.shape), seed0)).pin_memory()
+        self.host_w = [torch.from_numpy(wl.make_weights(L["shape"], seed0 + i)).pin_memory()
+                       for i, L in enumerate(ch.layers)]
+        self.host_pw = {i: torch.from_numpy(wl.normal(tuple(P["w"].shape), seed0 + 700 + i, 0.05))
+                        .pin_memory() for i, P in ch.proj.items()}
+        self.host_out = torch.empty(ch.layers[-1]["out"].shape, dtype=torch.float32).pin_memory()
+        self._upload()
+        ch.binarize_weights()
+        ch.calibrate()                      # set-up: BatchNorm statistics of the seeded batch
+        self.launches = len(ch.layers) + ch.launches_per_forward()
+        self.macs = ch.macs()
+        self.conv_macs = [wl.macs(s) for s in ch.shapes]
+        self.images = batch
+        self.h2d = 4 * (self.host_x.numel() + sum(t.numel() for t in self.host_w) +
+                        sum(t.numel() for t in self.host_pw.values()))
+        self.d2h = 4 * self.host_out.numel()
+        self.act_bytes = 0
+        for s in ch.shapes:
+            ho, wo = wl.out_hw(s)
+            px = s.N * s.H * s.W
+            self.act_bytes += 4 * (px * s.C_in + px * ((s.C_in + 31) // 32) + 2 * px + s.N * ho * wo)
+        self.part_names = ("binarize_weights", "binactiv", "shortcut", "conv")
+
+    def _upload(self):
+        ch = self.ch
+        ch.x0.copy_(self.host_x, non_blocking=True)
+        for L, hw in zip(ch.layers, self.host_w):
+            L["w"].copy_(hw, non_blocking=True)
+        for i, P in ch.proj.items():
+            P["w"].copy_(self.host_pw[i], non_blocking=True)
+
+    def step(self, stream):
+        self.ch.binarize_weights(stream)
+        self.ch.forward(stream)
+
+    def e2e_step(self, stream):
+        self._upload()
+        self.step(stream)
+        self.host_out.copy_(self.ch.layers[-1]["out"], non_blocking=True)
+
+    def parts(self, stream):
+        B, ch = self.B, self.ch
+        for i, L in enumerate(ch.layers):
+            yield "binarize_weights", i, lambda L=L: B.xnor_binarize_weights(
+                L["w"], L["w_packed"], L["alpha"], stream)
+        for i, L in enumerate(ch.layers):
+            x = ch.layer_input(i)
+            yield "binactiv", i, lambda L=L, x=x: B.xnor_binactiv(
+                x, L["scale"], L["shift"], L["desc"], L["x_packed"], L["A"], L["K"], stream)
+            residual = None
+            if i % 2 == 1:
+                b0 = i - 1
+                if b0 in ch.proj:
+                    P = ch.proj[b0]
+                    yield "shortcut", i, lambda P=P, b0=b0: B.xnor_shortcut_conv1x1(
+                        ch.layer_input(b0), P["w"], ch.shapes[b0].stride, P["out"], stream)
+                    residual = P["out"]
+                else:
+                    residual = ch.layer_input(b0)
+            yield "conv", i, lambda L=L, residual=residual: B.xnor_conv2d_forward(
+                L["x_packed"], L["w_packed"], L["alpha"], L["K"], residual, L["desc"], L["out"],
+                None, stream)
+
+
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     import paper_1603_05279_b200 as X
-    from paper_1603_05279_b200.runner import LAUNCHES_PER_LAYER, LayerBuffers
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = du.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    du.init("nccl", local)
     X.load()
     X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2, "umma_i8": 3}[args.engine])
     stream = torch.cuda.current_stream()
 
-    # ---- synthetic inputs: every rank has its own batch of 256 (weak scaling, no exchange)
-    shapes = [wl.scaled(wl.ALEXNET[i], args.batch) for i in args.layer_ids]
-    layers = [LayerBuffers(s) for s in shapes]
-    host_x, host_w, host_out = [], [], []
-    for li, L in enumerate(layers):
-        seed = wl.layer_seed("alexnet", args.layer_ids[li]) + 100000 * rank
-        hx = torch.from_numpy(wl.make_input(L.shape, seed)).pin_memory()
-        hw = torch.from_numpy(wl.make_weights(L.shape, seed)).pin_memory()
-        host_x.append(hx)
-        host_w.append(hw)
-        host_out.append(torch.empty(L.out.shape, dtype=torch.float32).pin_memory())
-        L.x.copy_(hx)
-        L.w.copy_(hw)
+    # every rank has its own batch (weak scaling, no exchange on the data path)
+    if args.workload == "chain":
+        job = ChainJob(args.batch, rank)
+    else:
+        job = LayersJob(args.workload, args.layer_ids, args.batch, rank)
     torch.cuda.synchronize()
-
-    def step():
-        for L in layers:
-            L.forward(stream)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
 
     props = torch.cuda.get_device_properties(local)
     gpu_id = getattr(props, "uuid", None)
@@ -232,91 +379,75 @@ def run_ours(args):
     # ---- device-resident timing
     t_load0 = time.time()
     for _ in range(args.warmup):
-        step()
+        job.step(stream)
     torch.cuda.synchronize()
-    barrier()
+    du.barrier()
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     for _ in range(args.steps):
-        step()
+        job.step(stream)
     ev1.record(stream)
     torch.cuda.synchronize()
-    barrier()
+    du.barrier()
     elapsed_ms = ev0.elapsed_time(ev1)
 
-    # ---- per-kernel pass (same steps again, one event pair per launch group)
-    names = ("binarize_weights", "binactiv", "conv")
-    per = {n: [0.0] * len(layers) for n in names}
+    # ---- per-kernel pass (same steps again, one event pair per library call)
+    per = {n: {} for n in job.part_names}
     evs = []
     for _ in range(args.steps):
-        for li, L in enumerate(layers):
-            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-            e[0].record(stream)
-            L.binarize_weights(stream)
-            e[1].record(stream)
-            L.binactiv(stream)
-            e[2].record(stream)
-            L.conv(stream)
-            e[3].record(stream)
-            evs.append((li, e))
+        for name, idx, fn in job.parts(stream):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            evs.append((name, idx, a, b))
     torch.cuda.synchronize()
-    for li, e in evs:
-        for k, n in enumerate(names):
-            per[n][li] += e[k].elapsed_time(e[k + 1]) / args.steps
+    for name, idx, a, b in evs:
+        per[name][idx] = per[name].get(idx, 0.0) + a.elapsed_time(b) / args.steps
+    # keep the GPU busy a little longer so that the clock sampler sees it under load
+    t_busy = time.time()
+    while time.time() - t_busy < 0.6:
+        job.step(stream)
+        torch.cuda.synchronize()
     t_load1 = time.time()
 
     # ---- end to end: pinned host -> device, block, device -> pinned host, every step
-    def e2e_step():
-        for li, L in enumerate(layers):
-            L.x.copy_(host_x[li], non_blocking=True)
-            L.w.copy_(host_w[li], non_blocking=True)
-            L.forward(stream)
-            host_out[li].copy_(L.out, non_blocking=True)
-
     for _ in range(min(args.warmup, 3)):
-        e2e_step()
+        job.e2e_step(stream)
     torch.cuda.synchronize()
-    barrier()
+    du.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        e2e_step()
+        job.e2e_step(stream)
     e1.record(stream)
     torch.cuda.synchronize()
-    barrier()
+    du.barrier()
     e2e_ms = e0.elapsed_time(e1)
     sampler.stop()
     X.xnor_check_device(stream)
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    elapsed_ms, e2e_ms = du.max_over_ranks([elapsed_ms, e2e_ms], device="cuda")
 
-    macs_step = sum(wl.macs(L.shape) for L in layers)
-    images_step = args.batch
-    sec = elapsed_ms / 1e3
-    value = world * macs_step * args.steps / sec / 1e12
-    e2e_value = world * macs_step * args.steps / (e2e_ms / 1e3) / 1e12
-    h2d = sum(t.numel() * 4 for t in host_x) + sum(t.numel() * 4 for t in host_w)
-    d2h = sum(t.numel() * 4 for t in host_out)
+    value = du.job_throughput(job.macs, args.steps, world, elapsed_ms) / 1e12
+    e2e_value = du.job_throughput(job.macs, args.steps, world, e2e_ms) / 1e12
 
-    full = args.batch == 256 and args.layer_ids == [0, 1, 2, 3]
+    full = args.batch == default_batch(args.workload) and \
+        (args.workload == "chain" or args.layer_ids == list(range(len(wl.CONFIGS[args.workload]))))
     peaks = measured_peaks()
     clocks = sampler.summary(t_load0, t_load1)
-    conv_ms = sum(per["conv"])
-    conv_macs = macs_step
+    conv_ms = sum(per["conv"].values())
+    conv_macs = sum(job.conv_macs)
     engine = args.engine
-    if engine == "auto":
-        engine = "umma" if all(s.stride == 1 for s in shapes) else "mixed"
+    n_conv = len(job.conv_macs)
     if engine != "popc":
         # tensor-core peak for the operand type in use = measured bf16 peak x the nominal
         # ratio of that type to bf16 (e2m1: 9 / 2.25 = 4, int8: 2); the sustained figure,
         # because the kernel is timed inside a long step.  2 flops per 1-bit MAC.
         ratio, kind = (2, "int8") if engine == "umma_i8" else (4, "e2m1 (fp4)")
         roofline = {"kernel": "BinConv tensor-core kernel (one launch per layer, %d per step)"
-                              % len(layers), "bound": "tensor",
+                              % n_conv, "bound": "tensor",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12,
                     "peak": ratio * peaks["bf16_sustained"], "unit": "TFLOP/s",
                     "peak_source": "%d x %s sustained bf16 TFLOP/s (nominal %s : bf16 ratio)"
@@ -324,24 +455,29 @@ def run_ours(args):
     else:
         clk = (clocks["sm_mhz"] or 1965.0) * 1e6
         peak = POPC_PER_CLK_PER_SM * 32 * props.multi_processor_count * clk * 2 / 1e12
-        roofline = {"kernel": "binconv_popc_kernel (4 launches per step)", "bound": "alu",
+        roofline = {"kernel": "binconv_popc_kernel (%d launches per step)" % n_conv,
+                    "bound": "alu",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12, "peak": peak,
                     "unit": "TFLOP/s",
                     "peak_source": "derived: 16 popc/clk/SM x 32 bits x %d SMs x median SM clock "
                                    "during the run" % props.multi_processor_count,
                     "traffic": None}
     roofline["frac"] = roofline["achieved"] / roofline["peak"]
-    act_bytes = sum(L.binactiv_bytes() for L in layers)
-    act_ms = sum(per["binactiv"])
+    act_ms = sum(per["binactiv"].values())
+
+    def ordered(d):
+        return [round(d[k], 4) for k in sorted(d)]
+
     breakdown = {
-        "per_layer_ms": {n: [round(v, 4) for v in per[n]] for n in names},
-        "conv_TMACs": [round(wl.macs(L.shape) / (per["conv"][i] / 1e3) / 1e12, 2)
-                       for i, L in enumerate(layers)],
-        "binactiv_GBs": round(act_bytes / (act_ms / 1e3) / 1e9, 1),
-        "binactiv_frac_of_hbm": round(act_bytes / (act_ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4),
+        "per_layer_ms": {n: ordered(per[n]) for n in job.part_names},
+        "conv_TMACs": [round(job.conv_macs[i] / (per["conv"][k] / 1e3) / 1e12, 2)
+                       for i, k in enumerate(sorted(per["conv"]))],
+        "binactiv_GBs": round(job.act_bytes / (act_ms / 1e3) / 1e9, 1),
+        "binactiv_frac_of_hbm": round(job.act_bytes / (act_ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4),
         "hbm_peak_gbs": peaks["hbm_gbs"], "peaks": peaks["source"],
     }
 
+    name = WORKLOAD_NAMES[args.workload]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
@@ -352,26 +488,26 @@ def run_ours(args):
                   else "e2m1 (fp4) tensor-core operands from 1-bit words, exact integer sums in "
                        "fp32, fp32 scaling"),
         "data": "synthetic",
-        "config": {"workload": WORKLOAD if full else "subset of " + WORKLOAD,
-                   "layers": [s.name for s in shapes],
-                   "batch_per_gpu": images_step, "engine": engine,
+        "config": {"workload": name if full else "subset of " + name,
+                   "layers": [s.name for s in job.shapes],
+                   "batch_per_gpu": job.images, "engine": engine,
                    "l2": "step working set %d MB of inputs+outputs (L2 is 126 MB); no flush"
-                         % ((h2d + d2h) // 1000000),
+                         % ((job.h2d + job.d2h + (job.act_bytes if args.workload == "chain" else 0))
+                            // 1000000),
                    "step": "weight binarisation + BN/BinActiv + BinConv for each layer"},
-        "images_per_s": world * images_step * args.steps / sec,
+        "images_per_s": du.job_throughput(job.images, args.steps, world, elapsed_ms),
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
-        "gpu_launches": LAUNCHES_PER_LAYER * len(layers) * args.steps,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": job.h2d,
+                "d2h_bytes_per_step": job.d2h, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": job.launches * args.steps,
         "roofline": roofline,
         "kernels": breakdown,
     }
     if rank == 0:
         if world == 1 and full and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline()
+            line["cpu_baseline"] = cpu_baseline(args.workload, args.layer_ids, args.batch)
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    du.finish()
 
 
 def main():
@@ -384,12 +520,17 @@ def main():
                     help="images per layer per step of the reference (oracle) arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_i8"])
-    ap.add_argument("--layers", default="0,1,2,3",
-                    help="subset of the four layers (profiling runs only; the bench line is the "
-                         "default: all four)")
-    ap.add_argument("--batch", type=int, default=256, help="images per GPU (default 256)")
+    ap.add_argument("--workload", default="alexnet", choices=sorted(WORKLOAD_NAMES),
+                    help="shape set (the bench line proper is the default, alexnet)")
+    ap.add_argument("--layers", default="",
+                    help="subset of the workload's layers, e.g. 0,2 (profiling runs only)")
+    ap.add_argument("--batch", type=int, default=0, help="images per GPU (default: the workload's)")
     args = ap.parse_args()
-    args.layer_ids = [int(t) for t in args.layers.split(",")]
+    if args.batch <= 0:
+        args.batch = default_batch(args.workload)
+    n_layers = 16 if args.workload == "chain" else len(wl.CONFIGS[args.workload])
+    args.layer_ids = [int(t) for t in args.layers.split(",")] if args.layers else \
+        list(range(n_layers))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -65,3 +65,96 @@ class LayerBuffers:
 
 # kernels launched by one forward(): binarize 1, binactiv 2 (pack, box filter), conv 1
 LAUNCHES_PER_LAYER = 4
+
+
+class ChainRunner:
+    """The 16 binary 3x3 layers of the ResNet-18 variant (Section 4.2) as 8 basic blocks:
+
+        y1 = BinConv1(BinActiv(BN1(x)))
+        y2 = BinConv2(BinActiv(BN2(y1))) + shortcut(x)
+
+    shortcut = identity, or the fp32 1x1 stride-2 projection where the shape
+    changes.  Launch sequence and buffers only; every step is a library call.
+    BatchNorm enters as per-channel (scale, shift) vectors that the caller sets
+    (see `calibrate`).
+    """
+
+    def __init__(self, N, device="cuda", keep_acc=False):
+        self.N = N
+        self.shapes = wl.chain_shapes(N)
+        self.device = device
+        s0 = self.shapes[0]
+        self.x0 = torch.empty((N, s0.C_in, s0.H, s0.W), dtype=torch.float32, device=device)
+        self.layers = []
+        for s in self.shapes:
+            d = B.desc_of(s)
+            L = {"shape": s, "desc": d}
+            L["w"] = torch.empty((s.C_out, s.C_in, s.k, s.k), dtype=torch.float32, device=device)
+            L["w_packed"], L["alpha"] = B.alloc_weights(s.C_out, s.C_in, s.k, s.k, device)
+            L["x_packed"], L["A"], L["K"] = B.alloc_binactiv(d, device)
+            L["scale"] = torch.ones((s.C_in,), dtype=torch.float32, device=device)
+            L["shift"] = torch.zeros((s.C_in,), dtype=torch.float32, device=device)
+            L["out"] = B.alloc_out(d, device=device)
+            L["acc"] = B.alloc_out(d, torch.int32, device) if keep_acc else None
+            self.layers.append(L)
+        # projection shortcuts: one per block whose first layer has stride 2
+        self.proj = {}
+        for i in range(0, len(self.shapes), 2):
+            s = self.shapes[i]
+            if s.stride != 1 or s.C_in != s.C_out:
+                ho, wo = wl.out_hw(s)
+                self.proj[i] = {
+                    "w": torch.empty((s.C_out, s.C_in), dtype=torch.float32, device=device),
+                    "out": torch.empty((N, s.C_out, ho, wo), dtype=torch.float32, device=device)}
+
+    def layer_input(self, i):
+        return self.x0 if i == 0 else self.layers[i - 1]["out"]
+
+    def binarize_weights(self, stream=None):
+        for L in self.layers:
+            B.xnor_binarize_weights(L["w"], L["w_packed"], L["alpha"], stream)
+
+    def run_layer(self, i, stream=None):
+        """BN -> BinActiv -> BinConv of layer i (plus the block's shortcut on odd i)."""
+        L = self.layers[i]
+        x = self.layer_input(i)
+        B.xnor_binactiv(x, L["scale"], L["shift"], L["desc"], L["x_packed"], L["A"], L["K"], stream)
+        residual = None
+        if i % 2 == 1:
+            b0 = i - 1
+            if b0 in self.proj:
+                P = self.proj[b0]
+                B.xnor_shortcut_conv1x1(self.layer_input(b0), P["w"], self.shapes[b0].stride,
+                                        P["out"], stream)
+                residual = P["out"]
+            else:
+                residual = self.layer_input(b0)
+        B.xnor_conv2d_forward(L["x_packed"], L["w_packed"], L["alpha"], L["K"], residual,
+                              L["desc"], L["out"], L["acc"], stream)
+        return residual
+
+    def forward(self, stream=None):
+        for i in range(len(self.layers)):
+            self.run_layer(i, stream)
+        return self.layers[-1]["out"]
+
+    def calibrate(self, eps=1e-5, stream=None):
+        """Sets every BatchNorm to the statistics of its own input on the current batch
+        (biased variance, gamma = 1, beta = 0), layer by layer.  Set-up, not the timed path:
+        the statistics are plain torch reductions; the folded (scale, shift) vectors are what
+        the library (and any checker) receives."""
+        for i, L in enumerate(self.layers):
+            x = self.layer_input(i).double()
+            mean = x.mean(dim=(0, 2, 3))
+            var = x.var(dim=(0, 2, 3), unbiased=False)
+            scale = 1.0 / torch.sqrt(var + eps)
+            L["scale"].copy_(scale.float())
+            L["shift"].copy_((-mean * scale).float())
+            self.run_layer(i, stream)
+
+    def launches_per_forward(self):
+        # per layer: pack, box filter, conv; plus one kernel per projection shortcut
+        return 3 * len(self.layers) + len(self.proj)
+
+    def macs(self):
+        return sum(wl.macs(s) for s in self.shapes)
