@@ -191,7 +191,8 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
  *                        alternative, kept for comparison)
  */
 typedef enum {
-  XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2, XNOR_ENGINE_UMMA_I8 = 3
+  XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2, XNOR_ENGINE_UMMA_I8 = 3,
+  XNOR_ENGINE_TC = 4
 } xnor_engine;
 xnor_status xnor_set_engine(xnor_engine e);
 xnor_engine xnor_get_engine(void);

@@ -44,6 +44,12 @@ bool umma_i8_supported(const ConvGeom &g);
 cudaError_t launch_binconv_i8(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
                               float *out, int32_t *acc_out, cudaStream_t st);
+// Persistent tensor-core engine (strides 1 and 2).
+bool umma_tc_supported(const ConvGeom &g);
+cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                              const float *K, const float *residual, const ConvGeom &g,
+                              float *out, int32_t *acc_out, cudaStream_t st);
+cudaError_t read_status_tc(int *status);
 // Read (and clear if set) the device status word of each tensor-core kernel.
 cudaError_t read_status_fp4(int *status);
 cudaError_t read_status_i8(int *status);
