@@ -26,7 +26,9 @@
  *    means +1.
  *  - Bit packing is along channels in 32-bit words: channel c is bit (c % 32)
  *    of word (c / 32); Cw = ceil(C_in / 32) words per pixel or filter tap;
- *    unused high bits of the last word are 0 in both operands.
+ *    unused high bits of the last word are 0 in both operands.  Activation
+ *    words are pixel-major ([N][H][W][Cw]); filter words are stored in the
+ *    order xnor_binarize_weights documents.
  *  - Zero padding: a filter tap that falls outside the image contributes 0 to
  *    the binary convolution and 0 to the box filter that makes K.
  */
@@ -75,7 +77,13 @@ int xnor_out_extent(int in, int k, int stride, int pad);
  * inference; the real-valued weights are not needed afterwards.
  *
  *   w         in   fp32 [C_out][C_in][k_h][k_w]
- *   w_packed  out  u32  [C_out][k_h][k_w][Cw]   sign bits, channel-innermost
+ *   w_packed  out  u32  [P][C_out][2], P = ceil(k_h*k_w*Cw / 2): sign bits in
+ *                  "word-pair-major" order.  With f = (ky*k_w + kx)*Cw + cw the
+ *                  index of a 32-channel word inside a filter, word f of filter
+ *                  co is element [f/2][co][f%2]; when k_h*k_w*Cw is odd the last
+ *                  pair is padded with a 0 word.  (Words 2j and 2j+1 of all
+ *                  filters - one 64-channel step of the contraction - are
+ *                  contiguous, which is how the convolution reads them.)
  *   alpha     out  fp32 [C_out]
  *
  * INVALID_ARG: null or misaligned pointer, non-positive size.
@@ -148,7 +156,7 @@ xnor_status xnor_binactiv_static(const float *x, const float *bn_scale, const fl
  * by all filters of the layer and differs per image; alpha is per filter.
  *
  *   x_packed  in   u32  [N][H][W][Cw]            from xnor_binactiv
- *   w_packed  in   u32  [C_out][k_h][k_w][Cw]    from xnor_binarize_weights
+ *   w_packed  in   u32  [P][C_out][2]             from xnor_binarize_weights
  *   alpha     in   fp32 [C_out]
  *   K         in   fp32 [N][H_out][W_out]
  *   residual  in   fp32 [N][C_out][H_out][W_out] or NULL; added after the scaling

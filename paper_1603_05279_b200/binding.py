@@ -189,7 +189,8 @@ def xnor_shortcut_conv1x1(x, w, stride, out, stream=None):
 # ---- buffer helpers (allocation only; torch owns the memory) -------------------------------
 def alloc_weights(C_out, C_in, k_h, k_w, device="cuda"):
     Cw = (C_in + 31) // 32
-    return (torch.empty((C_out, k_h, k_w, Cw), dtype=torch.int32, device=device),
+    pairs = (k_h * k_w * Cw + 1) // 2          # word-pair-major layout, see include/xnor.h
+    return (torch.empty((pairs, C_out, 2), dtype=torch.int32, device=device),
             torch.empty((C_out,), dtype=torch.float32, device=device))
 
 

@@ -1,4 +1,4 @@
-// Weight binarisation: B = sign(W) bit-packed along channels, alpha = ||W||_1/n
+// Weight binarisation: B = sign(W) bit-packed along channels (word-pair-major), alpha = ||W||_1/n
 // per filter (Section 3.1, Eq. 4 and Eq. 6).  One thread block per filter.
 #include "common.cuh"
 
@@ -9,7 +9,7 @@ namespace {
 constexpr int kThreads = 256;
 
 __global__ void __launch_bounds__(kThreads)
-binarize_weights_kernel(const float *__restrict__ w, int C, int taps, int Cw,
+binarize_weights_kernel(const float *__restrict__ w, int Co, int C, int taps, int Cw,
                         uint32_t *__restrict__ w_packed, float *__restrict__ alpha) {
   extern __shared__ uint32_t words[];  // [taps][Cw]
   __shared__ double red[kThreads / 32];
@@ -39,8 +39,9 @@ binarize_weights_kernel(const float *__restrict__ w, int C, int taps, int Cw,
     for (int i = 0; i < kThreads / 32; ++i) s += red[i];
     alpha[co] = (float)(s / (double)n);
   }
-  uint32_t *dst = w_packed + (size_t)co * nwords;
-  for (int j = threadIdx.x; j < nwords; j += kThreads) dst[j] = words[j];
+  // word-pair-major layout (see packed_weight_index); an odd word count is padded with 0
+  for (int j = threadIdx.x; j < ((nwords + 1) & ~1); j += kThreads)
+    w_packed[packed_weight_index(Co, co, j)] = j < nwords ? words[j] : 0u;
 }
 
 }  // namespace
@@ -50,7 +51,7 @@ cudaError_t launch_binarize_weights(const float *w, int Co, int C, int kh, int k
   const int taps = kh * kw, Cw = (C + 31) / 32;
   const size_t smem = (size_t)taps * Cw * sizeof(uint32_t);
   if (smem > 48 * 1024) return cudaErrorInvalidValue;
-  binarize_weights_kernel<<<Co, kThreads, smem, st>>>(w, C, taps, Cw, w_packed, alpha);
+  binarize_weights_kernel<<<Co, kThreads, smem, st>>>(w, Co, C, taps, Cw, w_packed, alpha);
   return cudaGetLastError();
 }
 

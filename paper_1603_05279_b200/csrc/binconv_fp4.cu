@@ -331,16 +331,18 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_fp4_kernel(const Fp4Param
       const int row = pt & (kFilters - 1), par = pt >> 7;
       const int co = co0 + row;
       const bool row_live = co < P.Co;
-      const uint32_t *f_ptr = P.wp + (size_t)(row_live ? co : 0) * taps * P.Cw + cw0 + par;
+      const int f_co = row_live ? co : 0;
+      int f_word = cw0 + par;                         // word index of (tap f_tap, word f_wb) in the row
       int f_wb = 0, f_tap = row_live ? 0 : taps;      // dead rows never fetch
       uint32_t pf[kPrefetch][WPT];
       auto fetch = [&](uint32_t dst[WPT]) {
         if (f_tap < taps) {
 #pragma unroll
           for (int i = 0; i < WPT; ++i)
-            dst[i] = f_wb + 2 * i + par < cwn ? __ldg(f_ptr + f_wb + 2 * i) : 0u;
+            dst[i] = f_wb + 2 * i + par < cwn
+                         ? __ldg(P.wp + packed_weight_index(P.Co, f_co, f_word + f_wb + 2 * i)) : 0u;
           f_wb += WPS;
-          if (f_wb >= cwn_e) { f_wb = 0; ++f_tap; f_ptr += P.Cw; }
+          if (f_wb >= cwn_e) { f_wb = 0; ++f_tap; f_word += P.Cw; }
         } else {
 #pragma unroll
           for (int i = 0; i < WPT; ++i) dst[i] = 0u;

@@ -263,15 +263,18 @@ __global__ void __launch_bounds__(kThreads, 2) binconv_i8_kernel(const UmmaParam
       // refilled right after it is expanded, so a load has kPrefetch stages to land.
       const int co = co0 + pt;
       const bool row_live = pt < NT && co < P.Co;
-      const uint32_t *f_ptr = P.wp + (size_t)(row_live ? co : 0) * taps * P.Cw + cw0;
+      const int f_co = row_live ? co : 0;
+      int f_word = cw0;                               // word index of (tap f_tap, word 0 of the chunk)
       int f_wb = 0, f_tap = row_live ? 0 : taps;     // dead rows never fetch
       uint32_t pf[kPrefetch][WPS];
       auto fetch = [&](uint32_t dst[WPS]) {
         if (f_tap < taps) {
 #pragma unroll
-          for (int wi = 0; wi < WPS; ++wi) dst[wi] = f_wb + wi < cwn ? __ldg(f_ptr + f_wb + wi) : 0u;
+          for (int wi = 0; wi < WPS; ++wi)
+            dst[wi] = f_wb + wi < cwn
+                          ? __ldg(P.wp + packed_weight_index(P.Co, f_co, f_word + f_wb + wi)) : 0u;
           f_wb += WPS;
-          if (f_wb >= cwn) { f_wb = 0; ++f_tap; f_ptr += P.Cw; }
+          if (f_wb >= cwn) { f_wb = 0; ++f_tap; f_word += P.Cw; }
         } else {
 #pragma unroll
           for (int wi = 0; wi < WPS; ++wi) dst[wi] = 0u;

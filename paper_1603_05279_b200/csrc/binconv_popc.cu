@@ -75,7 +75,8 @@ binconv_popc_kernel(const uint32_t *__restrict__ xp, const uint32_t *__restrict_
       const int ft = idx / cwn;           // f*taps + tap
       const int f = ft / taps;
       uint32_t v = 0u;
-      if (co0 + f < P.Co) v = __ldg(wp + ((size_t)co0 * taps + ft) * P.Cw + cw0 + cw);
+      if (co0 + f < P.Co)
+        v = __ldg(wp + packed_weight_index(P.Co, co0 + f, (ft - f * taps) * P.Cw + cw0 + cw));
       wts[ft * P.cwc + cw] = v;
     }
     __syncthreads();

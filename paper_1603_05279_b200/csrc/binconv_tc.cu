@@ -22,26 +22,30 @@
 //        0, so padded taps contribute exactly 0 with no mask or correction.
 //        Stream positions that are padding give junk rows that are never stored.
 //    B (N = NT rows)  = a slab of NT filters, expanded from bits by producer
-//        warps into a ring of shared-memory stages, in the order of a table of
-//        K-steps (one MMA of K = 64 = two 32-channel pieces each) that every
-//        CTA builds once.  A piece is (tap, channel word); when the number of
-//        channel words is odd the last word of two consecutive taps shares an
-//        MMA, so no K-step is wasted on padding.
+//        warps into a ring of shared-memory stages.  One MMA (a K-step, K = 64)
+//        consumes two 32-channel pieces; a piece is one packed word (tap,
+//        channel word) of a filter row, and K-step j takes words 2j and 2j+1
+//        of the row in memory order, so a step may straddle two taps and no
+//        step is wasted on channel padding.  The host precomputes, per step,
+//        the A-operand descriptor (start of the lower-addressed piece, distance
+//        to the other one) and whether the two pieces are swapped.
 //
 //  Encodings.  A packed word holds 32 sign bits; it becomes 32 e2m1 nibbles in
 //  four registers, register r holding channels r, r+4, ..., r+28.  Activations
 //  are +-{2, 1, 0.5, 0.5} for r = 0..3, weights +-{0.5, 1, 2, 2}: every product
 //  is the product of the two signs.
 //
-//  Roles (480 threads, one CTA per SM, CTAs loop over work items = (pixel
-//  tile, filter slab)): warps 0-7 epilogue (tensor memory -> registers ->
-//  coalesced NCHW stores of D * K * alpha (+ residual)), warp 8 issues the
-//  MMAs, warps 9-12 expand weights, warps 13-14 expand activation patches.
+//  Roles (512 threads, one CTA per SM, CTAs loop over work items = (pixel
+//  tile, filter slab)): warps 0-3 epilogue (tensor memory -> registers ->
+//  coalesced NCHW stores of D * K * alpha (+ residual)), warp 4 issues the
+//  MMAs, warps 5-12 expand weights, warps 13-15 expand activation patches.
 //  Accumulators are double-buffered in tensor memory so the epilogue of one
 //  item overlaps the MMAs of the next.  Every wait is bounded: on expiry the
 //  CTA records XNOR_ERR_TIMEOUT in a device status word, stops, frees its
 //  tensor memory and exits.
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "umma_common.cuh"
@@ -49,25 +53,49 @@
 namespace xnor {
 
 __device__ int g_status_tc = 0;
+#ifdef XNOR_TRACE
+// cycle totals of one warp per role of one CTA: [0..7] mma, [8..15] weights, [16..23] patch,
+// [24..31] epilogue
+__device__ long long g_tc_trace[64];
+#define TR_DECL(first) long long tr_t = 0, tr_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}; \
+  const bool tr_on = blockIdx.x == 1 && (threadIdx.x & 31) == 0 && (first)
+#define TR_T0 do { if (tr_on) tr_t = clock64(); } while (0)
+#define TR_ADD(i) do { if (tr_on) { const long long n_ = clock64(); tr_a[(i) & 7] += n_ - tr_t; tr_t = n_; } } while (0)
+#define TR_FLUSH(base) do { if (tr_on) { for (int q_ = 0; q_ < 8; ++q_) g_tc_trace[(base) + q_] += tr_a[q_]; } } while (0)
+#else
+#define TR_DECL(first)
+#define TR_T0 do {} while (0)
+#define TR_ADD(i) do {} while (0)
+#define TR_FLUSH(base) do {} while (0)
+#endif
 
 namespace {
 
 using namespace umma;
 
-constexpr int kEpiWarps = 8;
-constexpr int kMmaWarp = 8;
-constexpr int kWgtWarp0 = 9, kWgtWarps = 4, kWgtThreads = 32 * kWgtWarps;
-constexpr int kPatWarp0 = 13, kPatWarps = 2, kPatThreads = 32 * kPatWarps;
-constexpr int kThreads = 32 * (kPatWarp0 + kPatWarps);     // 480
+// nanoseconds a waiting role sleeps between polls of its barrier
+#ifndef XNOR_SLEEP_EPI
+#define XNOR_SLEEP_EPI 200
+#endif
+#ifndef XNOR_SLEEP_PAT
+#define XNOR_SLEEP_PAT 200
+#endif
+#ifndef XNOR_SLEEP_WGT
+#define XNOR_SLEEP_WGT 50
+#endif
+
+constexpr int kEpiWarps = 4;
+constexpr int kMmaWarp = 4;
+constexpr int kWgtWarp0 = 5, kWgtWarps = 8, kWgtThreads = 32 * kWgtWarps;
+constexpr int kPatWarp0 = 13, kPatWarps = 3, kPatThreads = 32 * kPatWarps;
+constexpr int kThreads = 32 * (kPatWarp0 + kPatWarps);     // 512: 16 warps, 128 registers each
 constexpr int kTileM = 128;          // stream positions per tile = tensor-memory lanes
 constexpr int kTmemCols = 512;
 constexpr int kSfCol = 480;          // columns [480, 512): unit block scales
 constexpr int kMaxAccCols = 480;
 constexpr int kMaxStages = 6;
 constexpr int kMaxPatchBufs = 4;
-constexpr int kMaxSteps = 1024;      // K-steps (MMAs) per work item
-constexpr int kPrefetch = 3;         // weight stages whose packed words are in flight
-constexpr int kUnits = 4;            // (row, K-step) units per weight thread per stage
+constexpr int kMaxSteps = 800;       // K-steps (MMAs) per work item (< 1024: swap_mask)
 constexpr size_t kCtrlBytes = 512;
 constexpr size_t kSmemMax = 232448 - 1024;
 
@@ -88,29 +116,58 @@ struct TcParams {
   int nsteps;                  // K-steps per item
   int mps;                     // K-steps per weight stage
   int stages;
-  int rows_mod, grp_steps;     // weight-thread mapping (see weight producer)
   uint32_t patch_bytes, stage_bytes;
-  uint32_t off_table, off_ring, off_patch;   // byte offsets in dynamic shared memory
+  int rows_mod, grp_steps;     // weight-thread mapping (see weight producer)
+  uint32_t off_ring, off_patch;  // byte offsets in dynamic shared memory
   uint32_t idesc;
   uint32_t tail_mask;          // bits of real channels in the last word
+  // Low word of the A-operand descriptor of every K-step (start address relative to the
+  // patch in bits 0-13, leading-dimension offset in bits 16-29; the high word is the same
+  // for all).  It lives in the kernel parameters so that the MMA issuer reads and offsets
+  // it on the uniform datapath: an MMA is as short as 32 cycles, and descriptors that pass
+  // through per-thread registers cost more than that to issue.
+  uint32_t adesc_lo[kMaxSteps];
+  uint32_t swap_mask[32];              // bit j: word 2j+1 is the first piece of step j
+  int row_words;               // packed words per filter row = k_h*k_w*Cw
+  uint32_t div_wq_m, div_hq_m; // multipliers and shifts of the exact divisions by Wq and Hq
+  int div_wq_s, div_hq_s;      // (dividends below 2^31)
 };
 
-// One K-step: A-operand start offset inside a patch, distance between its two
-// 32-channel pieces, and the two packed words of a filter row it consumes
-// (index within the row's [tap][Cw] words; 0xFFFFFFFF = no second piece).
-struct __align__(16) KStep {
-  uint32_t a_off, a_lbo, gw1, gw2;
-};
-
-__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
-                                          uint32_t idesc, uint32_t sfa, uint32_t sfb,
-                                          uint32_t accumulate) {
+// One MMA, issued by the elected lane while the whole warp stays converged (so that the
+// descriptor arithmetic around it can stay on the uniform datapath).  Descriptors are
+// passed as their two 32-bit halves.
+__device__ __forceinline__ void umma_mxf4_elected(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                                  uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                  uint32_t sf, uint32_t accumulate,
+                                                  uint32_t elected) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.ne.b32 q, %8, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %5, [%7], [%7], p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
+        "r"(sf), "r"(elected)
       : "memory");
+}
+
+__device__ __forceinline__ void umma_commit_elected(uint32_t bar, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(elected) : "memory");
+}
+
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+      "elect.sync rx|px, %1;\n\t"
+      "@px mov.s32 %0, 1;\n\t}"
+      : "+r"(pred) : "r"(0xFFFFFFFFu));
+  return pred;
 }
 
 // 32 sign bits -> 32 e2m1 nibbles (sign in bit 3 of a nibble, magnitude code
@@ -129,7 +186,7 @@ __device__ __forceinline__ void expand_signs(uint32_t w, uint32_t v[4]) {
 }
 
 // Shift of a filter tap inside a phase plane, and the plane it reads.
-__device__ __forceinline__ void tap_geometry(const TcParams &P, int tap, int &phase, int &shift) {
+inline void tap_geometry(const TcParams &P, int tap, int &phase, int &shift) {
   const int ky = tap / P.kw, kx = tap - ky * P.kw;
   const int ay = ky - P.pad, ax = kx - P.pad;
   // floor division / non-negative remainder by the stride
@@ -141,50 +198,35 @@ __device__ __forceinline__ void tap_geometry(const TcParams &P, int tap, int &ph
 }
 
 // Piece (tap, w) -> byte offset of its A operand inside a patch.
-__device__ __forceinline__ uint32_t piece_offset(const TcParams &P, int tap, int w) {
+inline uint32_t piece_offset(const TcParams &P, int tap, int w) {
   int phase, shift;
   tap_geometry(P, tap, phase, shift);
   return (uint32_t)(phase * P.Cw + w) * ((uint32_t)P.ppix * 16u) + (uint32_t)shift * 16u;
 }
 
-// K-step j of the fixed order: for every pair of taps (t, t+1): the word pairs
-// of t, the word pairs of t+1, then (Cw odd only) the last words of t and t+1
-// together.  A lone last tap pairs its last word with nothing.
-__device__ void build_kstep(const TcParams &P, int j, KStep &ks) {
-  const int taps = P.kh * P.kw, Cw = P.Cw, h = Cw >> 1;
-  int t1, w1, t2, w2;
-  if ((Cw & 1) == 0) {
-    t1 = j / h; w1 = 2 * (j - t1 * h); t2 = t1; w2 = w1 + 1;
-  } else {
-    const int per_pair = 2 * h + 1;
-    const int pp = j / per_pair, rem = j - pp * per_pair;
-    const int ta = 2 * pp;
-    const bool lone = ta + 1 >= taps;          // last tap without a partner
-    if (rem < h) { t1 = ta; w1 = 2 * rem; t2 = t1; w2 = w1 + 1; }
-    else if (!lone && rem < 2 * h) { t1 = ta + 1; w1 = 2 * (rem - h); t2 = t1; w2 = w1 + 1; }
-    else { t1 = ta; w1 = Cw - 1; t2 = lone ? -1 : ta + 1; w2 = Cw - 1; }
+// K-step j: pieces = words 2j and 2j+1 of a filter row (flat index tap*Cw + w).  Returns
+// the low descriptor word of its A operand; *swap tells whether word 2j+1 comes first.
+inline uint32_t kstep_desc(const TcParams &P, int j, bool *swap) {
+  const int f1 = 2 * j, f2 = 2 * j + 1;
+  uint32_t o1 = piece_offset(P, f1 / P.Cw, f1 % P.Cw), lbo = 16u;   // lone piece: any in-bounds
+  *swap = false;                                                    // partner, its weights are 0
+  if (f2 < P.row_words) {
+    uint32_t o2 = piece_offset(P, f2 / P.Cw, f2 % P.Cw);
+    if (o2 < o1) { const uint32_t o = o1; o1 = o2; o2 = o; *swap = true; }
+    lbo = o2 - o1;
   }
-  ks.a_off = piece_offset(P, t1, w1);
-  ks.gw1 = (uint32_t)(t1 * Cw + w1);
-  if (t2 >= 0) {
-    uint32_t o2 = piece_offset(P, t2, w2);
-    ks.gw2 = (uint32_t)(t2 * Cw + w2);
-    if (o2 < ks.a_off) {       // the piece at the lower address goes first
-      const uint32_t o = ks.a_off, g = ks.gw1;
-      ks.a_off = o2; ks.gw1 = ks.gw2; o2 = o; ks.gw2 = g;
-    }
-    ks.a_lbo = o2 - ks.a_off;
-  } else {
-    ks.a_lbo = 16u;            // any in-bounds piece: its weights are 0
-    ks.gw2 = 0xFFFFFFFFu;
-  }
+  return (o1 >> 4) | ((lbo >> 4) << 16);
+}
+
+// Exact n / d for n < 2^31: q = (n * m) >> (31 + s) with m = ceil(2^(31+s) / d), s = ceil(log2 d).
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m, int s) {
+  return (uint32_t)(((uint64_t)n * m) >> (31 + s));
 }
 
 struct Smem {
   uint32_t wfull, wempty, pfull, pempty, afull, aempty;   // shared-space addresses of barrier arrays
   uint32_t *tmem_slot;
   volatile int *abort_flag;
-  const KStep *table;
   uint32_t ring, patch;                                   // shared-space byte addresses
 };
 
@@ -199,71 +241,110 @@ __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
   s.aempty = s.afull + 16u;
   s.tmem_slot = reinterpret_cast<uint32_t *>(smem + 8 * (2 * kMaxStages + 2 * kMaxPatchBufs + 4));
   s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
-  s.table = reinterpret_cast<const KStep *>(smem + P.off_table);
   s.ring = base + P.off_ring;
   s.patch = base + P.off_patch;
   return s;
 }
 
 // ------------------------------------------------------------------ MMA issuer (one warp)
+// All 32 lanes run this code converged; only the MMA and commit instructions are
+// predicated on the elected lane.  A wait's outcome is made warp-uniform with a vote.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity,
+                                               volatile int *abort_flag) {
+  return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, &g_status_tc));
+}
+
+// The MMAs of one full weight stage, unrolled.
+template <int MPS>
+__device__ __forceinline__ void issue_stage(const TcParams &P, int j0, uint32_t d_tmem,
+                                            uint32_t patch_lo, uint32_t a_hi, uint32_t b_lo,
+                                            uint32_t b_hi, uint32_t b_step, uint32_t tmem_sf,
+                                            uint32_t first, uint32_t el) {
+#pragma unroll
+  for (int jj = 0; jj < MPS; ++jj)
+    umma_mxf4_elected(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, a_hi, b_lo + (uint32_t)jj * b_step,
+                      b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u, el);
+}
+
 __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long long i1,
-                         uint32_t tmem_base, int lane) {
+                         uint32_t tmem_base) {
   const uint32_t tmem_sf = tmem_base + (uint32_t)kSfCol;
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
+  // descriptor halves: high word = stride between 8-row groups (128 B) and the version bit
+  const uint32_t desc_hi = (128u >> 4) | (1u << 14);
+  const uint32_t b_lo0 = ((S.ring & 0x3FFFFu) >> 4) | ((b_lbo >> 4) << 16);   // stage 0, K-step 0
+  const uint32_t b_step = (2u * b_lbo) >> 4;                                   // next K-step
+  const uint32_t stage_step = P.stage_bytes >> 4;
+  const uint32_t el = elect_one();
   int ws = 0, pb = 0;
   uint32_t wph = 0, pph = 0;
   long long k = 0;                       // items done by this CTA
-  int tile = (int)(i0 / P.nslabs), slab = (int)(i0 - (long long)tile * P.nslabs);
+  int slab = (int)(i0 % P.nslabs);
   bool ok = true, new_tile = true;
-  uint32_t patch_addr = 0;
+  uint32_t patch_lo = 0;                 // patch address in descriptor units
+  TR_DECL(true);
+  TR_T0;
   for (long long item = i0; item < i1 && ok; ++item, ++k) {
     if (new_tile) {
-      ok = mbar_wait(S.pfull + 8u * pb, pph, S.abort_flag, &g_status_tc);
+      ok = mbar_wait_warp(S.pfull + 8u * pb, pph, S.abort_flag);
+      TR_ADD(0);
       if (!ok) break;
-      patch_addr = S.patch + (uint32_t)pb * P.patch_bytes;
+      patch_lo = ((S.patch + (uint32_t)pb * P.patch_bytes) & 0x3FFFFu) >> 4;
     }
     const int ab = (int)(k % P.nacc);
     const uint32_t use = (uint32_t)(k / P.nacc);
-    ok = mbar_wait(S.aempty + 8u * ab, (use & 1u) ^ 1u, S.abort_flag, &g_status_tc);
+    ok = mbar_wait_warp(S.aempty + 8u * ab, (use & 1u) ^ 1u, S.abort_flag);
+    TR_ADD(1);
     if (!ok) break;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.NT);
-    uint32_t accumulate = 0;
     for (int st = 0; st < nst && ok; ++st) {
-      ok = mbar_wait(S.wfull + 8u * ws, wph, S.abort_flag, &g_status_tc);
+      const int j0 = st * P.mps;
+      const int nj = min(P.mps, P.nsteps - j0);
+      const uint32_t b_lo = b_lo0 + (uint32_t)ws * stage_step;
+      const uint32_t first = st == 0 ? 0u : 1u;     // the first MMA of an item overwrites
+      ok = mbar_wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
+      TR_ADD(2);
       if (!ok) break;
       tc_fence_after();
-      if (lane == 0) {
-        const int j0 = st * P.mps;
-        const int nj = min(P.mps, P.nsteps - j0);
-        uint32_t b_addr = S.ring + (uint32_t)ws * P.stage_bytes;
-        for (int jj = 0; jj < nj; ++jj) {
-          const KStep ks = S.table[j0 + jj];
-          umma_mxf4(d_tmem, make_desc(patch_addr + ks.a_off, ks.a_lbo, 128u),
-                    make_desc(b_addr, b_lbo, 128u), P.idesc, tmem_sf, tmem_sf, accumulate);
-          accumulate = 1;
-          b_addr += 2u * b_lbo;
-        }
-        umma_commit(S.wempty + 8u * ws);
+      TR_ADD(3);
+      if (nj == 4) issue_stage<4>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      else if (nj == 2) issue_stage<2>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      else if (nj == 8) issue_stage<8>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      else {
+        for (int jj = 0; jj < nj; ++jj)
+          umma_mxf4_elected(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, desc_hi,
+                            b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc, tmem_sf,
+                            jj == 0 ? first : 1u, el);
       }
-      __syncwarp();
+      TR_ADD(4);
+      umma_commit_elected(S.wempty + 8u * ws, el);
+      TR_ADD(5);
       if (++ws == P.stages) { ws = 0; wph ^= 1u; }
     }
     if (!ok) break;
     // next item: same tile (next slab) or the next tile
     new_tile = false;
-    if (++slab == P.nslabs) { slab = 0; ++tile; new_tile = true; }
-    if (lane == 0) {
-      umma_commit(S.afull + 8u * ab);
-      if (new_tile || item + 1 == i1) umma_commit(S.pempty + 8u * pb);
-    }
-    __syncwarp();
+    if (++slab == P.nslabs) { slab = 0; new_tile = true; }
+    umma_commit_elected(S.afull + 8u * ab, el);
+    if (new_tile || item + 1 == i1) umma_commit_elected(S.pempty + 8u * pb, el);
     if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
+    TR_ADD(6);
   }
+  TR_FLUSH(0);
 }
 
-// ------------------------------------------------------------------ weight producers (4 warps)
+// ------------------------------------------------------------------ weight producers (8 warps)
+// A stage holds mps K-steps of NT filter rows: plane (2 jj + piece) of NT x 16 bytes.  K-step
+// j consumes words 2j, 2j+1 of every filter row, which the word-pair-major weight layout
+// keeps contiguous over the filters: a warp reads 32 rows of one K-step as one 256-byte run.
+// Thread mapping: row = wt % rows_mod, and the 256 / rows_mod thread groups split the
+// stage's K-steps, gs = grp_steps each (unit u of a thread = K-step grp * gs + u of the stage).
+// The packed words of kPrefetch stages are in flight in registers.
+constexpr int kPrefetch = 4;
+constexpr int kUnits = 2;
+
 struct WCursor {
   long long item;
   int st, slab;
@@ -272,65 +353,69 @@ struct WCursor {
 __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long long i1, int wt,
                             int lane) {
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
-  const int row0 = wt % P.rows_mod, grp = wt / P.rows_mod;
-  const int gs = P.grp_steps;            // 1, 2 or 4
-  const int gs_log = 31 - __clz(gs);
-  const int nrows = P.NT > 128 ? 2 : 1;
-  const size_t row_words = (size_t)P.kh * P.kw * P.Cw;
+  const int row = wt % P.rows_mod, grp = wt / P.rows_mod;
+  const int gs = P.grp_steps;                      // 1 or 2
+  const bool grp_on = grp * gs < P.mps && row < P.NT;
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
   const int slab0 = (int)(i0 % P.nslabs);
   WCursor fc{i0, 0, slab0}, cc{i0, 0, slab0};
   auto advance = [&](WCursor &c) {
     if (++c.st == nst) { c.st = 0; ++c.item; if (++c.slab == P.nslabs) c.slab = 0; }
   };
-  uint32_t pf[kPrefetch][2 * kUnits];
-  // unit u = rr * gs + kk: filter row row0 + 128 rr, K-step (st * mps + grp * gs + kk)
-  auto fetch = [&](uint32_t dst[2 * kUnits], const WCursor &c) {
+  uint2 pf[kPrefetch][kUnits];
+  auto fetch = [&](uint2 dst[kUnits], const WCursor &c) {
+    const int co = c.slab * P.NT + row;
+    const bool on = grp_on && c.item < i1 && co < P.Co;
+    const int j0 = c.st * P.mps + grp * gs;
 #pragma unroll
     for (int u = 0; u < kUnits; ++u) {
-      dst[2 * u] = 0u; dst[2 * u + 1] = 0u;
-      const int rr = u >> gs_log, kk = u & (gs - 1);
-      const int row = row0 + 128 * rr;
-      const int j = c.st * P.mps + grp * gs + kk;
-      const int co = c.slab * P.NT + row;
-      if (c.item < i1 && rr < nrows && row < P.NT && co < P.Co && j < P.nsteps) {
-        const KStep ks = S.table[j];
-        const uint32_t *rowp = P.wp + (size_t)co * row_words;
-        dst[2 * u] = __ldg(rowp + ks.gw1);
-        if (ks.gw2 != 0xFFFFFFFFu) dst[2 * u + 1] = __ldg(rowp + ks.gw2);
-      }
+      const bool p = on && u < gs && j0 + u < P.nsteps;
+      const uint2 *src = reinterpret_cast<const uint2 *>(P.wp) +
+                         ((size_t)(p ? j0 + u : 0) * P.Co + (p ? co : 0));
+      dst[u] = p ? __ldg(src) : make_uint2(0u, 0u);
     }
   };
+  TR_DECL(wt < 32);
+  TR_T0;
 #pragma unroll
   for (int d = 0; d < kPrefetch; ++d) { fetch(pf[d], fc); advance(fc); }
   int ws = 0;
   uint32_t wph = 1;           // parity to wait for on the empty barriers
   bool ok = true;
+  const uint32_t row_off = (uint32_t)row * 16u;
   while (cc.item < i1 && ok) {
 #pragma unroll
     for (int d = 0; d < kPrefetch; ++d) {
       if (cc.item < i1 && ok) {
         ok = mbar_wait(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc);
+        TR_ADD(0);
         if (ok) {
-          const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes;
+          const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
+          const int co = cc.slab * P.NT + row;
+          const int jj0 = grp * gs;
+          const int j0 = cc.st * P.mps + jj0;
+          const bool on = grp_on && co < P.Co;
+          uint32_t v0[kUnits][4], v1[kUnits][4], a0[kUnits], a1[kUnits];
 #pragma unroll
           for (int u = 0; u < kUnits; ++u) {
-            const int rr = u >> gs_log, kk = u & (gs - 1);
-            const int row = row0 + 128 * rr;
-            const int jj = grp * gs + kk;
-            const int j = cc.st * P.mps + jj;
-            const int co = cc.slab * P.NT + row;
-            if (rr < nrows && row < P.NT && co < P.Co && j < P.nsteps) {
-              const bool two = S.table[j].gw2 != 0xFFFFFFFFu;
-              uint32_t v[4];
-              const uint32_t a = stage + (uint32_t)(2 * jj) * b_lbo + (uint32_t)row * 16u;
-              expand_signs<false>(pf[d][2 * u], v);
-              sts128(a, v[0], v[1], v[2], v[3]);
-              expand_signs<false>(pf[d][2 * u + 1], v);
-              if (!two) { v[0] = 0u; v[1] = 0u; v[2] = 0u; v[3] = 0u; }
-              sts128(a + b_lbo, v[0], v[1], v[2], v[3]);
+            const int j = j0 + u;
+            const bool swap = (P.swap_mask[(j >> 5) & 31] >> (j & 31)) & 1u;
+            const uint32_t keep = 2 * j + 1 < P.row_words ? 0xFFFFFFFFu : 0u;  // lone: partner 0
+            expand_signs<false>(pf[d][u].x, v0[u]);
+            expand_signs<false>(pf[d][u].y, v1[u]);
+            v1[u][0] &= keep; v1[u][1] &= keep; v1[u][2] &= keep; v1[u][3] &= keep;
+            const uint32_t a = stage + (uint32_t)(2 * (jj0 + u)) * b_lbo;
+            a0[u] = swap ? a + b_lbo : a;
+            a1[u] = swap ? a : a + b_lbo;
+          }
+#pragma unroll
+          for (int u = 0; u < kUnits; ++u) {
+            if (on && u < gs && j0 + u < P.nsteps) {
+              sts128(a0[u], v0[u][0], v0[u][1], v0[u][2], v0[u][3]);
+              sts128(a1[u], v1[u][0], v1[u][1], v1[u][2], v1[u][3]);
             }
           }
+          TR_ADD(1);
           fence_proxy_async();
           __syncwarp();
           if (lane == 0) mbar_arrive(S.wfull + 8u * ws);
@@ -338,13 +423,15 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
           advance(cc);
           fetch(pf[d], fc);
           advance(fc);
+          TR_ADD(2);
         }
       }
     }
   }
+  TR_FLUSH(8);
 }
 
-// ------------------------------------------------------------------ patch producers (2 warps)
+// ------------------------------------------------------------------ patch producers (3 warps)
 // Granule = (phase plane, stream position, group of up to 4 channel words).
 constexpr int kGranBatch = 4;
 
@@ -359,11 +446,14 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
   int pb = 0;
   uint32_t pph = 1;
   bool ok = true;
+  TR_DECL(pt < 32);
+  TR_T0;
   for (int tile = tile0; tile <= tile1 && ok; ++tile) {
-    ok = mbar_wait(S.pempty + 8u * pb, pph, S.abort_flag, &g_status_tc);
+    ok = mbar_wait_relaxed(S.pempty + 8u * pb, pph, S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
+    TR_ADD(0);
     if (!ok) break;
     const uint32_t patch = S.patch + (uint32_t)pb * P.patch_bytes;
-    const long long m0 = (long long)tile * kTileM;
+    const uint32_t m0 = (uint32_t)tile * kTileM;
     for (int g0 = pt; g0 < ngran; g0 += kPatThreads * kGranBatch) {
       uint32_t wv[kGranBatch][4];
       uint32_t dst[kGranBatch];
@@ -381,12 +471,12 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
           const int w0 = wg * 4;
           w0s[b] = w0;
           dst[b] = patch + (uint32_t)(phase * P.Cw + w0) * plane_bytes + (uint32_t)q * 16u;
-          const long long sq = m0 + q;
-          if (sq < P.L) {
-            const long long r = sq / P.Wq;
-            const int c = (int)(sq - r * P.Wq);
-            const long long n = r / P.Hq;
-            const int ry = (int)(r - n * P.Hq);
+          const uint32_t sq = m0 + (uint32_t)q;
+          if (sq < (uint32_t)P.L) {
+            const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
+            const int c = (int)(sq - r * (uint32_t)P.Wq);
+            const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
+            const int ry = (int)(r - n * (uint32_t)P.Hq);
             const int py = phase / s, px = phase - py * s;
             const int iy = (ry - P.leadY) * s + py, ix = (c - P.leadX) * s + px;
             if (ry >= P.leadY && c >= P.leadX && iy < P.H && ix < P.W) {
@@ -427,23 +517,22 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
         }
       }
     }
+    TR_ADD(1);
     fence_proxy_async();
     __syncwarp();
     if (lane == 0) mbar_arrive(S.pfull + 8u * pb);
     if (++pb == P.npb) { pb = 0; pph ^= 1u; }
   }
+  TR_FLUSH(16);
 }
 
 // ------------------------------------------------------------------ epilogue (8 warps)
-// Warp w reads tensor-memory lanes 32 (w & 3) .. +31 (pixels) and one half of the
-// slab's columns (filters).  Lane = pixel, so for one filter a warp stores 32
+// Warp w reads tensor-memory lanes 32 w .. +31 (pixels), all the slab's columns (filters).  Lane = pixel, so for one filter a warp stores 32
 // consecutive stream pixels: a contiguous run of the NCHW output row.
 __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, long long i1,
                               uint32_t tmem_base, int warp, int lane) {
-  const int quarter = warp & 3, half = warp >> 2;
-  const int nblk = P.NT / 16;
-  const int b_begin = half == 0 ? 0 : (nblk + 1) / 2;
-  const int b_end = half == 0 ? (nblk + 1) / 2 : nblk;
+  const int quarter = warp;
+  const int b_begin = 0, b_end = P.NT / 16;
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tile = (int)(i0 / P.nslabs), slab = (int)(i0 - (long long)tile * P.nslabs);
@@ -451,15 +540,17 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   float kv = 0.0f;
   size_t obase = 0;                       // offset of (image, filter 0, pixel)
   long long k = 0;
+  TR_DECL(warp == 0);
+  TR_T0;
   for (long long item = i0; item < i1 && ok; ++item, ++k) {
     if (new_tile) {
-      const long long m = (long long)tile * kTileM + quarter * 32 + lane;
-      valid = m < P.L;
+      const uint32_t m = (uint32_t)tile * kTileM + (uint32_t)(quarter * 32 + lane);
+      valid = m < (uint32_t)P.L;
       if (valid) {
-        const long long r = m / P.Wq;
-        const int ox = (int)(m - r * P.Wq);
-        const long long n = r / P.Hq;
-        const int oy = (int)(r - n * P.Hq);
+        const uint32_t r = fast_div(m, P.div_wq_m, P.div_wq_s);
+        const int ox = (int)(m - r * (uint32_t)P.Wq);
+        const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
+        const int oy = (int)(r - n * (uint32_t)P.Hq);
         valid = ox < P.Wo && oy < P.Ho;
         if (valid) {
           const size_t pix = (size_t)oy * P.Wo + ox;
@@ -470,7 +561,9 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     }
     const int ab = (int)(k % P.nacc);
     const uint32_t use = (uint32_t)(k / P.nacc);
-    ok = mbar_wait(S.afull + 8u * ab, use & 1u, S.abort_flag, &g_status_tc);
+    TR_ADD(0);
+    ok = mbar_wait_relaxed(S.afull + 8u * ab, use & 1u, S.abort_flag, &g_status_tc, XNOR_SLEEP_EPI);
+    TR_ADD(1);
     if (!ok) break;
     tc_fence_after();
     const uint32_t t_acc = t_lane + (uint32_t)(ab * P.NT);
@@ -548,10 +641,13 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     }
     new_tile = false;
     if (++slab == P.nslabs) { slab = 0; ++tile; new_tile = true; }
+    TR_ADD(2);
   }
+  TR_FLUSH(24);
 }
 
-__global__ void __launch_bounds__(kThreads, 1) binconv_tc_kernel(const TcParams P) {
+__global__ void __launch_bounds__(kThreads, 1)
+binconv_tc_kernel(const __grid_constant__ TcParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Smem S = carve(smem, P);
@@ -577,15 +673,6 @@ __global__ void __launch_bounds__(kThreads, 1) binconv_tc_kernel(const TcParams 
                  ::"r"(smem_u32(S.tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // the table of K-steps, once per CTA
-  {
-    KStep *table = reinterpret_cast<KStep *>(smem + P.off_table);
-    for (int j = tid; j < P.nsteps; j += kThreads) {
-      KStep ks;
-      build_kstep(P, j, ks);
-      table[j] = ks;
-    }
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -610,7 +697,7 @@ __global__ void __launch_bounds__(kThreads, 1) binconv_tc_kernel(const TcParams 
   const long long i1 = total * (blockIdx.x + 1) / gridDim.x;
   if (i0 < i1) {
     if (warp < kEpiWarps) epilogue_role(P, S, i0, i1, tmem_base, warp, lane);
-    else if (warp == kMmaWarp) mma_role(P, S, i0, i1, tmem_base, lane);
+    else if (warp == kMmaWarp) mma_role(P, S, i0, i1, tmem_base);
     else if (warp < kPatWarp0) weight_role(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
     else patch_role(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
   }
@@ -658,21 +745,20 @@ Plan make_plan(const ConvGeom &g) {
   P.NT = ((g.Co + P.nslabs - 1) / P.nslabs + 15) / 16 * 16;
   P.nacc = 2 * P.NT <= kMaxAccCols ? 2 : 1;
   // K-steps
-  const int taps = g.kh * g.kw, h = g.Cw / 2;
-  P.nsteps = (g.Cw % 2 == 0) ? taps * h : (taps / 2) * (2 * h + 1) + (taps % 2) * (h + 1);
-  if (P.nsteps < 1 || P.nsteps > kMaxSteps) return pl;
-  // weight-thread mapping: rows_mod threads cover the rows, the other thread groups take
-  // other K-steps of the stage
+  P.row_words = g.kh * g.kw * g.Cw;
+  P.nsteps = (P.row_words + 1) / 2;
+  if (P.nsteps > kMaxSteps) return pl;
+  // weight-thread mapping: rows_mod threads cover the rows of a K-step, the other thread
+  // groups take other K-steps of the stage; a stage is about 16 KB of expanded weights
   int ntp = 16;
   while (ntp < P.NT) ntp *= 2;                          // 16 .. 256
-  P.rows_mod = std::min(ntp, 128);
-  const int groups = kWgtThreads / P.rows_mod;          // 1, 2, 4, 8
+  P.rows_mod = ntp;
+  const int groups = kWgtThreads / P.rows_mod;          // 1 .. 16
   P.mps = std::max(2, std::min(8, 512 / ntp));
-  P.grp_steps = P.mps / groups;                         // 2 (x2 rows), 4, 4, 2, 1
+  P.grp_steps = std::max(1, P.mps / groups);            // 2, 2, 2, 1, 1
   P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NT * 32u;
-  // shared memory: control, table, weight ring, patch buffers
-  P.off_table = (uint32_t)kCtrlBytes;
-  P.off_ring = (uint32_t)((P.off_table + (size_t)P.nsteps * sizeof(KStep) + 127) / 128 * 128);
+  // shared memory: control, weight ring, patch buffers
+  P.off_ring = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
   const size_t avail = kSmemMax - P.off_ring;
   if ((size_t)P.patch_bytes + 2 * (size_t)P.stage_bytes > avail) return pl;
   // at least 2 stages and 1 patch; then patches up to 3, stages up to 6, one more patch
@@ -692,6 +778,20 @@ Plan make_plan(const ConvGeom &g) {
             ((uint32_t)(kTileM >> 4) << 24);
   const int crem = g.C - 32 * (g.Cw - 1);
   P.tail_mask = crem == 32 ? 0xFFFFFFFFu : ((1u << crem) - 1u);
+  for (int j = 0; j < 32; ++j) P.swap_mask[j] = 0u;
+  for (int j = 0; j < P.nsteps; ++j) {
+    bool swap;
+    P.adesc_lo[j] = kstep_desc(P, j, &swap);
+    if (swap) P.swap_mask[j >> 5] |= 1u << (j & 31);
+  }
+  auto magic = [](uint32_t d, uint32_t *m, int *sh) {
+    int l = 0;
+    while ((1u << l) < d) ++l;
+    *sh = l;
+    *m = (uint32_t)((((unsigned long long)1 << (31 + l)) + d - 1) / d);
+  };
+  magic((uint32_t)P.Wq, &P.div_wq_m, &P.div_wq_s);
+  magic((uint32_t)P.Hq, &P.div_hq_m, &P.div_hq_s);
   pl.ok = true;
   return pl;
 }
@@ -733,8 +833,19 @@ cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const floa
   const int sms = sm_count_cached();
   const unsigned grid = (unsigned)std::min<long long>(total, sms);
   binconv_tc_kernel<<<grid, kThreads, pl.smem, st>>>(P);
-  return cudaGetLastError();
+  { cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess && getenv("XNOR_DEBUG")) fprintf(stderr, "binconv_tc launch: %s (grid %u, smem %zu)\n", cudaGetErrorString(e_), grid, pl.smem); return e_; }
 }
+
+#ifdef XNOR_TRACE
+extern "C" int xnor_debug_trace_tc(long long *host64, int clear) {
+  cudaError_t e = cudaMemcpyFromSymbol(host64, g_tc_trace, sizeof(long long) * 64);
+  if (clear) {
+    long long z[64] = {};
+    cudaMemcpyToSymbol(g_tc_trace, z, sizeof(z));
+  }
+  return (int)e;
+}
+#endif
 
 cudaError_t read_status_tc(int *status) {
   cudaError_t e = cudaMemcpyFromSymbol(status, g_status_tc, sizeof(int));

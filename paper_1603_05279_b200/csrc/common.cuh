@@ -21,6 +21,14 @@ inline ConvGeom make_geom(const xnor_conv_desc &d) {
   return g;
 }
 
+// Packed weights are stored word-pair-major so that the convolution kernels read them
+// coalesced: with f = tap * Cw + cw the index of a word inside a filter (tap = ky * k_w + kx),
+// word f of filter co is element ((f / 2) * C_out + co) * 2 + f % 2.  Words 2j and 2j+1 of all
+// filters (one 64-channel step of the contraction) are contiguous.
+__host__ __device__ inline size_t packed_weight_index(int Co, int co, int f) {
+  return ((size_t)(f >> 1) * Co + co) * 2 + (f & 1);
+}
+
 // Launchers: return the cudaError_t of the launch (cudaGetLastError, cleared).
 cudaError_t launch_binarize_weights(const float *w, int Co, int C, int kh, int kw,
                                     uint32_t *w_packed, float *alpha, cudaStream_t st);

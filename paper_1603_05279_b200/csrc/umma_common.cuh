@@ -52,6 +52,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// Same, for roles that can afford a slower wake-up: between polls the thread sleeps, which
+// leaves the issue slots of its scheduler to the warps that have work.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
+                                                  volatile int *abort_flag, int *status_word,
+                                                  unsigned sleep_ns) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i) {
+      __nanosleep(sleep_ns);
+      if (mbar_try(bar, parity)) return true;
+    }
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      atomicExch(status_word, (int)XNOR_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }

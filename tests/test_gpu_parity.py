@@ -57,7 +57,7 @@ def check_block(oracle, x, w, stride, pad, scale=None, shift=None, residual=None
     g = gpu_block(x, w, stride, pad, scale, shift, residual, engine, alias_residual)
     r = oracle.xnor_block(x, w, stride, pad, scale, shift, residual)
     C = x.shape[1]
-    assert np.array_equal(unpack_weights(g["wp"], C), r.B), "sign(W) bits"
+    assert np.array_equal(unpack_weights(g["wp"], C, w.shape[2], w.shape[3]), r.B), "sign(W) bits"
     assert np.array_equal(unpack_activations(g["xp"], C), r.H), "sign(I) bits"
     assert_close(g["alpha"], r.alpha, "alpha")
     assert_close(g["A"], r.A, "A")

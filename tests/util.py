@@ -19,9 +19,18 @@ def unpack_activations(x_packed, C):
     return np.ascontiguousarray(unpack_bits(x_packed, C).transpose(0, 3, 1, 2))
 
 
-def unpack_weights(w_packed, C):
-    """[Co][kh][kw][Cw] words -> +-1 [Co][C][kh][kw]."""
-    return np.ascontiguousarray(unpack_bits(w_packed, C).transpose(0, 3, 1, 2))
+def unpack_weights(w_packed, C, kh, kw):
+    """Word-pair-major words [pairs][Co][2] -> +-1 [Co][C][kh][kw].  Word f = (ky*kw + kx)*Cw + cw
+    of filter co is element [f // 2][co][f % 2]; an odd word count is padded with a 0 word."""
+    w = np.ascontiguousarray(w_packed)
+    pairs, Co, _ = w.shape
+    Cw = (C + 31) // 32
+    nwords = kh * kw * Cw
+    assert pairs == (nwords + 1) // 2
+    flat = w.transpose(1, 0, 2).reshape(Co, pairs * 2)
+    assert not flat[:, nwords:].any(), "padding word must be 0"
+    words = np.ascontiguousarray(flat[:, :nwords]).reshape(Co, kh, kw, Cw)
+    return np.ascontiguousarray(unpack_bits(words, C).transpose(0, 3, 1, 2))
 
 
 def assert_close(gpu, ref, what, rel=REL_TOL):
