@@ -358,7 +358,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     du.init("nccl", local)
     X.load()
-    X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2, "umma_i8": 3}[args.engine])
+    X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2}[args.engine])
     stream = torch.cuda.current_stream()
 
     # every rank has its own batch (weak scaling, no exchange on the data path)
@@ -445,7 +445,7 @@ def run_ours(args):
         # tensor-core peak for the operand type in use = measured bf16 peak x the nominal
         # ratio of that type to bf16 (e2m1: 9 / 2.25 = 4, int8: 2); the sustained figure,
         # because the kernel is timed inside a long step.  2 flops per 1-bit MAC.
-        ratio, kind = (2, "int8") if engine == "umma_i8" else (4, "e2m1 (fp4)")
+        ratio, kind = 4, "e2m1 (fp4)"
         roofline = {"kernel": "BinConv tensor-core kernel (one launch per layer, %d per step)"
                               % n_conv, "bound": "tensor",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12,
@@ -483,8 +483,6 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": ("u32 bit words (XOR+popcount), int32 sums, fp32 scaling" if engine == "popc"
-                  else "int8 +-1/0 tensor-core operands from 1-bit words, int32 sums, fp32 scaling"
-                  if engine == "umma_i8"
                   else "e2m1 (fp4) tensor-core operands from 1-bit words, exact integer sums in "
                        "fp32, fp32 scaling"),
         "data": "synthetic",
@@ -519,7 +517,7 @@ def main():
     ap.add_argument("--ref-images", type=int, default=8,
                     help="images per layer per step of the reference (oracle) arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_i8"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma"])
     ap.add_argument("--workload", default="alexnet", choices=sorted(WORKLOAD_NAMES),
                     help="shape set (the bench line proper is the default, alexnet)")
     ap.add_argument("--layers", default="",

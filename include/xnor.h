@@ -188,20 +188,17 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
 
 /*
  * Which BinConv engine xnor_conv2d_forward uses.  XNOR_ENGINE_AUTO (default)
- * picks by shape: the tensor-core engine where it applies (stride 1), else
- * the CUDA-core one.  Process-wide; meant for tests and measurements.  With an
- * engine forced, xnor_conv2d_forward returns UNSUPPORTED for shapes that
- * engine does not cover.
- *   XNOR_ENGINE_POPC     CUDA-core XOR + population count, any supported shape
- *   XNOR_ENGINE_UMMA     5th-generation tensor cores, 4-bit (e2m1) operands built
- *                        from the sign bits, exact fp32 accumulation of integers
- *   XNOR_ENGINE_UMMA_I8  same, int8 operands and int32 accumulation (the slower
- *                        alternative, kept for comparison)
+ * picks by shape: the tensor-core engine where it applies, else the CUDA-core
+ * one.  Process-wide; meant for tests and measurements.  With an engine
+ * forced, xnor_conv2d_forward returns UNSUPPORTED for shapes that engine does
+ * not cover.
+ *   XNOR_ENGINE_POPC   CUDA-core XOR + population count, any supported shape
+ *   XNOR_ENGINE_UMMA   5th-generation tensor cores (tcgen05), 4-bit (e2m1)
+ *                      operands built from the sign bits, exact fp32
+ *                      accumulation of integers; strides 1 and 2, shapes whose
+ *                      activation patch fits shared memory
  */
-typedef enum {
-  XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2, XNOR_ENGINE_UMMA_I8 = 3,
-  XNOR_ENGINE_TC = 4
-} xnor_engine;
+typedef enum { XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2 } xnor_engine;
 xnor_status xnor_set_engine(xnor_engine e);
 xnor_engine xnor_get_engine(void);
 

@@ -45,8 +45,7 @@ int xnor_out_extent(int in, int k, int stride, int pad) {
 }
 
 xnor_status xnor_set_engine(xnor_engine e) {
-  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC && e != XNOR_ENGINE_UMMA &&
-      e != XNOR_ENGINE_UMMA_I8 && e != XNOR_ENGINE_TC)
+  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC && e != XNOR_ENGINE_UMMA)
     return XNOR_ERR_INVALID_ARG;
   g_engine = e;
   return XNOR_OK;
@@ -105,34 +104,23 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
   if ((long long)d->C_in * d->k_h * d->k_w >= (1LL << 24)) return XNOR_ERR_UNSUPPORTED;
   const xnor::ConvGeom g = xnor::make_geom(*d);
   const cudaStream_t st = (cudaStream_t)cuda_stream;
-  if (g_engine == XNOR_ENGINE_UMMA_I8) {
-    if (!xnor::umma_i8_supported(g)) return XNOR_ERR_UNSUPPORTED;
-    return from_cuda(xnor::launch_binconv_i8(x_packed, w_packed, alpha, K, residual, g, out,
-                                             acc_out, st));
-  }
   const bool tc_ok = xnor::umma_tc_supported(g);
-  if (g_engine == XNOR_ENGINE_TC && !tc_ok) return XNOR_ERR_UNSUPPORTED;
-  if ((g_engine == XNOR_ENGINE_TC || g_engine == XNOR_ENGINE_AUTO) && tc_ok)
+  if (g_engine == XNOR_ENGINE_UMMA && !tc_ok) return XNOR_ERR_UNSUPPORTED;
+  if (g_engine != XNOR_ENGINE_POPC && tc_ok)
     return from_cuda(xnor::launch_binconv_tc(x_packed, w_packed, alpha, K, residual, g, out,
                                              acc_out, st));
-  const bool fp4_ok = xnor::umma_fp4_supported(g);
-  if (g_engine == XNOR_ENGINE_UMMA && !fp4_ok) return XNOR_ERR_UNSUPPORTED;
-  if (g_engine != XNOR_ENGINE_POPC && fp4_ok)
-    return from_cuda(xnor::launch_binconv_fp4(x_packed, w_packed, alpha, K, residual, g, out,
-                                              acc_out, st));
   return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, out,
                                              acc_out, (cudaStream_t)cuda_stream));
 }
 
 xnor_status xnor_check_device(void *cuda_stream) {
-  int s4 = 0, s8 = 0, st = 0;
+  int st = 0;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess ||
-      xnor::read_status_fp4(&s4) != cudaSuccess || xnor::read_status_i8(&s8) != cudaSuccess ||
       xnor::read_status_tc(&st) != cudaSuccess) {
     (void)cudaGetLastError();
     return XNOR_ERR_CUDA;
   }
-  return (s4 == 0 && s8 == 0 && st == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
+  return st == 0 ? XNOR_OK : XNOR_ERR_TIMEOUT;
 }
 
 xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,

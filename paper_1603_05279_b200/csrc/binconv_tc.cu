@@ -87,7 +87,7 @@ using namespace umma;
 constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
 constexpr int kWgtWarp0 = 5, kWgtWarps = 8, kWgtThreads = 32 * kWgtWarps;
-constexpr int kPatWarp0 = 13, kPatWarps = 3, kPatThreads = 32 * kPatWarps;
+constexpr int kPatWarp0 = 13, kPatWarps = 3;
 constexpr int kThreads = 32 * (kPatWarp0 + kPatWarps);     // 512: 16 warps, 128 registers each
 constexpr int kTileM = 128;          // stream positions per tile = tensor-memory lanes
 constexpr int kTmemCols = 512;
@@ -383,135 +383,138 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
   uint32_t wph = 1;           // parity to wait for on the empty barriers
   bool ok = true;
   const uint32_t row_off = (uint32_t)row * 16u;
+#pragma unroll 1
   while (cc.item < i1 && ok) {
+    ok = mbar_wait(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc);
+    TR_ADD(0);
+    if (!ok) break;
+    const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
+    const int co = cc.slab * P.NT + row;
+    const int jj0 = grp * gs;
+    const int j0 = cc.st * P.mps + jj0;
+    const bool on = grp_on && co < P.Co;
+    uint32_t v0[kUnits][4], v1[kUnits][4], a0[kUnits], a1[kUnits];
 #pragma unroll
-    for (int d = 0; d < kPrefetch; ++d) {
-      if (cc.item < i1 && ok) {
-        ok = mbar_wait(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc);
-        TR_ADD(0);
-        if (ok) {
-          const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
-          const int co = cc.slab * P.NT + row;
-          const int jj0 = grp * gs;
-          const int j0 = cc.st * P.mps + jj0;
-          const bool on = grp_on && co < P.Co;
-          uint32_t v0[kUnits][4], v1[kUnits][4], a0[kUnits], a1[kUnits];
+    for (int u = 0; u < kUnits; ++u) {
+      const int j = j0 + u;
+      const bool swap = (P.swap_mask[(j >> 5) & 31] >> (j & 31)) & 1u;
+      const uint32_t keep = 2 * j + 1 < P.row_words ? 0xFFFFFFFFu : 0u;  // lone: partner 0
+      expand_signs<false>(pf[0][u].x, v0[u]);
+      expand_signs<false>(pf[0][u].y, v1[u]);
+      v1[u][0] &= keep; v1[u][1] &= keep; v1[u][2] &= keep; v1[u][3] &= keep;
+      const uint32_t a = stage + (uint32_t)(2 * (jj0 + u)) * b_lbo;
+      a0[u] = swap ? a + b_lbo : a;
+      a1[u] = swap ? a : a + b_lbo;
+    }
 #pragma unroll
-          for (int u = 0; u < kUnits; ++u) {
-            const int j = j0 + u;
-            const bool swap = (P.swap_mask[(j >> 5) & 31] >> (j & 31)) & 1u;
-            const uint32_t keep = 2 * j + 1 < P.row_words ? 0xFFFFFFFFu : 0u;  // lone: partner 0
-            expand_signs<false>(pf[d][u].x, v0[u]);
-            expand_signs<false>(pf[d][u].y, v1[u]);
-            v1[u][0] &= keep; v1[u][1] &= keep; v1[u][2] &= keep; v1[u][3] &= keep;
-            const uint32_t a = stage + (uint32_t)(2 * (jj0 + u)) * b_lbo;
-            a0[u] = swap ? a + b_lbo : a;
-            a1[u] = swap ? a : a + b_lbo;
-          }
-#pragma unroll
-          for (int u = 0; u < kUnits; ++u) {
-            if (on && u < gs && j0 + u < P.nsteps) {
-              sts128(a0[u], v0[u][0], v0[u][1], v0[u][2], v0[u][3]);
-              sts128(a1[u], v1[u][0], v1[u][1], v1[u][2], v1[u][3]);
-            }
-          }
-          TR_ADD(1);
-          fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(S.wfull + 8u * ws);
-          if (++ws == P.stages) { ws = 0; wph ^= 1u; }
-          advance(cc);
-          fetch(pf[d], fc);
-          advance(fc);
-          TR_ADD(2);
-        }
+    for (int u = 0; u < kUnits; ++u) {
+      if (on && u < gs && j0 + u < P.nsteps) {
+        sts128(a0[u], v0[u][0], v0[u][1], v0[u][2], v0[u][3]);
+        sts128(a1[u], v1[u][0], v1[u][1], v1[u][2], v1[u][3]);
       }
     }
+    TR_ADD(1);
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(S.wfull + 8u * ws);
+    if (++ws == P.stages) { ws = 0; wph ^= 1u; }
+    advance(cc);
+    // the queue of packed words moves up one stage; the freed slot is refilled
+#pragma unroll
+    for (int d = 0; d + 1 < kPrefetch; ++d)
+#pragma unroll
+      for (int u = 0; u < kUnits; ++u) pf[d][u] = pf[d + 1][u];
+    fetch(pf[kPrefetch - 1], fc);
+    advance(fc);
+    TR_ADD(2);
   }
   TR_FLUSH(8);
 }
 
 // ------------------------------------------------------------------ patch producers (3 warps)
-// Granule = (phase plane, stream position, group of up to 4 channel words).
-constexpr int kGranBatch = 4;
+// Each warp expands whole tiles on its own (warp p takes this CTA's tiles p, p + 3, ...), so
+// the global-load latency of up to three tiles overlaps; a tile's patch buffer is its index
+// modulo the number of buffers.  For every (phase plane, group of up to 4 channel words) a
+// lane walks the patch's stream positions, kPosBatch of them in flight at a time.
+constexpr int kPosBatch = 2;
 
 __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long long i1, int pt,
                            int lane) {
   const int tile0 = (int)(i0 / P.nslabs), tile1 = (int)((i1 - 1) / P.nslabs);
   const int s = P.stride, phases = s * s;
-  const int wgroups = (P.Cw + 3) >> 2;
-  const int ngran = phases * P.ppix * wgroups;
   const uint32_t plane_bytes = (uint32_t)P.ppix * 16u;
   const bool vec = (P.Cw & 3) == 0;
-  int pb = 0;
-  uint32_t pph = 1;
+  const int pw = pt >> 5;                       // patch warp 0..2
+  // nibble masks of the channel tail, one per expanded register
+  uint32_t tm[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) tm[r] = ((P.tail_mask >> r) & 0x11111111u) * 0xFu;
   bool ok = true;
   TR_DECL(pt < 32);
   TR_T0;
-  for (int tile = tile0; tile <= tile1 && ok; ++tile) {
+#pragma unroll 1
+  for (int tile = tile0 + pw; tile <= tile1 && ok; tile += kPatWarps) {
+    const int seq = tile - tile0;               // this CTA's tiles in order
+    const int pb = seq % P.npb;
+    const uint32_t pph = ((uint32_t)(seq / P.npb) & 1u) ^ 1u;
     ok = mbar_wait_relaxed(S.pempty + 8u * pb, pph, S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
     TR_ADD(0);
     if (!ok) break;
     const uint32_t patch = S.patch + (uint32_t)pb * P.patch_bytes;
     const uint32_t m0 = (uint32_t)tile * kTileM;
-    for (int g0 = pt; g0 < ngran; g0 += kPatThreads * kGranBatch) {
-      uint32_t wv[kGranBatch][4];
-      uint32_t dst[kGranBatch];
-      int w0s[kGranBatch];
+#pragma unroll 1
+    for (int phase = 0; phase < phases; ++phase) {
+      const int py = phase / s, px = phase - py * s;
+#pragma unroll 1
+      for (int w0 = 0; w0 < P.Cw; w0 += 4) {
+        const uint32_t dst0 = patch + (uint32_t)(phase * P.Cw + w0) * plane_bytes;
+        const bool has_tail = w0 + 4 >= P.Cw;   // this group holds the last word
+#pragma unroll 1
+        for (int q0 = lane; q0 < P.ppix; q0 += 32 * kPosBatch) {
+          uint32_t wv[kPosBatch][4];
+          bool real[kPosBatch];
 #pragma unroll
-      for (int b = 0; b < kGranBatch; ++b) {
-        const int g = g0 + b * kPatThreads;
-        wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
-        dst[b] = 0u;
-        w0s[b] = -1;
-        if (g < ngran) {
-          // g = (phase * wgroups + wg) * ppix + q : consecutive threads take consecutive pixels
-          const int pw = g / P.ppix, q = g - pw * P.ppix;
-          const int phase = pw / wgroups, wg = pw - phase * wgroups;
-          const int w0 = wg * 4;
-          w0s[b] = w0;
-          dst[b] = patch + (uint32_t)(phase * P.Cw + w0) * plane_bytes + (uint32_t)q * 16u;
-          const uint32_t sq = m0 + (uint32_t)q;
-          if (sq < (uint32_t)P.L) {
-            const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
-            const int c = (int)(sq - r * (uint32_t)P.Wq);
-            const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
-            const int ry = (int)(r - n * (uint32_t)P.Hq);
-            const int py = phase / s, px = phase - py * s;
-            const int iy = (ry - P.leadY) * s + py, ix = (c - P.leadX) * s + px;
-            if (ry >= P.leadY && c >= P.leadX && iy < P.H && ix < P.W) {
-              const uint32_t *src = P.xp + (((size_t)n * P.H + iy) * P.W + ix) * P.Cw + w0;
-              if (vec) {
-                const uint4 t = __ldg(reinterpret_cast<const uint4 *>(src));
-                wv[b][0] = t.x; wv[b][1] = t.y; wv[b][2] = t.z; wv[b][3] = t.w;
-              } else {
+          for (int b = 0; b < kPosBatch; ++b) {
+            const int q = q0 + 32 * b;
+            wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
+            real[b] = false;
+            const uint32_t sq = m0 + (uint32_t)q;
+            if (q < P.ppix && sq < (uint32_t)P.L) {
+              const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
+              const int c = (int)(sq - r * (uint32_t)P.Wq);
+              const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
+              const int ry = (int)(r - n * (uint32_t)P.Hq);
+              const int iy = (ry - P.leadY) * s + py, ix = (c - P.leadX) * s + px;
+              if (ry >= P.leadY && c >= P.leadX && iy < P.H && ix < P.W) {
+                const uint32_t *src = P.xp + (((size_t)n * P.H + iy) * P.W + ix) * P.Cw + w0;
+                real[b] = true;
+                if (vec) {
+                  const uint4 t = __ldg(reinterpret_cast<const uint4 *>(src));
+                  wv[b][0] = t.x; wv[b][1] = t.y; wv[b][2] = t.z; wv[b][3] = t.w;
+                } else {
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  if (w0 + i < P.Cw) wv[b][i] = __ldg(src + i);
-              }
-              w0s[b] = w0 | 0x40000000;      // marks a real pixel
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int b = 0; b < kGranBatch; ++b) {
-        if (w0s[b] >= 0) {
-          const bool real = (w0s[b] & 0x40000000) != 0;
-          const int w0 = w0s[b] & 0xFFFF;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            if (w0 + i < P.Cw) {
-              uint32_t v[4] = {0u, 0u, 0u, 0u};
-              if (real) {
-                expand_signs<true>(wv[b][i], v);
-                if (w0 + i == P.Cw - 1 && P.tail_mask != 0xFFFFFFFFu) {
-                  // channels beyond C_in are the value 0
-#pragma unroll
-                  for (int r = 0; r < 4; ++r) v[r] &= ((P.tail_mask >> r) & 0x11111111u) * 0xFu;
+                  for (int i = 0; i < 4; ++i)
+                    if (w0 + i < P.Cw) wv[b][i] = __ldg(src + i);
                 }
               }
-              sts128(dst[b] + (uint32_t)i * plane_bytes, v[0], v[1], v[2], v[3]);
+            }
+          }
+#pragma unroll
+          for (int b = 0; b < kPosBatch; ++b) {
+            const int q = q0 + 32 * b;
+            if (q < P.ppix) {
+              const uint32_t keep = real[b] ? 0xFFFFFFFFu : 0u;    // padding expands to 0
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                if (w0 + i < P.Cw) {
+                  uint32_t v[4];
+                  expand_signs<true>(wv[b][i], v);
+                  const bool last = has_tail && w0 + i == P.Cw - 1;   // channels beyond C_in are 0
+#pragma unroll
+                  for (int r = 0; r < 4; ++r) v[r] &= last ? (tm[r] & keep) : keep;
+                  sts128(dst0 + (uint32_t)i * plane_bytes + (uint32_t)q * 16u, v[0], v[1], v[2], v[3]);
+                }
+              }
             }
           }
         }
@@ -521,18 +524,18 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     fence_proxy_async();
     __syncwarp();
     if (lane == 0) mbar_arrive(S.pfull + 8u * pb);
-    if (++pb == P.npb) { pb = 0; pph ^= 1u; }
   }
   TR_FLUSH(16);
 }
 
-// ------------------------------------------------------------------ epilogue (8 warps)
-// Warp w reads tensor-memory lanes 32 w .. +31 (pixels), all the slab's columns (filters).  Lane = pixel, so for one filter a warp stores 32
-// consecutive stream pixels: a contiguous run of the NCHW output row.
+// ------------------------------------------------------------------ epilogue (4 warps)
+// Warp w reads tensor-memory lanes 32 w .. +31 (pixels), all the slab's columns (filters).
+// Lane = pixel, so for one filter a warp stores 32 consecutive stream pixels: a contiguous
+// run of the NCHW output row.
 __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, long long i1,
                               uint32_t tmem_base, int warp, int lane) {
   const int quarter = warp;
-  const int b_begin = 0, b_end = P.NT / 16;
+  const int b_end = P.NT / 16;
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tile = (int)(i0 / P.nslabs), slab = (int)(i0 - (long long)tile * P.nslabs);
@@ -605,39 +608,23 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       }
     };
 
-    // two register sets: the load of the next 16 columns is in flight while the
-    // current 16 are scaled and stored
-    int32_t ra[16], rb[16];
-    if (b_begin < b_end) {
-      tmem_ld16(t_acc + (uint32_t)(b_begin * 16), ra);
-      tmem_wait16(ra);
-    }
-    for (int b = b_begin; b < b_end; b += 2) {
-      const bool more1 = b + 1 < b_end, more2 = b + 2 < b_end;
-      if (more1) tmem_ld16(t_acc + (uint32_t)((b + 1) * 16), rb);
-      else {                                     // ra was the last load: release the buffer
+    // One copy of the code: the next 16 columns are being loaded into `nx` while the
+    // current 16 (copied out to `cur`) are scaled and stored.
+    int32_t nx[16], cur[16];
+    tmem_ld16(t_acc, nx);
+#pragma unroll 1
+    for (int b = 0; b < b_end; ++b) {
+      tmem_wait16(nx);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) cur[j] = nx[j];
+      if (b + 1 < b_end) {
+        tmem_ld16(t_acc + (uint32_t)((b + 1) * 16), nx);
+      } else {                                   // that was the last load: release the buffer
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
       }
-      emit(b, ra);
-      if (more1) {
-        tmem_wait16(rb);
-        if (more2) {
-          tmem_ld16(t_acc + (uint32_t)((b + 2) * 16), ra);
-        } else {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
-        }
-        emit(b + 1, rb);
-        if (more2) tmem_wait16(ra);
-      }
-    }
-    if (b_begin >= b_end) {                      // a warp with no columns still releases
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
+      emit(b, cur);
     }
     new_tile = false;
     if (++slab == P.nslabs) { slab = 0; ++tile; new_tile = true; }
@@ -658,7 +645,7 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
       mbar_init(S.wempty + 8u * i, 1);
     }
     for (int i = 0; i < kMaxPatchBufs; ++i) {
-      mbar_init(S.pfull + 8u * i, kPatWarps);
+      mbar_init(S.pfull + 8u * i, 1);
       mbar_init(S.pempty + 8u * i, 1);
     }
     for (int i = 0; i < 2; ++i) {

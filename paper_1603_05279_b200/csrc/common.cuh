@@ -43,24 +43,13 @@ cudaError_t launch_binactiv_static(const float *x, const float *scale, const flo
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st);
-// Tensor-core engines (stride 1): 4-bit operands (default) and int8 operands.
-bool umma_fp4_supported(const ConvGeom &g);
-cudaError_t launch_binconv_fp4(const uint32_t *xp, const uint32_t *wp, const float *alpha,
-                               const float *K, const float *residual, const ConvGeom &g,
-                               float *out, int32_t *acc_out, cudaStream_t st);
-bool umma_i8_supported(const ConvGeom &g);
-cudaError_t launch_binconv_i8(const uint32_t *xp, const uint32_t *wp, const float *alpha,
-                              const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, cudaStream_t st);
 // Persistent tensor-core engine (strides 1 and 2).
 bool umma_tc_supported(const ConvGeom &g);
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
                               float *out, int32_t *acc_out, cudaStream_t st);
+// Reads (and clears if set) the device status word of the tensor-core kernel.
 cudaError_t read_status_tc(int *status);
-// Read (and clear if set) the device status word of each tensor-core kernel.
-cudaError_t read_status_fp4(int *status);
-cudaError_t read_status_i8(int *status);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,
                                     int Co, int stride, float *out, cudaStream_t st);
 

@@ -35,9 +35,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false when the wait expired (XNOR_ERR_TIMEOUT is then
 // recorded in *status_word and the CTA-wide abort flag is raised) or when
 // another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          int *status_word) {
-  if (mbar_try(bar, parity)) return true;
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity,
+                                            volatile int *abort_flag, int *status_word) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
@@ -52,12 +51,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int *status_word) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status_word);
+}
+
 // Same, for roles that can afford a slower wake-up: between polls the thread sleeps, which
 // leaves the issue slots of its scheduler to the warps that have work.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
-                                                  volatile int *abort_flag, int *status_word,
-                                                  unsigned sleep_ns) {
-  if (mbar_try(bar, parity)) return true;
+static __device__ __noinline__ bool mbar_wait_relaxed_slow(uint32_t bar, uint32_t parity,
+                                                    volatile int *abort_flag, int *status_word,
+                                                    unsigned sleep_ns) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
@@ -72,6 +76,13 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
       return false;
     }
   }
+}
+
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
+                                                  volatile int *abort_flag, int *status_word,
+                                                  unsigned sleep_ns) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_relaxed_slow(bar, parity, abort_flag, status_word, sleep_ns);
 }
 
 __device__ __forceinline__ void fence_proxy_async() {

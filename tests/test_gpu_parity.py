@@ -12,9 +12,7 @@ from util import REL_TOL, assert_close, dev, host, unpack_activations, unpack_we
 
 pytestmark = pytest.mark.gpu
 
-ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_I8, B.XNOR_ENGINE_TC,
-           B.XNOR_ENGINE_AUTO]
-TENSOR_ENGINES = (B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_I8)   # stride 1 only
+ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_AUTO]
 
 
 def rng(seed):
@@ -93,7 +91,7 @@ def test_block_parity(oracle, shape, engine):
     g = rng(sum(shape))
     x = g.standard_normal((N, C, H, W)).astype(np.float32)
     w = g.standard_normal((Co, C, kh, kw)).astype(np.float32)
-    if (engine in TENSOR_ENGINES and s != 1) or (engine == B.XNOR_ENGINE_TC and s > 2):
+    if engine == B.XNOR_ENGINE_UMMA and s > 2:
         with pytest.raises(X.XnorError) as e:       # strides a tensor-core engine does not cover
             gpu_block(x, w, s, p, engine=engine)
         assert e.value.status == B.XNOR_ERR_UNSUPPORTED
