@@ -7,85 +7,195 @@ namespace xnor {
 
 namespace {
 
-constexpr int kPix = 32;      // pixels per block (one warp wide)
-constexpr int kMaxGroups = 8; // warps per block; each owns a subset of the channel words
+constexpr int kPix = 32;        // pixels per group: one warp wide
+constexpr int kWarps = 8;       // warps per block
+constexpr int kTileFloats = 32 * kPix;                 // one (32 channels x 32 pixels) tile
+constexpr int kBufsPerWarp = 2;
 
-// Block = kPix consecutive pixels (flat over n,h,w) x G warps.  Lane = pixel, so
-// each warp-level load of one channel is a contiguous 128-byte run of x.  Warp
-// g packs channel words g, g+G, ...  Words are staged in shared memory and
-// written as one contiguous run of kPix*Cw words.
-template <bool kHasBN>
-__global__ void __launch_bounds__(kPix * kMaxGroups)
-binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scale,
-                     const float *__restrict__ shift, long long total_pix, int C, int HW, int Cw,
-                     uint32_t *__restrict__ x_packed, float *__restrict__ A) {
-  extern __shared__ uint32_t tile[];            // [kPix][Cw]
-  __shared__ float sabs[kMaxGroups][kPix];
-  const int lane = threadIdx.x, g = threadIdx.y, G = blockDim.y;
-  const long long gp0 = (long long)blockIdx.x * kPix;
-  const long long gp = gp0 + lane;
-  const bool live = gp < total_pix;
-  const long long n = live ? gp / HW : 0;
-  const int p = live ? (int)(gp - n * HW) : 0;
-  const float *xb = x + (size_t)n * C * HW + p;
-
-  float asum = 0.0f;
-  for (int cw = g; cw < Cw; cw += G) {
-    const int c0 = cw * 32;
-    float v[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int c = c0 + j;
-      v[j] = (live && c < C) ? __ldcs(xb + (size_t)c * HW) : -1.0f;
-    }
-    uint32_t word = 0u;
-    float part = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int c = c0 + j;
-      if (c < C) {
-        float y = v[j];
-        if (kHasBN) y = __fmaf_rn(__ldg(scale + c), y, __ldg(shift + c));
-        word |= (y >= 0.0f ? 1u : 0u) << j;
-        part += fabsf(y);
-      }
-    }
-    asum += part;
-    tile[lane * Cw + cw] = word;
-  }
-  sabs[g][lane] = asum;
-  __syncthreads();
-  if (g == 0 && live) {
-    float s = 0.0f;
-    for (int i = 0; i < G; ++i) s += sabs[i][lane];
-    A[gp] = s / (float)C;
-  }
-  const long long nw = (total_pix - gp0 < kPix ? total_pix - gp0 : kPix) * Cw;
-  uint32_t *dst = x_packed + (size_t)gp0 * Cw;
-  for (int j = g * kPix + lane; j < nw; j += G * kPix) dst[j] = tile[j];
+__device__ __forceinline__ uint32_t smem_addr(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
 
-__global__ void box_filter_kernel(const float *__restrict__ A, int N, int H, int W, int kh,
-                                  int kw, int stride, int pad, int Ho, int Wo,
-                                  float *__restrict__ K) {
-  const long long total = (long long)N * Ho * Wo;
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
-  const int ox = (int)(i % Wo);
-  const int oy = (int)((i / Wo) % Ho);
-  const long long n = i / ((long long)Wo * Ho);
-  const float *a = A + (size_t)n * H * W;
+// Persistent blocks of 8 warps.  A task is (group of 32 consecutive pixels, flat over n,h,w;
+// 32-channel word): lane = pixel, so one channel of a task is a contiguous 128-byte run of
+// x.  The G warps of a pixel group take words g, g + G, ...; a block works on 8 / G pixel
+// groups at a time.  G = 1 (a warp packs whole pixel groups, no block-wide step) when there
+// are enough pixel groups to fill the GPU, else min(Cw, 8).  Input goes global -> shared with 4-byte cp.async, two tiles
+// per warp in flight while a third is processed, so the bytes in flight per SM (what HBM
+// bandwidth needs) do not depend on how the compiler schedules loads against their uses.
+// Packed words are staged and written as contiguous runs; A is reduced over the warps of a
+// pixel group in a fixed order.
+template <bool kHasBN>
+__global__ void __launch_bounds__(32 * kWarps)
+binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scale,
+                     const float *__restrict__ shift, long long total_pix, int C, int HW, int Cw,
+                     int G, int PG, uint32_t *__restrict__ x_packed, float *__restrict__ A) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  float *stage = reinterpret_cast<float *>(smem_raw);                      // [warp][buf][32][32]
+  float2 *bn = reinterpret_cast<float2 *>(stage + kWarps * kBufsPerWarp * kTileFloats);  // [Cw*32]
+  uint32_t *words = reinterpret_cast<uint32_t *>(bn + (kHasBN ? Cw * 32 : 0));  // [PG][32][Cw]
+  float *sabs = reinterpret_cast<float *>(words + PG * kPix * Cw);          // [PG][G][32]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int pgl = warp / G, g = warp - pgl * G;
+  const bool active = pgl < PG;
+  if (kHasBN) {
+    for (int c = threadIdx.x; c < Cw * 32; c += 32 * kWarps)
+      bn[c] = c < C ? make_float2(__ldg(scale + c), __ldg(shift + c)) : make_float2(0.0f, 0.0f);
+  }
+  __syncthreads();
+
+  const long long ngroups = (total_pix + kPix - 1) / kPix;
+  const long long nbatches = (ngroups + PG - 1) / PG;
+  const int nw = active ? (Cw - g + G - 1) / G : 0;        // words of this warp per pixel group
+  float *my_stage = stage + warp * kBufsPerWarp * kTileFloats;
+
+  // cp.async of one task's tile; always commits a group so that the group count is uniform
+  auto issue = [&](long long batch, int k, int buf) {
+    if (batch < nbatches && k < nw) {
+      const long long gp = (batch * PG + pgl) * kPix + lane;
+      if (gp < total_pix) {
+        const long long n = gp / HW;
+        const int p = (int)(gp - n * HW);
+        const int c0 = (g + k * G) * 32;
+        const float *src = x + ((size_t)n * C + c0) * HW + p;
+        uint32_t dst = smem_addr(my_stage + buf * kTileFloats + lane);
+        const int nc = min(32, C - c0);
+        if (nc == 32) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
+                         ::"r"(dst + (uint32_t)j * kPix * 4), "l"(src + (size_t)j * HW) : "memory");
+        } else {
+          for (int j = 0; j < nc; ++j)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
+                         ::"r"(dst + (uint32_t)j * kPix * 4), "l"(src + (size_t)j * HW) : "memory");
+        }
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  // this warp's tasks in order: (batch, k) with k = 0 .. nw-1
+  long long fb = blockIdx.x;      // batch of the next task to fetch
+  int fk = 0, fbuf = 0;
+  auto advance_fetch = [&]() {
+    if (++fk >= nw) { fk = 0; fb += gridDim.x; }
+    fbuf ^= 1;
+  };
+  issue(fb, fk, fbuf); advance_fetch();
+  issue(fb, fk, fbuf); advance_fetch();
+
+  int buf = 0;
+  for (long long batch = blockIdx.x; batch < nbatches; batch += gridDim.x) {
+    const long long gp0 = (batch * PG + pgl) * kPix;
+    const bool live = active && gp0 + lane < total_pix;
+    float asum = 0.0f;
+    for (int k = 0; k < nw; ++k) {
+      asm volatile("cp.async.wait_group 1;" ::: "memory");   // the older of the two tiles landed
+      const int cw = g + k * G;
+      const int c0 = cw * 32;
+      const float *t = my_stage + buf * kTileFloats + lane;
+      uint32_t word = 0u;
+      float part = 0.0f;
+      if (live) {
+        const float2 *ss = bn + c0;
+        if (c0 + 32 <= C) {
+          // two interleaved sums keep the additions from forming one long dependent chain
+          float p0 = 0.0f, p1 = 0.0f;
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float y0 = t[j * kPix], y1 = t[(j + 1) * kPix];
+            if (kHasBN) {
+              y0 = __fmaf_rn(ss[j].x, y0, ss[j].y);
+              y1 = __fmaf_rn(ss[j + 1].x, y1, ss[j + 1].y);
+            }
+            if (y0 >= 0.0f) word |= 1u << j;
+            if (y1 >= 0.0f) word |= 2u << j;
+            p0 += fabsf(y0);
+            p1 += fabsf(y1);
+          }
+          part = p0 + p1;
+        } else {
+          for (int j = 0; c0 + j < C; ++j) {
+            float y = t[j * kPix];
+            if (kHasBN) y = __fmaf_rn(ss[j].x, y, ss[j].y);
+            if (y >= 0.0f) word |= 1u << j;
+            part += fabsf(y);
+          }
+        }
+      }
+      asum += part;
+      words[(pgl * kPix + lane) * Cw + cw] = word;
+      issue(fb, fk, buf); advance_fetch();                   // refill the tile just consumed
+      buf ^= 1;
+    }
+    if (G == 1) {
+      // one warp owns the pixel group: no block-wide step, the warp's stream of tiles never stops
+      if (live) A[gp0 + lane] = asum / (float)C;
+      __syncwarp();
+      long long npix = total_pix - gp0;
+      if (npix > kPix) npix = kPix;
+      if (npix > 0) {
+        uint32_t *dst = x_packed + (size_t)gp0 * Cw;
+        const uint32_t *srcw = words + pgl * kPix * Cw;
+        for (int i = lane; i < (int)npix * Cw; i += 32) dst[i] = srcw[i];
+      }
+      __syncwarp();
+      continue;
+    }
+    if (active) sabs[(pgl * G + g) * kPix + lane] = asum;
+    __syncthreads();
+    if (active && g == 0 && live) {
+      float sum = 0.0f;
+      for (int i = 0; i < G; ++i) sum += sabs[(pgl * G + i) * kPix + lane];
+      A[gp0 + lane] = sum / (float)C;
+    }
+    // the PG pixel groups of a batch are consecutive: one contiguous run of words
+    const long long bp0 = batch * PG * kPix;
+    long long npix = total_pix - bp0;
+    if (npix > PG * kPix) npix = PG * kPix;
+    uint32_t *dst = x_packed + (size_t)bp0 * Cw;
+    for (int i = threadIdx.x; i < (int)npix * Cw; i += 32 * kWarps) dst[i] = words[i];
+    __syncthreads();
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+// K = box filter of zero-padded A.  One thread per output; blockIdx.y = image, so the index
+// arithmetic is 32-bit and cheap.  KS > 0: square KS x KS filter, every tap a predicated load
+// in straight-line code, so all of a thread's loads are in flight together (a loop with
+// run-time bounds issues them one L2 round trip at a time).  KS = 0: any size.
+template <int KS>
+__global__ void __launch_bounds__(256)
+box_filter_kernel(const float *__restrict__ A, int H, int W, int kh, int kw, int stride, int pad,
+                  int Ho, int Wo, float *__restrict__ K) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= Ho * Wo) return;
+  const int oy = i / Wo, ox = i - oy * Wo;
+  const float *a = A + (size_t)blockIdx.y * H * W;
+  const int y0 = oy * stride - pad, x0 = ox * stride - pad;
   float s = 0.0f;
-  for (int ky = 0; ky < kh; ++ky) {
-    const int iy = oy * stride + ky - pad;
-    if (iy < 0 || iy >= H) continue;
-    for (int kx = 0; kx < kw; ++kx) {
-      const int ix = ox * stride + kx - pad;
-      if (ix < 0 || ix >= W) continue;
-      s += __ldg(a + iy * W + ix);
+  if (KS > 0) {
+    float v[KS > 0 ? KS * KS : 1];
+#pragma unroll
+    for (int ky = 0; ky < KS; ++ky)
+#pragma unroll
+      for (int kx = 0; kx < KS; ++kx) {
+        const int iy = y0 + ky, ix = x0 + kx;
+        const bool in = iy >= 0 && iy < H && ix >= 0 && ix < W;
+        v[ky * KS + kx] = in ? __ldg(a + iy * W + ix) : 0.0f;
+      }
+#pragma unroll
+    for (int t = 0; t < KS * KS; ++t) s += v[t];
+  } else {
+    const int ky0 = y0 < 0 ? -y0 : 0, ky1 = min(kh, H - y0);
+    const int kx0 = x0 < 0 ? -x0 : 0, kx1 = min(kw, W - x0);
+    for (int ky = ky0; ky < ky1; ++ky) {
+      const float *row = a + (y0 + ky) * W + x0;
+      for (int kx = kx0; kx < kx1; ++kx) s += __ldg(row + kx);
     }
   }
-  K[i] = s / (float)(kh * kw);
+  K[(size_t)blockIdx.y * Ho * Wo + i] = s / (float)(kh * kw);
 }
 
 }  // namespace
@@ -94,21 +204,56 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
                             const ConvGeom &g, uint32_t *x_packed, float *A, float *K,
                             cudaStream_t st) {
   const long long total_pix = (long long)g.N * g.H * g.W;
-  const int G = g.Cw < kMaxGroups ? g.Cw : kMaxGroups;
-  const dim3 block(kPix, G);
-  const unsigned grid = (unsigned)((total_pix + kPix - 1) / kPix);
-  const size_t smem = (size_t)kPix * g.Cw * sizeof(uint32_t);
+  // with enough pixel groups to fill the GPU every warp packs whole pixel groups on its own;
+  // otherwise the channel words of a pixel group are spread over the warps of a block
+  const long long ngroups = (total_pix + kPix - 1) / kPix;
+  const int G = ngroups >= 2048 ? 1 : (g.Cw < kWarps ? g.Cw : kWarps);
+  const int PG = kWarps / G;
+  const size_t smem = (size_t)kWarps * kBufsPerWarp * kTileFloats * sizeof(float) +
+                      (scale ? (size_t)g.Cw * 32 * sizeof(float2) : 0) +
+                      (size_t)PG * kPix * g.Cw * sizeof(uint32_t) +
+                      (size_t)PG * G * kPix * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(binactiv_pack_kernel<true>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(binactiv_pack_kernel<false>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
+    attr_set = true;
+  }
+  if (smem > 100 * 1024) return cudaErrorInvalidValue;
+  int sms = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      (void)cudaGetLastError();
+      sms = 148;
+    }
+  }
+  const long long nbatches = ((total_pix + kPix - 1) / kPix + PG - 1) / PG;
+  const unsigned grid = (unsigned)(nbatches < 3ll * sms ? nbatches : 3ll * sms);   // 3 blocks fit an SM
   if (scale)
-    binactiv_pack_kernel<true><<<grid, block, smem, st>>>(x, scale, shift, total_pix, g.C,
-                                                          g.H * g.W, g.Cw, x_packed, A);
+    binactiv_pack_kernel<true><<<grid, 32 * kWarps, smem, st>>>(x, scale, shift, total_pix, g.C,
+                                                              g.H * g.W, g.Cw, G, PG, x_packed, A);
   else
-    binactiv_pack_kernel<false><<<grid, block, smem, st>>>(x, scale, shift, total_pix, g.C,
-                                                           g.H * g.W, g.Cw, x_packed, A);
+    binactiv_pack_kernel<false><<<grid, 32 * kWarps, smem, st>>>(x, scale, shift, total_pix, g.C,
+                                                               g.H * g.W, g.Cw, G, PG, x_packed, A);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const long long total_k = (long long)g.N * g.Ho * g.Wo;
-  box_filter_kernel<<<(unsigned)((total_k + 255) / 256), 256, 0, st>>>(
-      A, g.N, g.H, g.W, g.kh, g.kw, g.stride, g.pad, g.Ho, g.Wo, K);
+  if (g.N > 65535) return cudaErrorInvalidValue;
+  const dim3 kgrid((unsigned)((g.Ho * g.Wo + 255) / 256), (unsigned)g.N);
+  const int ks = g.kh == g.kw ? g.kh : 0;
+#define XNOR_BOX(KS) box_filter_kernel<KS><<<kgrid, 256, 0, st>>>(A, g.H, g.W, g.kh, g.kw, g.stride, \
+                                                                g.pad, g.Ho, g.Wo, K)
+  if (ks == 1) XNOR_BOX(1);
+  else if (ks == 3) XNOR_BOX(3);
+  else if (ks == 5) XNOR_BOX(5);
+  else if (ks == 7) XNOR_BOX(7);
+  else XNOR_BOX(0);
+#undef XNOR_BOX
   return cudaGetLastError();
 }
 
