@@ -564,6 +564,16 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     }
     const int ab = (int)(k % P.nacc);
     const uint32_t use = (uint32_t)(k / P.nacc);
+    if (P.residual != nullptr && valid) {
+      // The residual tile of this item is pulled into L2 while its MMAs run: the loads in the
+      // drain loop then see L2 latency only, and the bytes in flight are not bounded by registers.
+      const float *rp = P.residual + obase + (size_t)(slab * P.NT) * HoWo;
+      const int nf = min(P.NT, P.Co - slab * P.NT);
+      for (int j = 0; j < nf; ++j) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(rp));
+        rp += HoWo;
+      }
+    }
     TR_ADD(0);
     ok = mbar_wait_relaxed(S.afull + 8u * ab, use & 1u, S.abort_flag, &g_status_tc, XNOR_SLEEP_EPI);
     TR_ADD(1);
@@ -576,14 +586,24 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       if (!valid) return;
       const int co = co0 + b * 16;
       float *op = P.out + obase + (size_t)co * HoWo;
-      if (co + 16 <= P.Co && P.residual == nullptr && P.acc_out == nullptr) {
+      if (co + 16 <= P.Co && P.acc_out == nullptr) {
+        float res[16];
+        if (P.residual) {
+          const float *rp = P.residual + obase + (size_t)co * HoWo;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) res[j] = rp[(size_t)j * HoWo];
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) res[j] = 0.0f;
+        }
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
           const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
           const float a4[4] = {al.x, al.y, al.z, al.w};
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
-            *op = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
+            const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
+            *op = P.residual ? v + res[j4 * 4 + jj] : v;
             op += HoWo;
           }
         }
