@@ -343,18 +343,19 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
 // stage's K-steps, gs = grp_steps each (unit u of a thread = K-step grp * gs + u of the stage).
 // The packed words of kPrefetch stages are in flight in registers.
 constexpr int kPrefetch = 4;
-constexpr int kUnits = 2;
 
 struct WCursor {
   long long item;
   int st, slab;
 };
 
+// kUnits = grp_steps: K-steps a thread expands per stage.
+template <int kUnits>
 __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long long i1, int wt,
                             int lane) {
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const int row = wt % P.rows_mod, grp = wt / P.rows_mod;
-  const int gs = P.grp_steps;                      // 1 or 2
+  constexpr int gs = kUnits;
   const bool grp_on = grp * gs < P.mps && row < P.NT;
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
   const int slab0 = (int)(i0 % P.nslabs);
@@ -705,7 +706,11 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   if (i0 < i1) {
     if (warp < kEpiWarps) epilogue_role(P, S, i0, i1, tmem_base, warp, lane);
     else if (warp == kMmaWarp) mma_role(P, S, i0, i1, tmem_base);
-    else if (warp < kPatWarp0) weight_role(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
+    else if (warp < kPatWarp0) {
+      if (P.grp_steps == 4) weight_role<4>(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
+      else if (P.grp_steps == 2) weight_role<2>(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
+      else weight_role<1>(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
+    }
     else patch_role(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
   }
   tc_fence_before();
@@ -756,13 +761,14 @@ Plan make_plan(const ConvGeom &g) {
   P.nsteps = (P.row_words + 1) / 2;
   if (P.nsteps > kMaxSteps) return pl;
   // weight-thread mapping: rows_mod threads cover the rows of a K-step, the other thread
-  // groups take other K-steps of the stage; a stage is about 16 KB of expanded weights
+  // groups take other K-steps of the stage; a stage is up to 32 KB of expanded weights
   int ntp = 16;
   while (ntp < P.NT) ntp *= 2;                          // 16 .. 256
   P.rows_mod = ntp;
   const int groups = kWgtThreads / P.rows_mod;          // 1 .. 16
-  P.mps = std::max(2, std::min(8, 512 / ntp));
-  P.grp_steps = std::max(1, P.mps / groups);            // 2, 2, 2, 1, 1
+  P.mps = std::max(2, std::min(8, 1024 / ntp));
+  while (P.mps > 4 && P.nsteps < 3 * P.mps) P.mps /= 2;   // short items: smaller stages start sooner
+  P.grp_steps = std::max(1, P.mps / groups);            // 4, 4, 2, 1, 1
   P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NT * 32u;
   // shared memory: control, weight ring, patch buffers
   P.off_ring = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
