@@ -38,6 +38,18 @@ BF16_FALLBACK_TFLOPS = 1590.0
 # guide, arithmetic-instruction throughput table, compute capability 10.0); one result
 # covers 32 one-bit MACs.
 POPC_PER_CLK_PER_SM = 16
+# DRAM traffic of the dominant kernel from one ncu capture (profiles/step_kernels_alexnet.md):
+# dram__bytes_read.sum + dram__bytes_write.sum summed over the four BinConv launches of one
+# step of the default workload.  Valid only for the kernel source it was taken from.
+NCU_TRAFFIC = {"kernel_sha1": "UNSET", "bytes_per_step": 174.4e6}
+
+
+def kernel_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for f in ("binconv_tc.cu", "umma_common.cuh", "common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_1603_05279_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
 
 
 def measured_peaks():
@@ -463,6 +475,15 @@ def run_ours(args):
                                    "during the run" % props.multi_processor_count,
                     "traffic": None}
     roofline["frac"] = roofline["achieved"] / roofline["peak"]
+    if engine != "popc" and full and args.workload == "alexnet" and \
+            NCU_TRAFFIC["kernel_sha1"] == kernel_sha1():
+        roofline["traffic"] = NCU_TRAFFIC["bytes_per_step"]
+        roofline["traffic_note"] = ("bytes per step over the 4 launches; below the algorithmic "
+                                    "bytes because part of the output is still in L2 at kernel end")
+    roofline["algorithmic_bytes_per_step"] = sum(
+        4 * (s.N * s.H * s.W * ((s.C_in + 31) // 32) + s.C_out * s.k * s.k * ((s.C_in + 31) // 32)
+             + s.N * wl.out_hw(s)[0] * wl.out_hw(s)[1] * (1 + s.C_out) + s.C_out)
+        for s in job.shapes)
     act_ms = sum(per["binactiv"].values())
 
     def ordered(d):

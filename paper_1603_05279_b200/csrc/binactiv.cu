@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t smem_addr(const void *p) {
 // bandwidth needs) do not depend on how the compiler schedules loads against their uses.
 // Packed words are staged and written as contiguous runs; A is reduced over the warps of a
 // pixel group in a fixed order.
-template <bool kHasBN>
+template <bool kHasBN, bool kVec16>
 __global__ void __launch_bounds__(32 * kWarps)
 binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scale,
                      const float *__restrict__ shift, long long total_pix, int C, int HW, int Cw,
@@ -50,8 +50,27 @@ binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scal
   float *my_stage = stage + warp * kBufsPerWarp * kTileFloats;
 
   // cp.async of one task's tile; always commits a group so that the group count is uniform
+  constexpr bool vec16 = kVec16;          // every 4-pixel chunk of x is 16-byte aligned (HW % 4 == 0)
   auto issue = [&](long long batch, int k, int buf) {
-    if (batch < nbatches && k < nw) {
+    if (batch < nbatches && k < nw && vec16) {
+      // a lane copies 4 consecutive pixels of one channel: 8 copies per tile instead of 32
+      const long long gp = (batch * PG + pgl) * kPix + 4 * (lane & 7);
+      const int c0 = (g + k * G) * 32;
+      if (gp < total_pix) {                 // total_pix is a multiple of 4 here
+        const long long n = gp / HW;
+        const int p = (int)(gp - n * HW);
+        const int ch = lane >> 3;           // + 4 q
+        const float *src = x + ((size_t)n * C + c0 + ch) * HW + p;
+        uint32_t dst = smem_addr(my_stage + buf * kTileFloats + ch * kPix + 4 * (lane & 7));
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (c0 + ch + 4 * q < C)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                         ::"r"(dst + (uint32_t)q * 4 * kPix * 4), "l"(src + (size_t)q * 4 * HW)
+                         : "memory");
+        }
+      }
+    } else if (batch < nbatches && k < nw) {
       const long long gp = (batch * PG + pgl) * kPix + lane;
       if (gp < total_pix) {
         const long long n = gp / HW;
@@ -215,11 +234,13 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
                       (size_t)PG * G * kPix * sizeof(float);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(binactiv_pack_kernel<true>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(binactiv_pack_kernel<false>,
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaSuccess;
+    const void *kernels[4] = {(const void *)binactiv_pack_kernel<true, true>,
+                              (const void *)binactiv_pack_kernel<true, false>,
+                              (const void *)binactiv_pack_kernel<false, true>,
+                              (const void *)binactiv_pack_kernel<false, false>};
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+      e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
     attr_set = true;
   }
@@ -235,12 +256,12 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   }
   const long long nbatches = ((total_pix + kPix - 1) / kPix + PG - 1) / PG;
   const unsigned grid = (unsigned)(nbatches < 3ll * sms ? nbatches : 3ll * sms);   // 3 blocks fit an SM
-  if (scale)
-    binactiv_pack_kernel<true><<<grid, 32 * kWarps, smem, st>>>(x, scale, shift, total_pix, g.C,
-                                                              g.H * g.W, g.Cw, G, PG, x_packed, A);
-  else
-    binactiv_pack_kernel<false><<<grid, 32 * kWarps, smem, st>>>(x, scale, shift, total_pix, g.C,
-                                                               g.H * g.W, g.Cw, G, PG, x_packed, A);
+  const bool v16 = ((g.H * g.W) & 3) == 0;
+#define XNOR_PACK(BN, V16) binactiv_pack_kernel<BN, V16><<<grid, 32 * kWarps, smem, st>>>( \
+      x, scale, shift, total_pix, g.C, g.H * g.W, g.Cw, G, PG, x_packed, A)
+  if (scale) { if (v16) XNOR_PACK(true, true); else XNOR_PACK(true, false); }
+  else { if (v16) XNOR_PACK(false, true); else XNOR_PACK(false, false); }
+#undef XNOR_PACK
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (g.N > 65535) return cudaErrorInvalidValue;

@@ -386,7 +386,7 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
   const uint32_t row_off = (uint32_t)row * 16u;
 #pragma unroll 1
   while (cc.item < i1 && ok) {
-    ok = mbar_wait(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc);
+    ok = mbar_wait_relaxed(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc, XNOR_SLEEP_WGT);
     TR_ADD(0);
     if (!ok) break;
     const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
