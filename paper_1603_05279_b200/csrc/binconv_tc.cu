@@ -129,6 +129,7 @@ struct TcParams {
   uint32_t adesc_lo[kMaxSteps];
   uint32_t swap_mask[32];              // bit j: word 2j+1 is the first piece of step j
   int row_words;               // packed words per filter row = k_h*k_w*Cw
+  int any_swap;                // some bit of swap_mask is set
   uint32_t div_wq_m, div_hq_m; // multipliers and shifts of the exact divisions by Wq and Hq
   int div_wq_s, div_hq_s;      // (dividends below 2^31)
 };
@@ -342,15 +343,18 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
 // Thread mapping: row = wt % rows_mod, and the 256 / rows_mod thread groups split the
 // stage's K-steps, gs = grp_steps each (unit u of a thread = K-step grp * gs + u of the stage).
 // The packed words of kPrefetch stages are in flight in registers.
-constexpr int kPrefetch = 4;
+constexpr int kPrefetch = 3;
 
 struct WCursor {
   long long item;
   int st, slab;
 };
 
-// kUnits = grp_steps: K-steps a thread expands per stage.
-template <int kUnits>
+// kUnits = grp_steps: K-steps a thread expands per stage.  kSwap: some K-step has its two
+// pieces in descending address order (odd Cw or stride 2); otherwise the swap test is compiled
+// out.  The common stage (all its K-steps exist, none is the row's lone last word) takes a
+// path without per-step predicates.
+template <int kUnits, bool kSwap>
 __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long long i1, int wt,
                             int lane) {
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
@@ -358,22 +362,28 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
   constexpr int gs = kUnits;
   const bool grp_on = grp * gs < P.mps && row < P.NT;
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
+  const int jj0 = grp * gs;                         // first K-step of this thread inside a stage
+  const int nplain = (P.row_words >> 1);            // K-steps j < nplain have both words
   const int slab0 = (int)(i0 % P.nslabs);
   WCursor fc{i0, 0, slab0}, cc{i0, 0, slab0};
   auto advance = [&](WCursor &c) {
     if (++c.st == nst) { c.st = 0; ++c.item; if (++c.slab == P.nslabs) c.slab = 0; }
   };
+  const uint2 *wp2 = reinterpret_cast<const uint2 *>(P.wp);
   uint2 pf[kPrefetch][kUnits];
   auto fetch = [&](uint2 dst[kUnits], const WCursor &c) {
     const int co = c.slab * P.NT + row;
     const bool on = grp_on && c.item < i1 && co < P.Co;
-    const int j0 = c.st * P.mps + grp * gs;
+    const int j0 = c.st * P.mps + jj0;
+    if (on && j0 + gs <= P.nsteps) {
+      const uint2 *src = wp2 + ((size_t)j0 * P.Co + co);
 #pragma unroll
-    for (int u = 0; u < kUnits; ++u) {
-      const bool p = on && u < gs && j0 + u < P.nsteps;
-      const uint2 *src = reinterpret_cast<const uint2 *>(P.wp) +
-                         ((size_t)(p ? j0 + u : 0) * P.Co + (p ? co : 0));
-      dst[u] = p ? __ldg(src) : make_uint2(0u, 0u);
+      for (int u = 0; u < kUnits; ++u) dst[u] = __ldg(src + (size_t)u * P.Co);
+    } else {
+#pragma unroll
+      for (int u = 0; u < kUnits; ++u)
+        dst[u] = (on && j0 + u < P.nsteps) ? __ldg(wp2 + ((size_t)(j0 + u) * P.Co + co))
+                                           : make_uint2(0u, 0u);
     }
   };
   TR_DECL(wt < 32);
@@ -383,7 +393,7 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
   int ws = 0;
   uint32_t wph = 1;           // parity to wait for on the empty barriers
   bool ok = true;
-  const uint32_t row_off = (uint32_t)row * 16u;
+  const uint32_t row_off = (uint32_t)row * 16u + (uint32_t)(2 * jj0) * b_lbo;
 #pragma unroll 1
   while (cc.item < i1 && ok) {
     ok = mbar_wait_relaxed(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc, XNOR_SLEEP_WGT);
@@ -391,27 +401,40 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
     if (!ok) break;
     const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
     const int co = cc.slab * P.NT + row;
-    const int jj0 = grp * gs;
     const int j0 = cc.st * P.mps + jj0;
     const bool on = grp_on && co < P.Co;
-    uint32_t v0[kUnits][4], v1[kUnits][4], a0[kUnits], a1[kUnits];
+    if (on && j0 + gs <= nplain) {
+      // plain stage: every K-step of this thread exists and has both of its words
+      uint32_t sbits = 0u;                      // swap bits of K-steps j0 .. j0 + gs - 1
+      if (kSwap) {
+        const int wi = (j0 >> 5) & 31;
+        sbits = __funnelshift_r(P.swap_mask[wi], P.swap_mask[(wi + 1) & 31], j0 & 31);
+      }
 #pragma unroll
-    for (int u = 0; u < kUnits; ++u) {
-      const int j = j0 + u;
-      const bool swap = (P.swap_mask[(j >> 5) & 31] >> (j & 31)) & 1u;
-      const uint32_t keep = 2 * j + 1 < P.row_words ? 0xFFFFFFFFu : 0u;  // lone: partner 0
-      expand_signs<false>(pf[0][u].x, v0[u]);
-      expand_signs<false>(pf[0][u].y, v1[u]);
-      v1[u][0] &= keep; v1[u][1] &= keep; v1[u][2] &= keep; v1[u][3] &= keep;
-      const uint32_t a = stage + (uint32_t)(2 * (jj0 + u)) * b_lbo;
-      a0[u] = swap ? a + b_lbo : a;
-      a1[u] = swap ? a : a + b_lbo;
-    }
+      for (int u = 0; u < kUnits; ++u) {
+        uint32_t v0[4], v1[4];
+        expand_signs<false>(pf[0][u].x, v0);
+        expand_signs<false>(pf[0][u].y, v1);
+        const uint32_t a = stage + (uint32_t)(2 * u) * b_lbo;
+        const uint32_t sw = (kSwap && ((sbits >> u) & 1u)) ? b_lbo : 0u;
+        sts128(a + sw, v0[0], v0[1], v0[2], v0[3]);
+        sts128(a + b_lbo - sw, v1[0], v1[1], v1[2], v1[3]);
+      }
+    } else if (on) {
 #pragma unroll
-    for (int u = 0; u < kUnits; ++u) {
-      if (on && u < gs && j0 + u < P.nsteps) {
-        sts128(a0[u], v0[u][0], v0[u][1], v0[u][2], v0[u][3]);
-        sts128(a1[u], v1[u][0], v1[u][1], v1[u][2], v1[u][3]);
+      for (int u = 0; u < kUnits; ++u) {
+        const int j = j0 + u;
+        if (j < P.nsteps) {
+          const bool swap = (P.swap_mask[(j >> 5) & 31] >> (j & 31)) & 1u;
+          const uint32_t keep = j < nplain ? 0xFFFFFFFFu : 0u;   // lone last word: partner is 0
+          uint32_t v0[4], v1[4];
+          expand_signs<false>(pf[0][u].x, v0);
+          expand_signs<false>(pf[0][u].y, v1);
+          v1[0] &= keep; v1[1] &= keep; v1[2] &= keep; v1[3] &= keep;
+          const uint32_t a = stage + (uint32_t)(2 * u) * b_lbo;
+          sts128(swap ? a + b_lbo : a, v0[0], v0[1], v0[2], v0[3]);
+          sts128(swap ? a : a + b_lbo, v1[0], v1[1], v1[2], v1[3]);
+        }
       }
     }
     TR_ADD(1);
@@ -587,7 +610,18 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       if (!valid) return;
       const int co = co0 + b * 16;
       float *op = P.out + obase + (size_t)co * HoWo;
-      if (co + 16 <= P.Co && P.acc_out == nullptr) {
+      if (co + 16 <= P.Co && P.acc_out == nullptr && P.residual == nullptr) {
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4) {
+          const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
+          const float a4[4] = {al.x, al.y, al.z, al.w};
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            *op = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
+            op += HoWo;
+          }
+        }
+      } else if (co + 16 <= P.Co && P.acc_out == nullptr) {
         float res[16];
         if (P.residual) {
           const float *rp = P.residual + obase + (size_t)co * HoWo;
@@ -707,9 +741,16 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     if (warp < kEpiWarps) epilogue_role(P, S, i0, i1, tmem_base, warp, lane);
     else if (warp == kMmaWarp) mma_role(P, S, i0, i1, tmem_base);
     else if (warp < kPatWarp0) {
-      if (P.grp_steps == 4) weight_role<4>(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
-      else if (P.grp_steps == 2) weight_role<2>(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
-      else weight_role<1>(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
+      const int wt = tid - 32 * kWgtWarp0;
+      if (P.any_swap) {
+        if (P.grp_steps == 4) weight_role<4, true>(P, S, i0, i1, wt, lane);
+        else if (P.grp_steps == 2) weight_role<2, true>(P, S, i0, i1, wt, lane);
+        else weight_role<1, true>(P, S, i0, i1, wt, lane);
+      } else {
+        if (P.grp_steps == 4) weight_role<4, false>(P, S, i0, i1, wt, lane);
+        else if (P.grp_steps == 2) weight_role<2, false>(P, S, i0, i1, wt, lane);
+        else weight_role<1, false>(P, S, i0, i1, wt, lane);
+      }
     }
     else patch_role(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
   }
@@ -792,10 +833,11 @@ Plan make_plan(const ConvGeom &g) {
   const int crem = g.C - 32 * (g.Cw - 1);
   P.tail_mask = crem == 32 ? 0xFFFFFFFFu : ((1u << crem) - 1u);
   for (int j = 0; j < 32; ++j) P.swap_mask[j] = 0u;
+  P.any_swap = 0;
   for (int j = 0; j < P.nsteps; ++j) {
     bool swap;
     P.adesc_lo[j] = kstep_desc(P, j, &swap);
-    if (swap) P.swap_mask[j >> 5] |= 1u << (j & 31);
+    if (swap) { P.swap_mask[j >> 5] |= 1u << (j & 31); P.any_swap = 1; }
   }
   auto magic = [](uint32_t d, uint32_t *m, int *sh) {
     int l = 0;
