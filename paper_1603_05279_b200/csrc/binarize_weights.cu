@@ -16,28 +16,32 @@ binarize_weights_kernel(const float *__restrict__ w, int Co, int C, int taps, in
   const int co = blockIdx.x;
   const int n = C * taps;
   const int nwords = taps * Cw;
-  for (int j = threadIdx.x; j < nwords; j += kThreads) words[j] = 0u;
-  __syncthreads();
-
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float *wf = w + (size_t)co * n;
+  // A warp builds one packed word at a time: lane = channel within the word, the word is a
+  // ballot of (w >= 0).  No atomics, no divisions per weight.
   double l1 = 0.0;
-  for (int i = threadIdx.x; i < n; i += kThreads) {   // i = ci*taps + tap
-    const float v = wf[i];
-    l1 += fabs((double)v);
-    if (v >= 0.0f) {
-      const int ci = i / taps, tap = i - ci * taps;
-      atomicOr(&words[tap * Cw + (ci >> 5)], 1u << (ci & 31));
-    }
+  int tap = 0, cw = warp;                      // word f = tap * Cw + cw, visited in steps of 8
+  while (cw >= Cw) { cw -= Cw; ++tap; }
+  for (int f = warp; f < nwords; f += kThreads / 32) {
+    const int ci = cw * 32 + lane;
+    const bool in = ci < C;
+    const float v = in ? __ldg(wf + (size_t)ci * taps + tap) : -1.0f;
+    if (in) l1 += fabs((double)v);
+    const uint32_t word = __ballot_sync(0xffffffffu, in && v >= 0.0f);
+    if (lane == 0) words[f] = word;
+    cw += kThreads / 32;
+    while (cw >= Cw) { cw -= Cw; ++tap; }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = l1;
+  if (lane == 0) red[warp] = l1;
   __syncthreads();
   if (threadIdx.x == 0) {
-    double s = 0.0;
+    double sum = 0.0;
 #pragma unroll
-    for (int i = 0; i < kThreads / 32; ++i) s += red[i];
-    alpha[co] = (float)(s / (double)n);
+    for (int i = 0; i < kThreads / 32; ++i) sum += red[i];
+    alpha[co] = (float)(sum / (double)n);
   }
   // word-pair-major layout (see packed_weight_index); an odd word count is padded with 0
   for (int j = threadIdx.x; j < ((nwords + 1) & ~1); j += kThreads)
