@@ -370,7 +370,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     du.init("nccl", local)
     X.load()
-    X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2}[args.engine])
+    X.xnor_set_engine({"auto": 0, "popc": 1, "umma": 2, "umma_stream": 3}[args.engine])
     stream = torch.cuda.current_stream()
 
     # every rank has its own batch (weak scaling, no exchange on the data path)
@@ -555,7 +555,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true",
                     help="time call-by-call launches instead of a CUDA graph of the step")
-    ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_stream"])
     ap.add_argument("--workload", default="alexnet", choices=sorted(WORKLOAD_NAMES),
                     help="shape set (the bench line proper is the default, alexnet)")
     ap.add_argument("--layers", default="",

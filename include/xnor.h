@@ -196,9 +196,19 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
  *   XNOR_ENGINE_UMMA   5th-generation tensor cores (tcgen05), 4-bit (e2m1)
  *                      operands built from the sign bits, exact fp32
  *                      accumulation of integers; strides 1 and 2, shapes whose
- *                      activation patch fits shared memory
+ *                      activation patch fits shared memory.  The expanded
+ *                      filters of a slab stay in shared memory while a CTA
+ *                      walks the pixel tiles, when they fit
+ *   XNOR_ENGINE_UMMA_STREAM  the same engine with the schedule it falls back
+ *                      to when a slab does not fit: filters re-expanded
+ *                      through a ring of stages for every work item
  */
-typedef enum { XNOR_ENGINE_AUTO = 0, XNOR_ENGINE_POPC = 1, XNOR_ENGINE_UMMA = 2 } xnor_engine;
+typedef enum {
+  XNOR_ENGINE_AUTO = 0,
+  XNOR_ENGINE_POPC = 1,
+  XNOR_ENGINE_UMMA = 2,
+  XNOR_ENGINE_UMMA_STREAM = 3
+} xnor_engine;
 xnor_status xnor_set_engine(xnor_engine e);
 xnor_engine xnor_get_engine(void);
 

@@ -43,6 +43,14 @@
 //  item overlaps the MMAs of the next.  Every wait is bounded: on expiry the
 //  CTA records XNOR_ERR_TIMEOUT in a device status word, stops, frees its
 //  tensor memory and exits.
+//
+//  Two schedules.  "Resident": when the expanded rows of a filter slab fit in
+//  shared memory beside two patches, the slab is expanded ONCE per CTA and the
+//  CTA then walks the pixel tiles of that slab (items in slab-major order, one
+//  patch per item); the weight warps, idle after the fill, join the epilogue
+//  (three warps per quarter of the lanes, splitting the columns).  "Streaming":
+//  otherwise the weights of every item pass through a ring of stages (items in
+//  tile-major order, so that a patch serves all slabs of its tile).
 #include <algorithm>
 #include <cstdio>
 #include <cstdlib>
@@ -57,6 +65,8 @@ __device__ int g_status_tc = 0;
 // cycle totals of one warp per role of one CTA: [0..7] mma, [8..15] weights, [16..23] patch,
 // [24..31] epilogue
 __device__ long long g_tc_trace[64];
+// per CTA: clock at the start of the roles, at their end, SM id
+__device__ long long g_tc_cta[3 * 160];
 #define TR_DECL(first) long long tr_t = 0, tr_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}; \
   const bool tr_on = blockIdx.x == 1 && (threadIdx.x & 31) == 0 && (first)
 #define TR_T0 do { if (tr_on) tr_t = clock64(); } while (0)
@@ -93,10 +103,13 @@ constexpr int kTileM = 128;          // stream positions per tile = tensor-memor
 constexpr int kTmemCols = 512;
 constexpr int kSfCol = 480;          // columns [480, 512): unit block scales
 constexpr int kMaxAccCols = 480;
-constexpr int kMaxStages = 6;
+constexpr int kMaxAcc = 4;           // accumulator buffers
+constexpr int kMaxStages = 6;         // ring stages of the streaming schedule
+constexpr int kMaxBarStages = 32;    // stage barriers (the resident schedule has one stage per mps K-steps of a row)
+constexpr int kEpiSplitMax = 3;      // warps per lane quarter in the resident epilogue
 constexpr int kMaxPatchBufs = 4;
 constexpr int kMaxSteps = 800;       // K-steps (MMAs) per work item (< 1024: swap_mask)
-constexpr size_t kCtrlBytes = 512;
+constexpr size_t kCtrlBytes = 1024;
 constexpr size_t kSmemMax = 232448 - 1024;
 
 struct TcParams {
@@ -109,7 +122,7 @@ struct TcParams {
   int dymin, dxmin;
   long long L;                 // stream length N*Hq*Wq
   int ntiles, nslabs, NT;      // pixel tiles, filter slabs, filters per slab (multiple of 16)
-  int nacc;                    // accumulator buffers in tensor memory (1 or 2)
+  int nacc;                    // accumulator buffers in tensor memory (1 .. 4)
   int ppix;                    // stream positions staged per phase plane (128 + halo, rounded to 8)
   int nplanes;                 // stride*stride*Cw operand planes per patch
   int npb;                     // patch buffers
@@ -118,7 +131,9 @@ struct TcParams {
   int stages;
   uint32_t patch_bytes, stage_bytes;
   int rows_mod, grp_steps;     // weight-thread mapping (see weight producer)
-  uint32_t off_ring, off_patch;  // byte offsets in dynamic shared memory
+  uint32_t off_ring, off_patch, off_raw;  // byte offsets in dynamic shared memory
+  int nraw;                    // raw buffers per patch warp (1 or 2)
+  uint32_t raw_bytes;          // size of one: the packed input rows a patch can touch
   uint32_t idesc;
   uint32_t tail_mask;          // bits of real channels in the last word
   // Low word of the A-operand descriptor of every K-step (start address relative to the
@@ -129,6 +144,8 @@ struct TcParams {
   uint32_t adesc_lo[kMaxSteps];
   uint32_t swap_mask[32];              // bit j: word 2j+1 is the first piece of step j
   int row_words;               // packed words per filter row = k_h*k_w*Cw
+  int resident;                // 1: resident schedule (stages = all stages of a slab)
+  int epi_split;               // warps per lane quarter that drain an accumulator
   int any_swap;                // some bit of swap_mask is set
   uint32_t div_wq_m, div_hq_m; // multipliers and shifts of the exact divisions by Wq and Hq
   int div_wq_s, div_hq_s;      // (dividends below 2^31)
@@ -225,25 +242,28 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m, int s) {
 }
 
 struct Smem {
-  uint32_t wfull, wempty, pfull, pempty, afull, aempty;   // shared-space addresses of barrier arrays
+  uint32_t wfull, wempty, pfull, pempty, afull, aempty, rawfull;   // shared-space addresses of barrier arrays
   uint32_t *tmem_slot;
   volatile int *abort_flag;
-  uint32_t ring, patch;                                   // shared-space byte addresses
+  uint32_t ring, patch, raw;                              // shared-space byte addresses
 };
 
 __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
   Smem s;
   const uint32_t base = smem_u32(smem);
   s.wfull = base;
-  s.wempty = s.wfull + 8u * kMaxStages;
-  s.pfull = s.wempty + 8u * kMaxStages;
+  s.wempty = s.wfull + 8u * kMaxBarStages;
+  s.pfull = s.wempty + 8u * kMaxBarStages;
   s.pempty = s.pfull + 8u * kMaxPatchBufs;
   s.afull = s.pempty + 8u * kMaxPatchBufs;
-  s.aempty = s.afull + 16u;
-  s.tmem_slot = reinterpret_cast<uint32_t *>(smem + 8 * (2 * kMaxStages + 2 * kMaxPatchBufs + 4));
+  s.aempty = s.afull + 8u * kMaxAcc;
+  s.rawfull = s.aempty + 8u * kMaxAcc;
+  s.tmem_slot = reinterpret_cast<uint32_t *>(
+      smem + 8 * (2 * kMaxBarStages + 2 * kMaxPatchBufs + 2 * kMaxAcc + 2 * kPatWarps));
   s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
   s.ring = base + P.off_ring;
   s.patch = base + P.off_patch;
+  s.raw = base + P.off_raw;
   return s;
 }
 
@@ -267,6 +287,9 @@ __device__ __forceinline__ void issue_stage(const TcParams &P, int j0, uint32_t 
                       b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u, el);
 }
 
+// kRes: resident schedule.  The stage barriers are then waited for only on the first item of
+// a slab visit (the slab stays in shared memory afterwards) and released only on the last.
+template <bool kRes>
 __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long long i1,
                          uint32_t tmem_base) {
   const uint32_t tmem_sf = tmem_base + (uint32_t)kSfCol;
@@ -278,24 +301,27 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
   const uint32_t b_step = (2u * b_lbo) >> 4;                                   // next K-step
   const uint32_t stage_step = P.stage_bytes >> 4;
   const uint32_t el = elect_one();
-  int ws = 0, pb = 0;
+  int ws = 0, pb = 0, ab = 0;
   uint32_t wph = 0, pph = 0;
-  long long k = 0;                       // items done by this CTA
-  int slab = (int)(i0 % P.nslabs);
+  uint32_t aph = 1u;                     // parity to wait for on the accumulator's empty barrier
+  // streaming: item = tile * nslabs + slab; resident: item = slab * ntiles + tile
+  int slab = kRes ? 0 : (int)(i0 % P.nslabs);
+  int tile = kRes ? (int)(i0 % P.ntiles) : 0;
   bool ok = true, new_tile = true;
   uint32_t patch_lo = 0;                 // patch address in descriptor units
   TR_DECL(true);
   TR_T0;
-  for (long long item = i0; item < i1 && ok; ++item, ++k) {
+  const uint32_t nitems = (uint32_t)(i1 - i0);
+  for (uint32_t it = 0; it < nitems && ok; ++it) {
     if (new_tile) {
       ok = mbar_wait_warp(S.pfull + 8u * pb, pph, S.abort_flag);
       TR_ADD(0);
       if (!ok) break;
       patch_lo = ((S.patch + (uint32_t)pb * P.patch_bytes) & 0x3FFFFu) >> 4;
     }
-    const int ab = (int)(k % P.nacc);
-    const uint32_t use = (uint32_t)(k / P.nacc);
-    ok = mbar_wait_warp(S.aempty + 8u * ab, (use & 1u) ^ 1u, S.abort_flag);
+    const bool visit_first = !kRes || it == 0 || tile == 0;
+    const bool visit_last = !kRes || it + 1 == nitems || tile + 1 == P.ntiles;
+    ok = mbar_wait_warp(S.aempty + 8u * ab, aph, S.abort_flag);
     TR_ADD(1);
     if (!ok) break;
     tc_fence_after();
@@ -305,10 +331,12 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
       const int nj = min(P.mps, P.nsteps - j0);
       const uint32_t b_lo = b_lo0 + (uint32_t)ws * stage_step;
       const uint32_t first = st == 0 ? 0u : 1u;     // the first MMA of an item overwrites
-      ok = mbar_wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
-      TR_ADD(2);
-      if (!ok) break;
-      tc_fence_after();
+      if (visit_first) {
+        ok = mbar_wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
+        TR_ADD(2);
+        if (!ok) break;
+        tc_fence_after();
+      }
       TR_ADD(3);
       if (nj == 4) issue_stage<4>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
       else if (nj == 2) issue_stage<2>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
@@ -320,17 +348,27 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
                             jj == 0 ? first : 1u, el);
       }
       TR_ADD(4);
-      umma_commit_elected(S.wempty + 8u * ws, el);
+      if (visit_last) umma_commit_elected(S.wempty + 8u * ws, el);
       TR_ADD(5);
-      if (++ws == P.stages) { ws = 0; wph ^= 1u; }
+      if (++ws == P.stages) { ws = 0; if (!kRes) wph ^= 1u; }
     }
     if (!ok) break;
-    // next item: same tile (next slab) or the next tile
-    new_tile = false;
-    if (++slab == P.nslabs) { slab = 0; new_tile = true; }
-    umma_commit_elected(S.afull + 8u * ab, el);
-    if (new_tile || item + 1 == i1) umma_commit_elected(S.pempty + 8u * pb, el);
-    if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
+    if (kRes) {
+      // every item has its own patch; the barrier phase of the slab flips with the visit
+      if (visit_last) wph ^= 1u;
+      if (++tile == P.ntiles) tile = 0;
+      umma_commit_elected(S.afull + 8u * ab, el);
+      umma_commit_elected(S.pempty + 8u * pb, el);
+      if (++pb == P.npb) { pb = 0; pph ^= 1u; }
+    } else {
+      // next item: same tile (next slab) or the next tile
+      new_tile = false;
+      if (++slab == P.nslabs) { slab = 0; new_tile = true; }
+      umma_commit_elected(S.afull + 8u * ab, el);
+      if (new_tile || it + 1 == nitems) umma_commit_elected(S.pempty + 8u * pb, el);
+      if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
+    }
+    if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
     TR_ADD(6);
   }
   TR_FLUSH(0);
@@ -354,9 +392,14 @@ struct WCursor {
 // pieces in descending address order (odd Cw or stride 2); otherwise the swap test is compiled
 // out.  The common stage (all its K-steps exist, none is the row's lone last word) takes a
 // path without per-step predicates.
+// The role fills the stages of `nitems` consecutive items, the first of slab `slab0` (the
+// slabs then follow cyclically), waiting for the empty barriers with parity `wph0` on the
+// first round.  Streaming: all items of the CTA in one call.  Resident: one call per slab
+// visit with nitems = 1 (the ring then has one stage per stage of the slab).
 template <int kUnits, bool kSwap>
-__device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long long i1, int wt,
-                            int lane) {
+__device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, int slab0,
+                            uint32_t wph0, int wt, int lane) {
+  const long long i0 = 0, i1 = nitems;
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const int row = wt % P.rows_mod, grp = wt / P.rows_mod;
   constexpr int gs = kUnits;
@@ -364,7 +407,6 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
   const int jj0 = grp * gs;                         // first K-step of this thread inside a stage
   const int nplain = (P.row_words >> 1);            // K-steps j < nplain have both words
-  const int slab0 = (int)(i0 % P.nslabs);
   WCursor fc{i0, 0, slab0}, cc{i0, 0, slab0};
   auto advance = [&](WCursor &c) {
     if (++c.st == nst) { c.st = 0; ++c.item; if (++c.slab == P.nslabs) c.slab = 0; }
@@ -391,7 +433,7 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
 #pragma unroll
   for (int d = 0; d < kPrefetch; ++d) { fetch(pf[d], fc); advance(fc); }
   int ws = 0;
-  uint32_t wph = 1;           // parity to wait for on the empty barriers
+  uint32_t wph = wph0;        // parity to wait for on the empty barriers
   bool ok = true;
   const uint32_t row_off = (uint32_t)row * 16u + (uint32_t)(2 * jj0) * b_lbo;
 #pragma unroll 1
@@ -453,92 +495,166 @@ __device__ void weight_role(const TcParams &P, const Smem &S, long long i0, long
     TR_ADD(2);
   }
   TR_FLUSH(8);
+  return ok;
+}
+
+template <int kUnits>
+__device__ __forceinline__ bool weight_role_swap(const TcParams &P, const Smem &S,
+                                                 long long nitems, int slab0, uint32_t wph0,
+                                                 int wt, int lane) {
+  return P.any_swap ? weight_role<kUnits, true>(P, S, nitems, slab0, wph0, wt, lane)
+                    : weight_role<kUnits, false>(P, S, nitems, slab0, wph0, wt, lane);
+}
+
+__device__ __forceinline__ bool weight_dispatch(const TcParams &P, const Smem &S, long long nitems,
+                                                int slab0, uint32_t wph0, int wt, int lane) {
+  if (P.grp_steps == 4) return weight_role_swap<4>(P, S, nitems, slab0, wph0, wt, lane);
+  if (P.grp_steps == 2) return weight_role_swap<2>(P, S, nitems, slab0, wph0, wt, lane);
+  return weight_role_swap<1>(P, S, nitems, slab0, wph0, wt, lane);
 }
 
 // ------------------------------------------------------------------ patch producers (3 warps)
-// Each warp expands whole tiles on its own (warp p takes this CTA's tiles p, p + 3, ...), so
-// the global-load latency of up to three tiles overlaps; a tile's patch buffer is its index
-// modulo the number of buffers.  For every (phase plane, group of up to 4 channel words) a
-// lane walks the patch's stream positions, kPosBatch of them in flight at a time.
-constexpr int kPosBatch = 2;
-
+// Each warp builds whole patches on its own (warp p takes the CTA's patches p, p + active,
+// ...), so up to three patches are in the making; a patch's buffer is its index modulo the
+// number of buffers.  The packed pixels a patch touches are ONE contiguous range of x_packed:
+// input rows g0 .. g1 - 1 of the N*H rows (images follow one another in memory, the zero
+// rows and columns of the stream exist only in the patch).  Lane 0 brings that range into a
+// raw buffer of the warp with one bulk copy (an aligned superset inside the tensor; the
+// ragged last words of the tensor, if any, by plain loads), one patch ahead when the warp
+// has two raw buffers; the warp then expands from shared memory, a stream position per lane.
+// Streaming: one patch per tile of the CTA's range.  Resident (kRes): one patch per item.
+template <bool kRes>
 __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long long i1, int pt,
                            int lane) {
-  const int tile0 = (int)(i0 / P.nslabs), tile1 = (int)((i1 - 1) / P.nslabs);
+  const int tile0 = kRes ? 0 : (int)(i0 / P.nslabs);
+  const uint32_t npatches = kRes ? (uint32_t)(i1 - i0)
+                                 : (uint32_t)((i1 - 1) / P.nslabs) - (uint32_t)tile0 + 1u;
+  const uint32_t tile_r0 = kRes ? (uint32_t)(i0 % P.ntiles) : 0u;   // resident: tile of the first item
   const int s = P.stride, phases = s * s;
   const uint32_t plane_bytes = (uint32_t)P.ppix * 16u;
   const bool vec = (P.Cw & 3) == 0;
   const int pw = pt >> 5;                       // patch warp 0..2
+  // A barrier's parity tells apart only two consecutive uses of a buffer, so no warp may run
+  // more than one use ahead of the consumer: at most npb warps take part.
+  const int active = min(kPatWarps, P.npb);
+  if (pw >= active) return;
   // nibble masks of the channel tail, one per expanded register
   uint32_t tm[4];
 #pragma unroll
   for (int r = 0; r < 4; ++r) tm[r] = ((P.tail_mask >> r) & 0x11111111u) * 0xFu;
+  const uint32_t row_bytes = (uint32_t)P.W * (uint32_t)P.Cw * 4u;
+  const size_t tensor_bytes = (size_t)P.N * P.H * row_bytes;
+  const uint32_t raw0 = S.raw + (uint32_t)(pw * P.nraw) * P.raw_bytes;
+  const uint32_t rbar0 = S.rawfull + 8u * (uint32_t)(pw * 2);
+
+  auto tile_of = [&](uint32_t seq) {
+    return kRes ? (int)((tile_r0 + seq) % (uint32_t)P.ntiles) : tile0 + (int)seq;
+  };
+  // input rows [g0, g1) (of the N*H rows of the tensor) that the patch of a tile reads
+  auto row_range = [&](int tile, int &g0, int &g1) {
+    const uint32_t m0 = (uint32_t)tile * kTileM;
+    const uint32_t mlast = min(m0 + (uint32_t)P.ppix - 1u, (uint32_t)P.L - 1u);
+    const uint32_t r0 = fast_div(m0, P.div_wq_m, P.div_wq_s);
+    const uint32_t r1 = fast_div(mlast, P.div_wq_m, P.div_wq_s);
+    const uint32_t n0 = fast_div(r0, P.div_hq_m, P.div_hq_s);
+    const uint32_t n1 = fast_div(r1, P.div_hq_m, P.div_hq_s);
+    const int ry0 = (int)(r0 - n0 * (uint32_t)P.Hq), ry1 = (int)(r1 - n1 * (uint32_t)P.Hq);
+    const int t0 = min(max((ry0 - P.leadY) * s, 0), P.H);
+    const int t1 = min(max((ry1 - P.leadY) * s + s, 0), P.H);
+    g0 = (int)n0 * P.H + t0;
+    g1 = (int)n1 * P.H + t1;
+  };
+  // lane 0: starts the copy of a patch's rows into raw buffer rb
+  auto start_copy = [&](uint32_t seq, int rb) {
+    int g0, g1;
+    row_range(tile_of(seq), g0, g1);
+    const uint32_t bar = rbar0 + 8u * (uint32_t)rb;
+    const uint32_t dst = raw0 + (uint32_t)rb * P.raw_bytes;
+    if (g1 <= g0) { mbar_arrive(bar); return; }          // nothing but padding
+    const size_t b0 = (size_t)g0 * row_bytes, b1 = (size_t)g1 * row_bytes;
+    const size_t a0 = b0 & ~(size_t)15;
+    const size_t a1 = min((b1 + 15) & ~(size_t)15, tensor_bytes & ~(size_t)15);
+    const uint32_t bulk = a1 > a0 ? (uint32_t)(a1 - a0) : 0u;
+    for (size_t b = a0 + bulk; b < b1; b += 4)           // at most 3 words, at the tensor's end
+      sts32(dst + (uint32_t)(b - a0), __ldg(P.xp + (b >> 2)));
+    if (bulk) {
+      mbar_arrive_expect_tx(bar, bulk);
+      bulk_copy_g2s(dst, reinterpret_cast<const uint8_t *>(P.xp) + a0, bulk, bar);
+    } else {
+      mbar_arrive(bar);
+    }
+  };
+
   bool ok = true;
+  bool pend[2] = {false, false};          // a copy into the raw buffer has not been consumed
+  uint32_t rph[2] = {0u, 0u};             // parity of the raw buffer's next completion
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const uint32_t seq = (uint32_t)(pw + r * active);
+    if (r < P.nraw && seq < npatches) {
+      if (lane == 0) start_copy(seq, r);
+      pend[r] = true;
+    }
+  }
+  int rb = 0;
   TR_DECL(pt < 32);
   TR_T0;
 #pragma unroll 1
-  for (int tile = tile0 + pw; tile <= tile1 && ok; tile += kPatWarps) {
-    const int seq = tile - tile0;               // this CTA's tiles in order
-    const int pb = seq % P.npb;
-    const uint32_t pph = ((uint32_t)(seq / P.npb) & 1u) ^ 1u;
+  for (uint32_t seq = (uint32_t)pw; seq < npatches && ok; seq += (uint32_t)active) {   // in order
+    const int tile = tile_of(seq);
+    const int pb = (int)(seq % (uint32_t)P.npb);
+    const uint32_t pph = ((seq / (uint32_t)P.npb) & 1u) ^ 1u;
+    int g0, g1;
+    row_range(tile, g0, g1);
+    const uint32_t rbar = rbar0 + 8u * (uint32_t)rb;
+    ok = mbar_wait_relaxed(rbar, rb ? rph[1] : rph[0], S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
+    if (!ok) break;
+    if (rb) { pend[1] = false; rph[1] ^= 1u; } else { pend[0] = false; rph[0] ^= 1u; }
     ok = mbar_wait_relaxed(S.pempty + 8u * pb, pph, S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
     TR_ADD(0);
     if (!ok) break;
     const uint32_t patch = S.patch + (uint32_t)pb * P.patch_bytes;
     const uint32_t m0 = (uint32_t)tile * kTileM;
+    const uint32_t raw = raw0 + (uint32_t)rb * P.raw_bytes +
+                         (uint32_t)(((size_t)g0 * row_bytes) & 15u);   // where row g0 starts
 #pragma unroll 1
-    for (int phase = 0; phase < phases; ++phase) {
-      const int py = phase / s, px = phase - py * s;
+    for (int q = lane; q < P.ppix; q += 32) {
+      const uint32_t sq = m0 + (uint32_t)q;
+      const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
+      const int c = (int)(sq - r * (uint32_t)P.Wq);
+      const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
+      const int ry = (int)(r - n * (uint32_t)P.Hq);
+      const bool in = sq < (uint32_t)P.L && ry >= P.leadY && c >= P.leadX;
+      const int rrow = (ry - P.leadY) * s, rcol = (c - P.leadX) * s;
+      const int grow = (int)n * P.H + rrow - g0;     // row inside the raw range (+ py)
 #pragma unroll 1
-      for (int w0 = 0; w0 < P.Cw; w0 += 4) {
-        const uint32_t dst0 = patch + (uint32_t)(phase * P.Cw + w0) * plane_bytes;
-        const bool has_tail = w0 + 4 >= P.Cw;   // this group holds the last word
+      for (int phase = 0; phase < phases; ++phase) {
+        const int py = phase / s, px = phase - py * s;
+        const bool real = in && rrow + py < P.H && rcol + px < P.W;
+        const uint32_t keep = real ? 0xFFFFFFFFu : 0u;        // padding expands to 0
+        const uint32_t src = raw + (uint32_t)(((grow + py) * P.W + rcol + px) * P.Cw) * 4u;
+        const uint32_t dst = patch + (uint32_t)(phase * P.Cw) * plane_bytes + (uint32_t)q * 16u;
 #pragma unroll 1
-        for (int q0 = lane; q0 < P.ppix; q0 += 32 * kPosBatch) {
-          uint32_t wv[kPosBatch][4];
-          bool real[kPosBatch];
+        for (int w0 = 0; w0 < P.Cw; w0 += 4) {
+          uint32_t wv[4] = {0u, 0u, 0u, 0u};
+          if (real) {
+            if (vec) {
+              lds128(src + (uint32_t)w0 * 4u, wv);
+            } else {
 #pragma unroll
-          for (int b = 0; b < kPosBatch; ++b) {
-            const int q = q0 + 32 * b;
-            wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
-            real[b] = false;
-            const uint32_t sq = m0 + (uint32_t)q;
-            if (q < P.ppix && sq < (uint32_t)P.L) {
-              const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
-              const int c = (int)(sq - r * (uint32_t)P.Wq);
-              const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
-              const int ry = (int)(r - n * (uint32_t)P.Hq);
-              const int iy = (ry - P.leadY) * s + py, ix = (c - P.leadX) * s + px;
-              if (ry >= P.leadY && c >= P.leadX && iy < P.H && ix < P.W) {
-                const uint32_t *src = P.xp + (((size_t)n * P.H + iy) * P.W + ix) * P.Cw + w0;
-                real[b] = true;
-                if (vec) {
-                  const uint4 t = __ldg(reinterpret_cast<const uint4 *>(src));
-                  wv[b][0] = t.x; wv[b][1] = t.y; wv[b][2] = t.z; wv[b][3] = t.w;
-                } else {
-#pragma unroll
-                  for (int i = 0; i < 4; ++i)
-                    if (w0 + i < P.Cw) wv[b][i] = __ldg(src + i);
-                }
-              }
+              for (int i = 0; i < 4; ++i)
+                if (w0 + i < P.Cw) wv[i] = lds32(src + (uint32_t)(w0 + i) * 4u);
             }
           }
 #pragma unroll
-          for (int b = 0; b < kPosBatch; ++b) {
-            const int q = q0 + 32 * b;
-            if (q < P.ppix) {
-              const uint32_t keep = real[b] ? 0xFFFFFFFFu : 0u;    // padding expands to 0
+          for (int i = 0; i < 4; ++i) {
+            if (w0 + i < P.Cw) {
+              uint32_t v[4];
+              expand_signs<true>(wv[i], v);
+              const bool last = w0 + i == P.Cw - 1;           // channels beyond C_in are 0
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                if (w0 + i < P.Cw) {
-                  uint32_t v[4];
-                  expand_signs<true>(wv[b][i], v);
-                  const bool last = has_tail && w0 + i == P.Cw - 1;   // channels beyond C_in are 0
-#pragma unroll
-                  for (int r = 0; r < 4; ++r) v[r] &= last ? (tm[r] & keep) : keep;
-                  sts128(dst0 + (uint32_t)i * plane_bytes + (uint32_t)q * 16u, v[0], v[1], v[2], v[3]);
-                }
-              }
+              for (int rr = 0; rr < 4; ++rr) v[rr] &= last ? (tm[rr] & keep) : keep;
+              sts128(dst + (uint32_t)(w0 + i) * plane_bytes, v[0], v[1], v[2], v[3]);
             }
           }
         }
@@ -547,7 +663,23 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     TR_ADD(1);
     fence_proxy_async();
     __syncwarp();
-    if (lane == 0) mbar_arrive(S.pfull + 8u * pb);
+    const uint32_t next = seq + (uint32_t)(P.nraw * active);   // reuses this raw buffer
+    if (lane == 0) {
+      mbar_arrive(S.pfull + 8u * pb);
+      if (next < npatches) start_copy(next, rb);
+    }
+    if (next < npatches) { if (rb) pend[1] = true; else pend[0] = true; }
+    if (++rb == P.nraw) rb = 0;
+  }
+  if (!ok) {
+    // gave up: a copy still in flight must land before the CTA's shared memory is released
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (pend[r]) {
+        const uint32_t bar = rbar0 + 8u * (uint32_t)r;
+        for (int i = 0; i < (1 << 20) && !mbar_try(bar, rph[r]); ++i) {}
+      }
+    }
   }
   TR_FLUSH(16);
 }
@@ -556,39 +688,59 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
 // Warp w reads tensor-memory lanes 32 w .. +31 (pixels), all the slab's columns (filters).
 // Lane = pixel, so for one filter a warp stores 32 consecutive stream pixels: a contiguous
 // run of the NCHW output row.
-__device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, long long i1,
-                              uint32_t tmem_base, int warp, int lane) {
-  const int quarter = warp;
+// Drains items [i0, i1), the k0-th and following of the CTA.  Of every item this warp takes
+// the 16-column groups e, e + esplit, ... (esplit warps share a quarter of the lanes).
+template <bool kRes>
+__device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, long long i1,
+                              long long k0, uint32_t tmem_base, int quarter, int e, int lane) {
   const int b_end = P.NT / 16;
+  const int esplit = kRes ? P.epi_split : 1;
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-  int tile = (int)(i0 / P.nslabs), slab = (int)(i0 - (long long)tile * P.nslabs);
-  bool new_tile = true, valid = false, ok = true;
-  float kv = 0.0f;
-  size_t obase = 0;                       // offset of (image, filter 0, pixel)
-  long long k = 0;
-  TR_DECL(warp == 0);
-  TR_T0;
-  for (long long item = i0; item < i1 && ok; ++item, ++k) {
-    if (new_tile) {
-      const uint32_t m = (uint32_t)tile * kTileM + (uint32_t)(quarter * 32 + lane);
-      valid = m < (uint32_t)P.L;
-      if (valid) {
-        const uint32_t r = fast_div(m, P.div_wq_m, P.div_wq_s);
-        const int ox = (int)(m - r * (uint32_t)P.Wq);
-        const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
-        const int oy = (int)(r - n * (uint32_t)P.Hq);
-        valid = ox < P.Wo && oy < P.Ho;
-        if (valid) {
-          const size_t pix = (size_t)oy * P.Wo + ox;
-          kv = __ldg(P.K + (size_t)n * HoWo + pix);
-          obase = (size_t)n * P.Co * HoWo + pix;
-        }
+  int tile, slab;
+  if (kRes) { slab = (int)(i0 / P.ntiles); tile = (int)(i0 - (long long)slab * P.ntiles); }
+  else { tile = (int)(i0 / P.nslabs); slab = (int)(i0 - (long long)tile * P.nslabs); }
+  bool ok = true;
+  // this lane's output pixel in a tile: whether it exists, its K, offset of (image, filter 0, pixel)
+  struct Pix { bool valid; float kv; size_t obase; };
+  auto decode = [&](int t) {
+    Pix px{false, 0.0f, 0};
+    const uint32_t m = (uint32_t)t * kTileM + (uint32_t)(quarter * 32 + lane);
+    if (m < (uint32_t)P.L) {
+      const uint32_t r = fast_div(m, P.div_wq_m, P.div_wq_s);
+      const int ox = (int)(m - r * (uint32_t)P.Wq);
+      const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
+      const int oy = (int)(r - n * (uint32_t)P.Hq);
+      if (ox < P.Wo && oy < P.Ho) {
+        const size_t pix = (size_t)oy * P.Wo + ox;
+        px.valid = true;
+        px.kv = __ldg(P.K + (size_t)n * HoWo + pix);
+        px.obase = (size_t)n * P.Co * HoWo + pix;
       }
     }
-    const int ab = (int)(k % P.nacc);
-    const uint32_t use = (uint32_t)(k / P.nacc);
-    if (P.residual != nullptr && valid) {
+    return px;
+  };
+  Pix px = decode(tile);
+  int ab = (int)(k0 % P.nacc);            // accumulator buffer of the next item and the parity
+  uint32_t fph = (uint32_t)(k0 / P.nacc) & 1u;   // of its full barrier
+  TR_DECL(quarter == 0 && e == 0);
+  TR_T0;
+  const uint32_t nitems = (uint32_t)(i1 - i0);
+  for (uint32_t it = 0; it < nitems && ok; ++it) {
+    const bool valid = px.valid;
+    const float kv = px.kv;
+    const size_t obase = px.obase;
+    // the item after this one; its pixel is decoded (and its K loaded) while this one drains
+    int ntile = tile, nslab = slab;
+    bool next_new;
+    if (kRes) {
+      next_new = true;
+      if (++ntile == P.ntiles) { ntile = 0; ++nslab; }
+    } else {
+      next_new = false;
+      if (++nslab == P.nslabs) { nslab = 0; ++ntile; next_new = true; }
+    }
+    if (P.residual != nullptr && valid && e == 0) {
       // The residual tile of this item is pulled into L2 while its MMAs run: the loads in the
       // drain loop then see L2 latency only, and the bytes in flight are not bounded by registers.
       const float *rp = P.residual + obase + (size_t)(slab * P.NT) * HoWo;
@@ -599,12 +751,14 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       }
     }
     TR_ADD(0);
-    ok = mbar_wait_relaxed(S.afull + 8u * ab, use & 1u, S.abort_flag, &g_status_tc, XNOR_SLEEP_EPI);
+    ok = mbar_wait_relaxed(S.afull + 8u * ab, fph, S.abort_flag, &g_status_tc, XNOR_SLEEP_EPI);
     TR_ADD(1);
     if (!ok) break;
     tc_fence_after();
     const uint32_t t_acc = t_lane + (uint32_t)(ab * P.NT);
     const int co0 = slab * P.NT;
+    Pix npx = px;
+    if (next_new && it + 1 < nitems) npx = decode(ntile);
 
     auto emit = [&](int b, const int32_t r[16]) {
       if (!valid) return;
@@ -666,14 +820,14 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     // One copy of the code: the next 16 columns are being loaded into `nx` while the
     // current 16 (copied out to `cur`) are scaled and stored.
     int32_t nx[16], cur[16];
-    tmem_ld16(t_acc, nx);
+    tmem_ld16(t_acc + (uint32_t)(e * 16), nx);
 #pragma unroll 1
-    for (int b = 0; b < b_end; ++b) {
+    for (int b = e; b < b_end; b += esplit) {
       tmem_wait16(nx);
 #pragma unroll
       for (int j = 0; j < 16; ++j) cur[j] = nx[j];
-      if (b + 1 < b_end) {
-        tmem_ld16(t_acc + (uint32_t)((b + 1) * 16), nx);
+      if (b + esplit < b_end) {
+        tmem_ld16(t_acc + (uint32_t)((b + esplit) * 16), nx);
       } else {                                   // that was the last load: release the buffer
         tc_fence_before();
         __syncwarp();
@@ -681,13 +835,17 @@ __device__ void epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       }
       emit(b, cur);
     }
-    new_tile = false;
-    if (++slab == P.nslabs) { slab = 0; ++tile; new_tile = true; }
+    px = npx;
+    tile = ntile;
+    slab = nslab;
+    if (++ab == P.nacc) { ab = 0; fph ^= 1u; }
     TR_ADD(2);
   }
   TR_FLUSH(24);
+  return ok;
 }
 
+template <bool kRes>
 __global__ void __launch_bounds__(kThreads, 1)
 binconv_tc_kernel(const __grid_constant__ TcParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -695,7 +853,7 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   const Smem S = carve(smem, P);
 
   if (tid == 0) {
-    for (int i = 0; i < kMaxStages; ++i) {
+    for (int i = 0; i < kMaxBarStages; ++i) {
       mbar_init(S.wfull + 8u * i, kWgtWarps);
       mbar_init(S.wempty + 8u * i, 1);
     }
@@ -703,9 +861,10 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
       mbar_init(S.pfull + 8u * i, 1);
       mbar_init(S.pempty + 8u * i, 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 2 * kPatWarps; ++i) mbar_init(S.rawfull + 8u * i, 1);
+    for (int i = 0; i < kMaxAcc; ++i) {
       mbar_init(S.afull + 8u * i, 1);
-      mbar_init(S.aempty + 8u * i, kEpiWarps);
+      mbar_init(S.aempty + 8u * i, kRes ? kEpiWarps * P.epi_split : kEpiWarps);
     }
     *S.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -733,29 +892,52 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   __syncthreads();
   tc_fence_after();
 
-  // this CTA's contiguous range of work items; item = tile * nslabs + slab
+  // this CTA's contiguous range of work items; item = tile * nslabs + slab (streaming) or
+  // slab * ntiles + tile (resident)
   const long long total = (long long)P.ntiles * P.nslabs;
   const long long i0 = total * blockIdx.x / gridDim.x;
   const long long i1 = total * (blockIdx.x + 1) / gridDim.x;
+#ifdef XNOR_TRACE
+  if (tid == 0 && blockIdx.x < 160) {
+    long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));
+    uint32_t sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_));
+    g_tc_cta[3 * blockIdx.x] = t_; g_tc_cta[3 * blockIdx.x + 2] = sm_;
+  }
+#endif
   if (i0 < i1) {
-    if (warp < kEpiWarps) epilogue_role(P, S, i0, i1, tmem_base, warp, lane);
-    else if (warp == kMmaWarp) mma_role(P, S, i0, i1, tmem_base);
-    else if (warp < kPatWarp0) {
-      const int wt = tid - 32 * kWgtWarp0;
-      if (P.any_swap) {
-        if (P.grp_steps == 4) weight_role<4, true>(P, S, i0, i1, wt, lane);
-        else if (P.grp_steps == 2) weight_role<2, true>(P, S, i0, i1, wt, lane);
-        else weight_role<1, true>(P, S, i0, i1, wt, lane);
-      } else {
-        if (P.grp_steps == 4) weight_role<4, false>(P, S, i0, i1, wt, lane);
-        else if (P.grp_steps == 2) weight_role<2, false>(P, S, i0, i1, wt, lane);
-        else weight_role<1, false>(P, S, i0, i1, wt, lane);
+    const int wt = tid - 32 * kWgtWarp0;
+    if (warp == kMmaWarp) mma_role<kRes>(P, S, i0, i1, tmem_base);
+    else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
+    else if (!kRes) {
+      if (warp < kEpiWarps) epilogue_role<false>(P, S, i0, i1, 0, tmem_base, warp, 0, lane);
+      else weight_dispatch(P, S, i1 - i0, (int)(i0 % P.nslabs), 1u, wt, lane);
+    } else {
+      // Slab visits of this CTA in order.  The weight warps expand the slab, then every
+      // worker warp drains its share of the visit's items.
+      const bool wgt = warp >= kWgtWarp0;
+      const int e = wgt ? 1 + (warp - kWgtWarp0) / 4 : 0;
+      long long it = i0;
+      uint32_t visit = 0;
+      bool ok = true;
+      while (it < i1 && ok) {
+        const int slab = (int)(it / P.ntiles);
+        const long long vend = min(i1, (long long)(slab + 1) * P.ntiles);
+        if (wgt) ok = weight_dispatch(P, S, 1, slab, (visit & 1u) ^ 1u, wt, lane);
+        if (ok && e < P.epi_split)
+          ok = epilogue_role<true>(P, S, it, vend, it - i0, tmem_base, warp & 3, e, lane);
+        it = vend;
+        ++visit;
       }
     }
-    else patch_role(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
   }
   tc_fence_before();
   __syncthreads();
+#ifdef XNOR_TRACE
+  if (tid == 0 && blockIdx.x < 160) {
+    long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));
+    g_tc_cta[3 * blockIdx.x + 1] = t_;
+  }
+#endif
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                  ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
@@ -770,7 +952,22 @@ struct Plan {
   bool ok;
 };
 
-Plan make_plan(const ConvGeom &g) {
+// Weight-thread mapping and stage size for slabs of NT filters: rows_mod threads cover the
+// rows of a K-step, the other thread groups take other K-steps of the stage; a stage is up to
+// 32 KB of expanded weights.
+void plan_stage(TcParams &P) {
+  int ntp = 16;
+  while (ntp < P.NT) ntp *= 2;                          // 16 .. 256
+  P.rows_mod = ntp;
+  const int groups = kWgtThreads / P.rows_mod;          // 1 .. 16
+  P.mps = std::max(2, std::min(8, 1024 / ntp));
+  while (P.mps > 4 && P.nsteps < 3 * P.mps) P.mps /= 2;   // short items: smaller stages start sooner
+  P.grp_steps = std::max(1, P.mps / groups);            // 4, 4, 2, 1, 1
+  P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NT * 32u;
+}
+
+// schedule: 0 = resident when the slab fits, 1 = streaming
+Plan make_plan(const ConvGeom &g, int schedule) {
   Plan pl{};
   pl.ok = false;
   TcParams &P = pl.P;
@@ -787,46 +984,69 @@ Plan make_plan(const ConvGeom &g) {
   const int Wd = std::max(std::max(Wc, g.Wo + dxmax - P.leadX), g.Wo);
   P.Hq = P.leadY + Hd; P.Wq = P.leadX + Wd;
   P.L = (long long)g.N * P.Hq * P.Wq;
-  if (P.L >= (1ll << 31)) return pl;
   P.ntiles = (int)((P.L + kTileM - 1) / kTileM);
   const int halo = (dymax - P.dymin) * P.Wq + (dxmax - P.dxmin);
   P.ppix = (kTileM + halo + 1 + 7) / 8 * 8;             // +1: a lone piece reads one pixel further
+  if (P.L + P.ppix + kTileM >= (1ll << 31)) return pl;  // stream positions stay below 2^31
+  // packed input rows one patch can touch: its stream rows, `stride` input rows each; the
+  // copy is an aligned superset (up to 12 bytes before, 15 after)
+  const long long raw_rows = ((long long)(P.ppix - 1) / P.Wq + 2) * s;
+  const long long raw_bytes = (raw_rows * g.W * g.Cw * 4 + 12 + 15 + 15) / 16 * 16;
+  if (raw_bytes > (long long)kSmemMax) return pl;
+  P.raw_bytes = (uint32_t)raw_bytes;
   P.nplanes = s * s * g.Cw;
   P.patch_bytes = (uint32_t)P.nplanes * (uint32_t)P.ppix * 16u;
-  // filter slabs: as few as fit the accumulator columns, double-buffered when possible
-  P.nslabs = (g.Co + 239) / 240;
-  P.NT = ((g.Co + P.nslabs - 1) / P.nslabs + 15) / 16 * 16;
-  P.nacc = 2 * P.NT <= kMaxAccCols ? 2 : 1;
   // K-steps
   P.row_words = g.kh * g.kw * g.Cw;
   P.nsteps = (P.row_words + 1) / 2;
   if (P.nsteps > kMaxSteps) return pl;
-  // weight-thread mapping: rows_mod threads cover the rows of a K-step, the other thread
-  // groups take other K-steps of the stage; a stage is up to 32 KB of expanded weights
-  int ntp = 16;
-  while (ntp < P.NT) ntp *= 2;                          // 16 .. 256
-  P.rows_mod = ntp;
-  const int groups = kWgtThreads / P.rows_mod;          // 1 .. 16
-  P.mps = std::max(2, std::min(8, 1024 / ntp));
-  while (P.mps > 4 && P.nsteps < 3 * P.mps) P.mps /= 2;   // short items: smaller stages start sooner
-  P.grp_steps = std::max(1, P.mps / groups);            // 4, 4, 2, 1, 1
-  P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NT * 32u;
-  // shared memory: control, weight ring, patch buffers
+  // shared memory: control, weight stages, patch buffers
   P.off_ring = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
   const size_t avail = kSmemMax - P.off_ring;
-  if ((size_t)P.patch_bytes + 2 * (size_t)P.stage_bytes > avail) return pl;
-  // at least 2 stages and 1 patch; then patches up to 3, stages up to 6, one more patch
-  int stages = 2, npb = 1;
-  auto fits = [&](int st, int pb) {
-    return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes <= avail;
+  // st weight stages, pb patch buffers, nraw raw buffers for each of the patch warps at work
+  auto fits = [&](int st, int pb, int nraw) {
+    return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes +
+           (size_t)(std::min(kPatWarps, pb) * nraw) * P.raw_bytes <= avail;
   };
-  while (stages < 4 && fits(stages + 1, npb)) ++stages;
-  while (npb < 3 && fits(stages, npb + 1)) ++npb;
-  while (stages < kMaxStages && fits(stages + 1, npb)) ++stages;
-  while (npb < kMaxPatchBufs && fits(stages, npb + 1)) ++npb;
+  const int min_slabs = (g.Co + 239) / 240;     // as few slabs as fit the accumulator columns
+  int stages = 0, npb = 0;
+  P.resident = 0;
+  if (schedule == 0) {
+    // Resident: the widest slab whose expanded rows fit beside two patches.  Every slab
+    // needs its own patch per tile and narrow MMAs re-read the pixel operand more often, so
+    // (measured) slabs below 128 filters pay only when one slab holds all filters.
+    for (int ns = min_slabs; ns <= 16 && !P.resident; ++ns) {
+      P.nslabs = ns;
+      P.NT = ((g.Co + ns - 1) / ns + 15) / 16 * 16;
+      if (P.NT < 128 && ns > 1) break;
+      plan_stage(P);
+      const int nst = (P.nsteps + P.mps - 1) / P.mps;
+      if (nst <= kMaxBarStages && fits(nst, 2, 1)) {
+        P.resident = 1;
+        stages = nst; npb = 2;
+        while (npb < kMaxPatchBufs && fits(stages, npb + 1, 1)) ++npb;
+      }
+    }
+  }
+  if (!P.resident) {
+    P.nslabs = min_slabs;
+    P.NT = ((g.Co + P.nslabs - 1) / P.nslabs + 15) / 16 * 16;
+    plan_stage(P);
+    if (!fits(2, 1, 1)) return pl;
+    // at least 2 stages and 1 patch; then patches up to 3, stages up to 6, one more patch
+    stages = 2; npb = 1;
+    while (stages < 4 && fits(stages + 1, npb, 1)) ++stages;
+    while (npb < 3 && fits(stages, npb + 1, 1)) ++npb;
+    while (stages < kMaxStages && fits(stages + 1, npb, 1)) ++stages;
+    while (npb < kMaxPatchBufs && fits(stages, npb + 1, 1)) ++npb;
+  }
+  P.nraw = fits(stages, npb, 2) ? 2 : 1;
+  P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
+  P.epi_split = std::min(kEpiSplitMax, P.NT / 16);
   P.stages = stages; P.npb = npb;
   P.off_patch = P.off_ring + (uint32_t)stages * P.stage_bytes;
-  pl.smem = (size_t)P.off_patch + (size_t)npb * P.patch_bytes;
+  P.off_raw = P.off_patch + (uint32_t)npb * P.patch_bytes;
+  pl.smem = (size_t)P.off_raw + (size_t)(std::min(kPatWarps, npb) * P.nraw) * P.raw_bytes;
   // block-scaled instruction descriptor: e2m1 x e2m1, ue8m0 scales, M = 128, N = NT
   P.idesc = (1u << 7) | (1u << 10) | ((uint32_t)(P.NT >> 3) << 17) | (1u << 23) |
             ((uint32_t)(kTileM >> 4) << 24);
@@ -866,32 +1086,41 @@ int sm_count_cached() {
 
 }  // namespace
 
-bool umma_tc_supported(const ConvGeom &g) { return make_plan(g).ok; }
+bool umma_tc_supported(const ConvGeom &g, bool streaming) {
+  return make_plan(g, streaming ? 1 : 0).ok;
+}
 
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, cudaStream_t st) {
-  Plan pl = make_plan(g);
+                              float *out, int32_t *acc_out, bool streaming, cudaStream_t st) {
+  Plan pl = make_plan(g, streaming ? 1 : 0);
   if (!pl.ok) return cudaErrorInvalidValue;
   TcParams &P = pl.P;
   P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
   P.out = out; P.acc_out = acc_out;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(binconv_tc_kernel,
+    cudaError_t e = cudaFuncSetAttribute(binconv_tc_kernel<false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kSmemMax);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(binconv_tc_kernel<true>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
     attr_set = true;
   }
   const long long total = (long long)P.ntiles * P.nslabs;
   const int sms = sm_count_cached();
   const unsigned grid = (unsigned)std::min<long long>(total, sms);
-  binconv_tc_kernel<<<grid, kThreads, pl.smem, st>>>(P);
+  if (P.resident) binconv_tc_kernel<true><<<grid, kThreads, pl.smem, st>>>(P);
+  else binconv_tc_kernel<false><<<grid, kThreads, pl.smem, st>>>(P);
   { cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess && getenv("XNOR_DEBUG")) fprintf(stderr, "binconv_tc launch: %s (grid %u, smem %zu)\n", cudaGetErrorString(e_), grid, pl.smem); return e_; }
 }
 
 #ifdef XNOR_TRACE
+extern "C" int xnor_debug_trace_cta(long long *host480) {
+  return (int)cudaMemcpyFromSymbol(host480, g_tc_cta, sizeof(long long) * 480);
+}
 extern "C" int xnor_debug_trace_tc(long long *host64, int clear) {
   cudaError_t e = cudaMemcpyFromSymbol(host64, g_tc_trace, sizeof(long long) * 64);
   if (clear) {

@@ -43,11 +43,12 @@ cudaError_t launch_binactiv_static(const float *x, const float *scale, const flo
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st);
-// Persistent tensor-core engine (strides 1 and 2).
-bool umma_tc_supported(const ConvGeom &g);
+// Persistent tensor-core engine (strides 1 and 2).  streaming: always take the schedule
+// that re-expands the filters per work item (otherwise only when a slab does not fit).
+bool umma_tc_supported(const ConvGeom &g, bool streaming);
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, cudaStream_t st);
+                              float *out, int32_t *acc_out, bool streaming, cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.
 cudaError_t read_status_tc(int *status);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,

@@ -12,7 +12,8 @@ from util import REL_TOL, assert_close, dev, host, unpack_activations, unpack_we
 
 pytestmark = pytest.mark.gpu
 
-ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_AUTO]
+ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM, B.XNOR_ENGINE_AUTO]
+TC_ENGINES = (B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM)
 
 
 def rng(seed):
@@ -91,7 +92,7 @@ def test_block_parity(oracle, shape, engine):
     g = rng(sum(shape))
     x = g.standard_normal((N, C, H, W)).astype(np.float32)
     w = g.standard_normal((Co, C, kh, kw)).astype(np.float32)
-    if engine == B.XNOR_ENGINE_UMMA and s > 2:
+    if engine in TC_ENGINES and s > 2:
         with pytest.raises(X.XnorError) as e:       # strides a tensor-core engine does not cover
             gpu_block(x, w, s, p, engine=engine)
         assert e.value.status == B.XNOR_ERR_UNSUPPORTED
