@@ -270,6 +270,25 @@ class LayersJob:
         for L in self.layers:
             L.forward(stream)
 
+    def step_branches(self, stream):
+        """The same step for graph capture: the layers do not depend on one another, so each
+        is its own branch of the graph (its launches keep their order) and the GPU may fill
+        the tail of one layer's kernel with another layer's blocks."""
+        torch = self.torch
+        if not hasattr(self, "_side"):
+            self._side = [torch.cuda.Stream() for _ in self.layers[1:]]
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        for L, s in zip(self.layers[1:], self._side):
+            s.wait_event(fork)
+            with torch.cuda.stream(s):
+                L.forward(s)
+        self.layers[0].forward(stream)
+        for s in self._side:
+            join = torch.cuda.Event()
+            join.record(s)
+            stream.wait_event(join)
+
     def e2e_step(self, stream):
         for li, L in enumerate(self.layers):
             L.x.copy_(self.host_x[li], non_blocking=True)
@@ -398,8 +417,12 @@ def run_ours(args):
     graph = None
     if not args.no_graph:
         graph = torch.cuda.CUDAGraph()
+        branches = hasattr(job, "step_branches") and not args.no_branches
         with torch.cuda.graph(graph):
-            job.step(torch.cuda.current_stream())
+            if branches:
+                job.step_branches(torch.cuda.current_stream())
+            else:
+                job.step(torch.cuda.current_stream())
         for _ in range(2):
             graph.replay()
         torch.cuda.synchronize()
@@ -527,7 +550,8 @@ def run_ours(args):
                          % ((job.h2d + job.d2h + (job.act_bytes if args.workload == "chain" else 0))
                             // 1000000),
                    "step": "weight binarisation + BN/BinActiv + BinConv for each layer",
-                   "launch": ("one CUDA graph per step" if graph is not None
+                   "launch": (("one CUDA graph per step, independent layers on parallel branches"
+                               if branches else "one CUDA graph per step") if graph is not None
                               else "one library call per kernel group")},
         "images_per_s": du.job_throughput(job.images, args.steps, world, elapsed_ms),
         "clocks": clocks,
@@ -553,6 +577,8 @@ def main():
     ap.add_argument("--ref-images", type=int, default=8,
                     help="images per layer per step of the reference (oracle) arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-branches", action="store_true",
+                    help="capture the step as one chain of launches (no parallel branches)")
     ap.add_argument("--no-graph", action="store_true",
                     help="time call-by-call launches instead of a CUDA graph of the step")
     ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_stream"])

@@ -542,6 +542,7 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
   uint32_t tm[4];
 #pragma unroll
   for (int r = 0; r < 4; ++r) tm[r] = ((P.tail_mask >> r) & 0x11111111u) * 0xFu;
+  const bool tail = P.tail_mask != 0xFFFFFFFFu;
   const uint32_t row_bytes = (uint32_t)P.W * (uint32_t)P.Cw * 4u;
   const size_t tensor_bytes = (size_t)P.N * P.H * row_bytes;
   const uint32_t raw0 = S.raw + (uint32_t)(pw * P.nraw) * P.raw_bytes;
@@ -617,44 +618,74 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     const uint32_t m0 = (uint32_t)tile * kTileM;
     const uint32_t raw = raw0 + (uint32_t)rb * P.raw_bytes +
                          (uint32_t)(((size_t)g0 * row_bytes) & 15u);   // where row g0 starts
+    // Two stream positions per lane and pass, their loads issued together.  Padding and the
+    // channel tail become the value 0 through the masks: keep (all or nothing) is folded into
+    // the sign mask and the magnitude constants, so a word costs a shift and one logic
+    // operation per register.
 #pragma unroll 1
-    for (int q = lane; q < P.ppix; q += 32) {
-      const uint32_t sq = m0 + (uint32_t)q;
-      const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
-      const int c = (int)(sq - r * (uint32_t)P.Wq);
-      const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
-      const int ry = (int)(r - n * (uint32_t)P.Hq);
-      const bool in = sq < (uint32_t)P.L && ry >= P.leadY && c >= P.leadX;
-      const int rrow = (ry - P.leadY) * s, rcol = (c - P.leadX) * s;
-      const int grow = (int)n * P.H + rrow - g0;     // row inside the raw range (+ py)
+    for (int q0 = lane; q0 < P.ppix; q0 += 64) {
+      bool in[2];
+      int rrow[2], rcol[2], grow[2];
+#pragma unroll
+      for (int b = 0; b < 2; ++b) {
+        const uint32_t sq = m0 + (uint32_t)(q0 + 32 * b);
+        const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
+        const int c = (int)(sq - r * (uint32_t)P.Wq);
+        const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
+        const int ry = (int)(r - n * (uint32_t)P.Hq);
+        in[b] = q0 + 32 * b < P.ppix && sq < (uint32_t)P.L && ry >= P.leadY && c >= P.leadX;
+        rrow[b] = (ry - P.leadY) * s;
+        rcol[b] = (c - P.leadX) * s;
+        grow[b] = (int)n * P.H + rrow[b] - g0;     // row inside the raw range (+ py)
+      }
+      const bool second = q0 + 32 < P.ppix;          // the lane has a second position
 #pragma unroll 1
       for (int phase = 0; phase < phases; ++phase) {
         const int py = phase / s, px = phase - py * s;
-        const bool real = in && rrow + py < P.H && rcol + px < P.W;
-        const uint32_t keep = real ? 0xFFFFFFFFu : 0u;        // padding expands to 0
-        const uint32_t src = raw + (uint32_t)(((grow + py) * P.W + rcol + px) * P.Cw) * 4u;
-        const uint32_t dst = patch + (uint32_t)(phase * P.Cw) * plane_bytes + (uint32_t)q * 16u;
+        uint32_t src[2], sm[2], mc[2][3];
+        bool real[2];
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+          real[b] = in[b] && rrow[b] + py < P.H && rcol[b] + px < P.W;
+          const uint32_t keep = real[b] ? 0xFFFFFFFFu : 0u;
+          src[b] = raw + (uint32_t)(((grow[b] + py) * P.W + rcol[b] + px) * P.Cw) * 4u;
+          sm[b] = 0x88888888u & keep;
+          mc[b][0] = 0xCCCCCCCCu & keep; mc[b][1] = 0xAAAAAAAAu & keep; mc[b][2] = 0x99999999u & keep;
+        }
+        const uint32_t dst = patch + (uint32_t)(phase * P.Cw) * plane_bytes + (uint32_t)q0 * 16u;
 #pragma unroll 1
         for (int w0 = 0; w0 < P.Cw; w0 += 4) {
-          uint32_t wv[4] = {0u, 0u, 0u, 0u};
-          if (real) {
-            if (vec) {
-              lds128(src + (uint32_t)w0 * 4u, wv);
-            } else {
+          uint32_t wv[2][4];
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                if (w0 + i < P.Cw) wv[i] = lds32(src + (uint32_t)(w0 + i) * 4u);
+          for (int b = 0; b < 2; ++b) {
+            wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
+            if (real[b]) {
+              if (vec) {
+                lds128(src[b] + (uint32_t)w0 * 4u, wv[b]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                  if (w0 + i < P.Cw) wv[b][i] = lds32(src[b] + (uint32_t)(w0 + i) * 4u);
+              }
             }
           }
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            if (w0 + i < P.Cw) {
-              uint32_t v[4];
-              expand_signs<true>(wv[i], v);
-              const bool last = w0 + i == P.Cw - 1;           // channels beyond C_in are 0
+          for (int b = 0; b < 2; ++b) {
+            if (b == 0 || second) {
 #pragma unroll
-              for (int rr = 0; rr < 4; ++rr) v[rr] &= last ? (tm[rr] & keep) : keep;
-              sts128(dst + (uint32_t)(w0 + i) * plane_bytes, v[0], v[1], v[2], v[3]);
+              for (int i = 0; i < 4; ++i) {
+                if (w0 + i < P.Cw) {
+                  const uint32_t w = wv[b][i];
+                  uint32_t v0 = ((w << 3) & sm[b]) ^ mc[b][0];
+                  uint32_t v1 = ((w << 2) & sm[b]) ^ mc[b][1];
+                  uint32_t v2 = ((w << 1) & sm[b]) ^ mc[b][2];
+                  uint32_t v3 = (w & sm[b]) ^ mc[b][2];
+                  if (tail && w0 + i == P.Cw - 1) {       // channels beyond C_in are 0
+                    v0 &= tm[0]; v1 &= tm[1]; v2 &= tm[2]; v3 &= tm[3];
+                  }
+                  sts128(dst + (uint32_t)(w0 + i) * plane_bytes + (uint32_t)(b * 32 * 16), v0, v1, v2, v3);
+                }
+              }
             }
           }
         }
@@ -696,6 +727,10 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   const int b_end = P.NT / 16;
   const int esplit = kRes ? P.epi_split : 1;
   const size_t HoWo = (size_t)P.Ho * P.Wo;
+  const uint32_t howo = (uint32_t)HoWo;
+  // the fast store paths: offsets of 16 consecutive filters fit 32 bits, no integer output
+  const bool small = HoWo < ((size_t)1 << 27) && P.acc_out == nullptr;
+  const bool plain = small && P.residual == nullptr, with_res = small && P.residual != nullptr;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tile, slab;
   if (kRes) { slab = (int)(i0 / P.ntiles); tile = (int)(i0 - (long long)slab * P.ntiles); }
@@ -760,39 +795,37 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     Pix npx = px;
     if (next_new && it + 1 < nitems) npx = decode(ntile);
 
+    // Every store address is formed on its own from the group's base (no chain of pointer
+    // increments).
     auto emit = [&](int b, const int32_t r[16]) {
       if (!valid) return;
       const int co = co0 + b * 16;
       float *op = P.out + obase + (size_t)co * HoWo;
-      if (co + 16 <= P.Co && P.acc_out == nullptr && P.residual == nullptr) {
+      if (co + 16 <= P.Co && plain) {
+        float4 al[4];
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4)
+          al[j4] = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
-          const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
-          const float a4[4] = {al.x, al.y, al.z, al.w};
+          const float a4[4] = {al[j4].x, al[j4].y, al[j4].z, al[j4].w};
 #pragma unroll
-          for (int jj = 0; jj < 4; ++jj) {
-            *op = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
-            op += HoWo;
-          }
+          for (int jj = 0; jj < 4; ++jj)
+            op[(uint32_t)(j4 * 4 + jj) * howo] =
+                __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
         }
-      } else if (co + 16 <= P.Co && P.acc_out == nullptr) {
+      } else if (co + 16 <= P.Co && with_res) {
+        const float *rp = P.residual + obase + (size_t)co * HoWo;
         float res[16];
-        if (P.residual) {
-          const float *rp = P.residual + obase + (size_t)co * HoWo;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) res[j] = rp[(size_t)j * HoWo];
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) res[j] = 0.0f;
-        }
+        for (int j = 0; j < 16; ++j) res[j] = rp[(size_t)j * HoWo];
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
           const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
           const float a4[4] = {al.x, al.y, al.z, al.w};
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
-            const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
-            *op = P.residual ? v + res[j4 * 4 + jj] : v;
+            *op = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]) + res[j4 * 4 + jj];
             op += HoWo;
           }
         }
