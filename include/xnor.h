@@ -198,16 +198,25 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
  *                      accumulation of integers; strides 1 and 2, shapes whose
  *                      activation patch fits shared memory.  The expanded
  *                      filters of a slab stay in shared memory while a CTA
- *                      walks the pixel tiles, when they fit
- *   XNOR_ENGINE_UMMA_STREAM  the same engine with the schedule it falls back
- *                      to when a slab does not fit: filters re-expanded
- *                      through a ring of stages for every work item
+ *                      walks the pixel tiles, when they fit; CTA pairs (one
+ *                      MMA instruction drives two SMs, each CTA holding half
+ *                      of the slab's filters) where the shape allows
+ *   The remaining values pin one variant of that engine (for tests and
+ *   measurements):
+ *   XNOR_ENGINE_UMMA_STREAM       one CTA per SM, filters re-expanded through
+ *                                 a ring of stages for every work item
+ *   XNOR_ENGINE_UMMA_SINGLE       one CTA per SM, resident filters if they fit
+ *   XNOR_ENGINE_UMMA_PAIR         CTA pairs, resident filters if they fit
+ *   XNOR_ENGINE_UMMA_PAIR_STREAM  CTA pairs, filters always re-expanded
  */
 typedef enum {
   XNOR_ENGINE_AUTO = 0,
   XNOR_ENGINE_POPC = 1,
   XNOR_ENGINE_UMMA = 2,
-  XNOR_ENGINE_UMMA_STREAM = 3
+  XNOR_ENGINE_UMMA_STREAM = 3,
+  XNOR_ENGINE_UMMA_SINGLE = 4,
+  XNOR_ENGINE_UMMA_PAIR = 5,
+  XNOR_ENGINE_UMMA_PAIR_STREAM = 6
 } xnor_engine;
 xnor_status xnor_set_engine(xnor_engine e);
 xnor_engine xnor_get_engine(void);

@@ -23,6 +23,9 @@ XNOR_ENGINE_AUTO = 0
 XNOR_ENGINE_POPC = 1
 XNOR_ENGINE_UMMA = 2
 XNOR_ENGINE_UMMA_STREAM = 3
+XNOR_ENGINE_UMMA_SINGLE = 4
+XNOR_ENGINE_UMMA_PAIR = 5
+XNOR_ENGINE_UMMA_PAIR_STREAM = 6
 
 EXPORTS = [
     "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",

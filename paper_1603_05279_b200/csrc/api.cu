@@ -45,8 +45,7 @@ int xnor_out_extent(int in, int k, int stride, int pad) {
 }
 
 xnor_status xnor_set_engine(xnor_engine e) {
-  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC && e != XNOR_ENGINE_UMMA &&
-      e != XNOR_ENGINE_UMMA_STREAM)
+  if ((int)e < (int)XNOR_ENGINE_AUTO || (int)e > (int)XNOR_ENGINE_UMMA_PAIR_STREAM)
     return XNOR_ERR_INVALID_ARG;
   g_engine = e;
   return XNOR_OK;
@@ -105,12 +104,17 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
   if ((long long)d->C_in * d->k_h * d->k_w >= (1LL << 24)) return XNOR_ERR_UNSUPPORTED;
   const xnor::ConvGeom g = xnor::make_geom(*d);
   const cudaStream_t st = (cudaStream_t)cuda_stream;
-  const bool streaming = g_engine == XNOR_ENGINE_UMMA_STREAM;
-  const bool tc_ok = xnor::umma_tc_supported(g, streaming);
-  if ((g_engine == XNOR_ENGINE_UMMA || streaming) && !tc_ok) return XNOR_ERR_UNSUPPORTED;
+  xnor::TcVariant variant = xnor::kTcAuto;
+  if (g_engine == XNOR_ENGINE_UMMA_STREAM) variant = xnor::kTcSingleStream;
+  else if (g_engine == XNOR_ENGINE_UMMA_SINGLE) variant = xnor::kTcSingle;
+  else if (g_engine == XNOR_ENGINE_UMMA_PAIR) variant = xnor::kTcPair;
+  else if (g_engine == XNOR_ENGINE_UMMA_PAIR_STREAM) variant = xnor::kTcPairStream;
+  const bool tc_ok = xnor::umma_tc_supported(g, variant);
+  if (g_engine != XNOR_ENGINE_AUTO && g_engine != XNOR_ENGINE_POPC && !tc_ok)
+    return XNOR_ERR_UNSUPPORTED;
   if (g_engine != XNOR_ENGINE_POPC && tc_ok)
     return from_cuda(xnor::launch_binconv_tc(x_packed, w_packed, alpha, K, residual, g, out,
-                                             acc_out, streaming, st));
+                                             acc_out, variant, st));
   return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, out,
                                              acc_out, (cudaStream_t)cuda_stream));
 }

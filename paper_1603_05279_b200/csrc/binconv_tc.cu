@@ -144,6 +144,8 @@ struct TcParams {
   uint32_t adesc_lo[kMaxSteps];
   uint32_t swap_mask[32];              // bit j: word 2j+1 is the first piece of step j
   int row_words;               // packed words per filter row = k_h*k_w*Cw
+  int pair;                    // 1: two CTAs (a cluster) share every MMA: 256 pixels x NT filters
+  int NTh;                     // filter rows of a slab that one CTA expands and holds: NT or NT/2
   int resident;                // 1: resident schedule (stages = all stages of a slab)
   int epi_split;               // warps per lane quarter that drain an accumulator
   int any_swap;                // some bit of swap_mask is set
@@ -176,6 +178,48 @@ __device__ __forceinline__ void umma_commit_elected(uint32_t bar, uint32_t elect
       "setp.ne.b32 q, %1, 0;\n\t"
       "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
       ::"r"(bar), "r"(elected) : "memory");
+}
+
+// The same for a CTA pair: one instruction drives the tensor cores of both SMs (M = 256: rows
+// 0-127 from this CTA's patch into its tensor memory, rows 128-255 the peer's; each CTA
+// supplies half of the N filter rows).  Commits signal the barrier at the same offset in both.
+__device__ __forceinline__ void umma_mxf4_pair_elected(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                                       uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                       uint32_t sf, uint32_t accumulate,
+                                                       uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.ne.b32 q, %8, 0;\n\t"
+      "@q tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], da, db, %5, [%7], [%7], p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
+        "r"(sf), "r"(elected)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_commit_pair_elected(uint32_t bar, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t.reg .b16 mask;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "mov.b16 mask, 3;\n\t"
+      "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], mask;\n\t}"
+      ::"r"(bar), "r"(elected) : "memory");
+}
+
+template <bool kPair>
+__device__ __forceinline__ void umma_issue(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                           uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t sf,
+                                           uint32_t accumulate, uint32_t elected) {
+  if (kPair) umma_mxf4_pair_elected(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, sf, accumulate, elected);
+  else umma_mxf4_elected(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, sf, accumulate, elected);
+}
+
+template <bool kPair>
+__device__ __forceinline__ void umma_commit_to(uint32_t bar, uint32_t elected) {
+  if (kPair) umma_commit_pair_elected(bar, elected);
+  else umma_commit_elected(bar, elected);
 }
 
 __device__ __forceinline__ uint32_t elect_one() {
@@ -246,6 +290,7 @@ struct Smem {
   uint32_t *tmem_slot;
   volatile int *abort_flag;
   uint32_t ring, patch, raw;                              // shared-space byte addresses
+  uint32_t rank;                                          // CTA rank in its pair (0 = issues the MMAs)
 };
 
 __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
@@ -264,6 +309,7 @@ __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
   s.ring = base + P.off_ring;
   s.patch = base + P.off_patch;
   s.raw = base + P.off_raw;
+  s.rank = P.pair ? cluster_ctarank() : 0u;
   return s;
 }
 
@@ -276,25 +322,25 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity,
 }
 
 // The MMAs of one full weight stage, unrolled.
-template <int MPS>
+template <int MPS, bool kPair>
 __device__ __forceinline__ void issue_stage(const TcParams &P, int j0, uint32_t d_tmem,
                                             uint32_t patch_lo, uint32_t a_hi, uint32_t b_lo,
                                             uint32_t b_hi, uint32_t b_step, uint32_t tmem_sf,
                                             uint32_t first, uint32_t el) {
 #pragma unroll
   for (int jj = 0; jj < MPS; ++jj)
-    umma_mxf4_elected(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, a_hi, b_lo + (uint32_t)jj * b_step,
+    umma_issue<kPair>(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, a_hi, b_lo + (uint32_t)jj * b_step,
                       b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u, el);
 }
 
 // kRes: resident schedule.  The stage barriers are then waited for only on the first item of
 // a slab visit (the slab stays in shared memory afterwards) and released only on the last.
-template <bool kRes>
+template <bool kRes, bool kPair>
 __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long long i1,
                          uint32_t tmem_base) {
   const uint32_t tmem_sf = tmem_base + (uint32_t)kSfCol;
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
-  const uint32_t b_lbo = (uint32_t)P.NT * 16u;
+  const uint32_t b_lbo = (uint32_t)P.NTh * 16u;
   // descriptor halves: high word = stride between 8-row groups (128 B) and the version bit
   const uint32_t desc_hi = (128u >> 4) | (1u << 14);
   const uint32_t b_lo0 = ((S.ring & 0x3FFFFu) >> 4) | ((b_lbo >> 4) << 16);   // stage 0, K-step 0
@@ -338,17 +384,17 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
         tc_fence_after();
       }
       TR_ADD(3);
-      if (nj == 4) issue_stage<4>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
-      else if (nj == 2) issue_stage<2>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
-      else if (nj == 8) issue_stage<8>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      if (nj == 4) issue_stage<4, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      else if (nj == 2) issue_stage<2, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      else if (nj == 8) issue_stage<8, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
       else {
         for (int jj = 0; jj < nj; ++jj)
-          umma_mxf4_elected(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, desc_hi,
+          umma_issue<kPair>(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, desc_hi,
                             b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc, tmem_sf,
                             jj == 0 ? first : 1u, el);
       }
       TR_ADD(4);
-      if (visit_last) umma_commit_elected(S.wempty + 8u * ws, el);
+      if (visit_last) umma_commit_to<kPair>(S.wempty + 8u * ws, el);
       TR_ADD(5);
       if (++ws == P.stages) { ws = 0; if (!kRes) wph ^= 1u; }
     }
@@ -357,15 +403,15 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
       // every item has its own patch; the barrier phase of the slab flips with the visit
       if (visit_last) wph ^= 1u;
       if (++tile == P.ntiles) tile = 0;
-      umma_commit_elected(S.afull + 8u * ab, el);
-      umma_commit_elected(S.pempty + 8u * pb, el);
+      umma_commit_to<kPair>(S.afull + 8u * ab, el);
+      umma_commit_to<kPair>(S.pempty + 8u * pb, el);
       if (++pb == P.npb) { pb = 0; pph ^= 1u; }
     } else {
       // next item: same tile (next slab) or the next tile
       new_tile = false;
       if (++slab == P.nslabs) { slab = 0; new_tile = true; }
-      umma_commit_elected(S.afull + 8u * ab, el);
-      if (new_tile || it + 1 == nitems) umma_commit_elected(S.pempty + 8u * pb, el);
+      umma_commit_to<kPair>(S.afull + 8u * ab, el);
+      if (new_tile || it + 1 == nitems) umma_commit_to<kPair>(S.pempty + 8u * pb, el);
       if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
     }
     if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
@@ -403,8 +449,9 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const int row = wt % P.rows_mod, grp = wt / P.rows_mod;
   constexpr int gs = kUnits;
-  const bool grp_on = grp * gs < P.mps && row < P.NT;
-  const uint32_t b_lbo = (uint32_t)P.NT * 16u;
+  const bool grp_on = grp * gs < P.mps && row < P.NTh;
+  const uint32_t b_lbo = (uint32_t)P.NTh * 16u;
+  const int row_co = (int)S.rank * P.NTh + row;          // this thread's filter inside a slab
   const int jj0 = grp * gs;                         // first K-step of this thread inside a stage
   const int nplain = (P.row_words >> 1);            // K-steps j < nplain have both words
   WCursor fc{i0, 0, slab0}, cc{i0, 0, slab0};
@@ -414,7 +461,7 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
   const uint2 *wp2 = reinterpret_cast<const uint2 *>(P.wp);
   uint2 pf[kPrefetch][kUnits];
   auto fetch = [&](uint2 dst[kUnits], const WCursor &c) {
-    const int co = c.slab * P.NT + row;
+    const int co = c.slab * P.NT + row_co;
     const bool on = grp_on && c.item < i1 && co < P.Co;
     const int j0 = c.st * P.mps + jj0;
     if (on && j0 + gs <= P.nsteps) {
@@ -442,7 +489,7 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
     TR_ADD(0);
     if (!ok) break;
     const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
-    const int co = cc.slab * P.NT + row;
+    const int co = cc.slab * P.NT + row_co;
     const int j0 = cc.st * P.mps + jj0;
     const bool on = grp_on && co < P.Co;
     if (on && j0 + gs <= nplain) {
@@ -482,7 +529,7 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
     TR_ADD(1);
     fence_proxy_async();
     __syncwarp();
-    if (lane == 0) mbar_arrive(S.wfull + 8u * ws);
+    if (lane == 0) { if (P.pair) mbar_arrive_cluster(S.wfull + 8u * ws, 0u); else mbar_arrive(S.wfull + 8u * ws); }
     if (++ws == P.stages) { ws = 0; wph ^= 1u; }
     advance(cc);
     // the queue of packed words moves up one stage; the freed slot is refilled
@@ -552,8 +599,10 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     return kRes ? (int)((tile_r0 + seq) % (uint32_t)P.ntiles) : tile0 + (int)seq;
   };
   // input rows [g0, g1) (of the N*H rows of the tensor) that the patch of a tile reads
+  // pairs: work tile t is stream tiles 2t (rank 0) and 2t + 1 (rank 1)
+  const uint32_t tmul = P.pair ? 2u : 1u;
   auto row_range = [&](int tile, int &g0, int &g1) {
-    const uint32_t m0 = (uint32_t)tile * kTileM;
+    const uint32_t m0 = ((uint32_t)tile * tmul + S.rank) * kTileM;
     const uint32_t mlast = min(m0 + (uint32_t)P.ppix - 1u, (uint32_t)P.L - 1u);
     const uint32_t r0 = fast_div(m0, P.div_wq_m, P.div_wq_s);
     const uint32_t r1 = fast_div(mlast, P.div_wq_m, P.div_wq_s);
@@ -615,7 +664,7 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     TR_ADD(0);
     if (!ok) break;
     const uint32_t patch = S.patch + (uint32_t)pb * P.patch_bytes;
-    const uint32_t m0 = (uint32_t)tile * kTileM;
+    const uint32_t m0 = ((uint32_t)tile * tmul + S.rank) * kTileM;
     const uint32_t raw = raw0 + (uint32_t)rb * P.raw_bytes +
                          (uint32_t)(((size_t)g0 * row_bytes) & 15u);   // where row g0 starts
     // Two stream positions per lane and pass, their loads issued together.  Padding and the
@@ -696,7 +745,7 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     __syncwarp();
     const uint32_t next = seq + (uint32_t)(P.nraw * active);   // reuses this raw buffer
     if (lane == 0) {
-      mbar_arrive(S.pfull + 8u * pb);
+      if (P.pair) mbar_arrive_cluster(S.pfull + 8u * pb, 0u); else mbar_arrive(S.pfull + 8u * pb);
       if (next < npatches) start_copy(next, rb);
     }
     if (next < npatches) { if (rb) pend[1] = true; else pend[0] = true; }
@@ -740,7 +789,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   struct Pix { bool valid; float kv; size_t obase; };
   auto decode = [&](int t) {
     Pix px{false, 0.0f, 0};
-    const uint32_t m = (uint32_t)t * kTileM + (uint32_t)(quarter * 32 + lane);
+    const uint32_t m = ((uint32_t)t * (P.pair ? 2u : 1u) + S.rank) * kTileM + (uint32_t)(quarter * 32 + lane);
     if (m < (uint32_t)P.L) {
       const uint32_t r = fast_div(m, P.div_wq_m, P.div_wq_s);
       const int ox = (int)(m - r * (uint32_t)P.Wq);
@@ -864,7 +913,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       } else {                                   // that was the last load: release the buffer
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
+        if (lane == 0) { if (P.pair) mbar_arrive_cluster(S.aempty + 8u * ab, 0u); else mbar_arrive(S.aempty + 8u * ab); }
       }
       emit(b, cur);
     }
@@ -878,7 +927,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   return ok;
 }
 
-template <bool kRes>
+template <bool kRes, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 binconv_tc_kernel(const __grid_constant__ TcParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -886,26 +935,36 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   const Smem S = carve(smem, P);
 
   if (tid == 0) {
+    // In a pair the producers of both CTAs arrive on the barriers of rank 0 (whose MMA warp
+    // waits for them); the MMA warp's commits reach the consumer barriers of both CTAs.
+    constexpr uint32_t kCtas = kPair ? 2u : 1u;
     for (int i = 0; i < kMaxBarStages; ++i) {
-      mbar_init(S.wfull + 8u * i, kWgtWarps);
+      mbar_init(S.wfull + 8u * i, kWgtWarps * kCtas);
       mbar_init(S.wempty + 8u * i, 1);
     }
     for (int i = 0; i < kMaxPatchBufs; ++i) {
-      mbar_init(S.pfull + 8u * i, 1);
+      mbar_init(S.pfull + 8u * i, kCtas);
       mbar_init(S.pempty + 8u * i, 1);
     }
     for (int i = 0; i < 2 * kPatWarps; ++i) mbar_init(S.rawfull + 8u * i, 1);
     for (int i = 0; i < kMaxAcc; ++i) {
       mbar_init(S.afull + 8u * i, 1);
-      mbar_init(S.aempty + 8u * i, kRes ? kEpiWarps * P.epi_split : kEpiWarps);
+      mbar_init(S.aempty + 8u * i, (kRes ? kEpiWarps * P.epi_split : kEpiWarps) * kCtas);
     }
     *S.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kMmaWarp) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(S.tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (kPair) {
+      // the same warp of both CTAs of the pair allocates, at the same shared-memory offset
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(S.tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(S.tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -924,12 +983,15 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // no CTA of a pair signals a barrier of the other before that one has set it up
+  if (kPair) cluster_sync();
 
-  // this CTA's contiguous range of work items; item = tile * nslabs + slab (streaming) or
-  // slab * ntiles + tile (resident)
+  // this CTA's (pair's) contiguous range of work items; item = tile * nslabs + slab
+  // (streaming) or slab * ntiles + tile (resident); for a pair a tile is two stream tiles
   const long long total = (long long)P.ntiles * P.nslabs;
-  const long long i0 = total * blockIdx.x / gridDim.x;
-  const long long i1 = total * (blockIdx.x + 1) / gridDim.x;
+  const unsigned unit = kPair ? blockIdx.x >> 1 : blockIdx.x, units = kPair ? gridDim.x >> 1 : gridDim.x;
+  const long long i0 = total * unit / units;
+  const long long i1 = total * (unit + 1) / units;
 #ifdef XNOR_TRACE
   if (tid == 0 && blockIdx.x < 160) {
     long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));
@@ -939,7 +1001,7 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
 #endif
   if (i0 < i1) {
     const int wt = tid - 32 * kWgtWarp0;
-    if (warp == kMmaWarp) mma_role<kRes>(P, S, i0, i1, tmem_base);
+    if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base); }
     else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
     else if (!kRes) {
       if (warp < kEpiWarps) epilogue_role<false>(P, S, i0, i1, 0, tmem_base, warp, 0, lane);
@@ -971,9 +1033,15 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     g_tc_cta[3 * blockIdx.x + 1] = t_;
   }
 #endif
+  // both CTAs of a pair are done with each other's barriers and tensor memory
+  if (kPair) cluster_sync();
   if (warp == kMmaWarp) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                 ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    if (kPair)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
+                   ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                   ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
   }
 }
 
@@ -990,17 +1058,24 @@ struct Plan {
 // 32 KB of expanded weights.
 void plan_stage(TcParams &P) {
   int ntp = 16;
-  while (ntp < P.NT) ntp *= 2;                          // 16 .. 256
+  while (ntp < P.NTh) ntp *= 2;                         // 16 .. 256
   P.rows_mod = ntp;
   const int groups = kWgtThreads / P.rows_mod;          // 1 .. 16
   P.mps = std::max(2, std::min(8, 1024 / ntp));
   while (P.mps > 4 && P.nsteps < 3 * P.mps) P.mps /= 2;   // short items: smaller stages start sooner
   P.grp_steps = std::max(1, P.mps / groups);            // 4, 4, 2, 1, 1
-  P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NT * 32u;
+  P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NTh * 32u;
 }
 
-// schedule: 0 = resident when the slab fits, 1 = streaming
-Plan make_plan(const ConvGeom &g, int schedule) {
+// Filters per slab for `ns` slabs.  A pair splits the rows of a slab between its two CTAs
+// (halves of a multiple of 16 rows each).
+int slab_width(int Co, int ns, bool pair) {
+  const int q = pair ? 32 : 16;
+  return ((Co + ns - 1) / ns + q - 1) / q * q;
+}
+
+// schedule: 0 = resident when the slab fits, 1 = streaming.  pair: CTA pairs (clusters of 2).
+Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
   Plan pl{};
   pl.ok = false;
   TcParams &P = pl.P;
@@ -1018,9 +1093,11 @@ Plan make_plan(const ConvGeom &g, int schedule) {
   P.Hq = P.leadY + Hd; P.Wq = P.leadX + Wd;
   P.L = (long long)g.N * P.Hq * P.Wq;
   P.ntiles = (int)((P.L + kTileM - 1) / kTileM);
+  P.pair = pair ? 1 : 0;
+  if (pair) P.ntiles = (P.ntiles + 1) / 2;               // a work tile is two stream tiles
   const int halo = (dymax - P.dymin) * P.Wq + (dxmax - P.dxmin);
   P.ppix = (kTileM + halo + 1 + 7) / 8 * 8;             // +1: a lone piece reads one pixel further
-  if (P.L + P.ppix + kTileM >= (1ll << 31)) return pl;  // stream positions stay below 2^31
+  if (P.L + P.ppix + 2 * kTileM >= (1ll << 31)) return pl;  // stream positions stay below 2^31
   // packed input rows one patch can touch: its stream rows, `stride` input rows each; the
   // copy is an aligned superset (up to 12 bytes before, 15 after)
   const long long raw_rows = ((long long)(P.ppix - 1) / P.Wq + 2) * s;
@@ -1041,7 +1118,9 @@ Plan make_plan(const ConvGeom &g, int schedule) {
     return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes +
            (size_t)(std::min(kPatWarps, pb) * nraw) * P.raw_bytes <= avail;
   };
-  const int min_slabs = (g.Co + 239) / 240;     // as few slabs as fit the accumulator columns
+  // as few slabs as fit two accumulators in the tensor-memory columns
+  const int max_nt = pair ? 224 : 240;
+  const int min_slabs = (g.Co + max_nt - 1) / max_nt;
   int stages = 0, npb = 0;
   P.resident = 0;
   if (schedule == 0) {
@@ -1050,7 +1129,8 @@ Plan make_plan(const ConvGeom &g, int schedule) {
     // (measured) slabs below 128 filters pay only when one slab holds all filters.
     for (int ns = min_slabs; ns <= 16 && !P.resident; ++ns) {
       P.nslabs = ns;
-      P.NT = ((g.Co + ns - 1) / ns + 15) / 16 * 16;
+      P.NT = slab_width(g.Co, ns, pair);
+      P.NTh = pair ? P.NT / 2 : P.NT;
       if (P.NT < 128 && ns > 1) break;
       plan_stage(P);
       const int nst = (P.nsteps + P.mps - 1) / P.mps;
@@ -1063,7 +1143,8 @@ Plan make_plan(const ConvGeom &g, int schedule) {
   }
   if (!P.resident) {
     P.nslabs = min_slabs;
-    P.NT = ((g.Co + P.nslabs - 1) / P.nslabs + 15) / 16 * 16;
+    P.NT = slab_width(g.Co, P.nslabs, pair);
+    P.NTh = pair ? P.NT / 2 : P.NT;
     plan_stage(P);
     if (!fits(2, 1, 1)) return pl;
     // at least 2 stages and 1 patch; then patches up to 3, stages up to 6, one more patch
@@ -1080,9 +1161,10 @@ Plan make_plan(const ConvGeom &g, int schedule) {
   P.off_patch = P.off_ring + (uint32_t)stages * P.stage_bytes;
   P.off_raw = P.off_patch + (uint32_t)npb * P.patch_bytes;
   pl.smem = (size_t)P.off_raw + (size_t)(std::min(kPatWarps, npb) * P.nraw) * P.raw_bytes;
-  // block-scaled instruction descriptor: e2m1 x e2m1, ue8m0 scales, M = 128, N = NT
+  // block-scaled instruction descriptor: e2m1 x e2m1, ue8m0 scales, M = 128 (256 for a
+  // pair), N = NT
   P.idesc = (1u << 7) | (1u << 10) | ((uint32_t)(P.NT >> 3) << 17) | (1u << 23) |
-            ((uint32_t)(kTileM >> 4) << 24);
+            ((uint32_t)((pair ? 2 * kTileM : kTileM) >> 4) << 24);
   const int crem = g.C - 32 * (g.Cw - 1);
   P.tail_mask = crem == 32 ? 0xFFFFFFFFu : ((1u << crem) - 1u);
   for (int j = 0; j < 32; ++j) P.swap_mask[j] = 0u;
@@ -1119,35 +1201,81 @@ int sm_count_cached() {
 
 }  // namespace
 
-bool umma_tc_supported(const ConvGeom &g, bool streaming) {
-  return make_plan(g, streaming ? 1 : 0).ok;
+namespace {
+
+// The plan of a variant.  kTcAuto (measured on the AlexNet and ResNet-18 shapes): one CTA per
+// SM unless only a pair, each CTA holding half of a slab, can keep the filters resident.
+Plan plan_variant(const ConvGeom &g, TcVariant v) {
+  switch (v) {
+    case kTcSingle: return make_plan(g, 0, false);
+    case kTcSingleStream: return make_plan(g, 1, false);
+    case kTcPair: return make_plan(g, 0, true);
+    case kTcPairStream: return make_plan(g, 1, true);
+    default: break;
+  }
+  Plan single = make_plan(g, 0, false);
+  if (single.ok && single.P.resident) return single;
+  Plan pair = make_plan(g, 0, true);
+  if (pair.ok && (pair.P.resident || !single.ok)) return pair;
+  return single;
 }
+
+template <bool kRes, bool kPair>
+cudaError_t launch_variant(const Plan &pl, unsigned units, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kPair ? 2 * units : units);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = pl.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kPair ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, binconv_tc_kernel<kRes, kPair>, pl.P);
+}
+
+}  // namespace
+
+bool umma_tc_supported(const ConvGeom &g, TcVariant v) { return plan_variant(g, v).ok; }
 
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, bool streaming, cudaStream_t st) {
-  Plan pl = make_plan(g, streaming ? 1 : 0);
+                              float *out, int32_t *acc_out, TcVariant variant, cudaStream_t st) {
+  Plan pl = plan_variant(g, variant);
   if (!pl.ok) return cudaErrorInvalidValue;
   TcParams &P = pl.P;
   P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
   P.out = out; P.acc_out = acc_out;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(binconv_tc_kernel<false>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmemMax);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(binconv_tc_kernel<true>,
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+    const void *kernels[4] = {(const void *)binconv_tc_kernel<false, false>,
+                              (const void *)binconv_tc_kernel<true, false>,
+                              (const void *)binconv_tc_kernel<false, true>,
+                              (const void *)binconv_tc_kernel<true, true>};
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+      e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)kSmemMax);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
     attr_set = true;
   }
   const long long total = (long long)P.ntiles * P.nslabs;
   const int sms = sm_count_cached();
-  const unsigned grid = (unsigned)std::min<long long>(total, sms);
-  if (P.resident) binconv_tc_kernel<true><<<grid, kThreads, pl.smem, st>>>(P);
-  else binconv_tc_kernel<false><<<grid, kThreads, pl.smem, st>>>(P);
-  { cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess && getenv("XNOR_DEBUG")) fprintf(stderr, "binconv_tc launch: %s (grid %u, smem %zu)\n", cudaGetErrorString(e_), grid, pl.smem); return e_; }
+  // one CTA per SM, or one pair per two SMs
+  const unsigned units = (unsigned)std::min<long long>(total, P.pair ? sms / 2 : sms);
+  cudaError_t e_;
+  if (P.pair) e_ = P.resident ? launch_variant<true, true>(pl, units, st) : launch_variant<false, true>(pl, units, st);
+  else e_ = P.resident ? launch_variant<true, false>(pl, units, st) : launch_variant<false, false>(pl, units, st);
+  if (e_ != cudaSuccess) {
+    (void)cudaGetLastError();
+    if (getenv("XNOR_DEBUG"))
+      fprintf(stderr, "binconv_tc launch: %s (units %u, pair %d, smem %zu)\n", cudaGetErrorString(e_),
+              units, P.pair, pl.smem);
+  }
+  return e_;
 }
 
 #ifdef XNOR_TRACE

@@ -43,12 +43,14 @@ cudaError_t launch_binactiv_static(const float *x, const float *scale, const flo
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st);
-// Persistent tensor-core engine (strides 1 and 2).  streaming: always take the schedule
-// that re-expands the filters per work item (otherwise only when a slab does not fit).
-bool umma_tc_supported(const ConvGeom &g, bool streaming);
+// Persistent tensor-core engine (strides 1 and 2).  Variants: one CTA per SM or CTA pairs
+// (one MMA drives two SMs), each with the filters of a slab resident in shared memory when
+// they fit or always streamed through a ring (re-expanded per work item).
+enum TcVariant { kTcAuto = 0, kTcSingle, kTcSingleStream, kTcPair, kTcPairStream };
+bool umma_tc_supported(const ConvGeom &g, TcVariant v);
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, bool streaming, cudaStream_t st);
+                              float *out, int32_t *acc_out, TcVariant v, cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.
 cudaError_t read_status_tc(int *status);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,

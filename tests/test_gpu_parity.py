@@ -12,8 +12,10 @@ from util import REL_TOL, assert_close, dev, host, unpack_activations, unpack_we
 
 pytestmark = pytest.mark.gpu
 
-ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM, B.XNOR_ENGINE_AUTO]
-TC_ENGINES = (B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM)
+ENGINES = [B.XNOR_ENGINE_POPC, B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM, B.XNOR_ENGINE_UMMA_SINGLE,
+           B.XNOR_ENGINE_UMMA_PAIR, B.XNOR_ENGINE_UMMA_PAIR_STREAM, B.XNOR_ENGINE_AUTO]
+TC_ENGINES = (B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM, B.XNOR_ENGINE_UMMA_SINGLE,
+              B.XNOR_ENGINE_UMMA_PAIR, B.XNOR_ENGINE_UMMA_PAIR_STREAM)
 
 
 def rng(seed):
