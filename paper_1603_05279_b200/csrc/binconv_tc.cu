@@ -1136,8 +1136,11 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
       const int nst = (P.nsteps + P.mps - 1) / P.mps;
       if (nst <= kMaxBarStages && fits(nst, 2, 1)) {
         P.resident = 1;
+        // three patches, then a second raw buffer per patch warp (a patch's rows are then on
+        // their way while the previous patch is expanded), then a fourth patch
         stages = nst; npb = 2;
-        while (npb < kMaxPatchBufs && fits(stages, npb + 1, 1)) ++npb;
+        if (fits(stages, 3, 1)) npb = 3;
+        if (npb == 3 && fits(stages, 3, 2) && fits(stages, 4, 2)) npb = 4;
       }
     }
   }
@@ -1151,8 +1154,8 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
     stages = 2; npb = 1;
     while (stages < 4 && fits(stages + 1, npb, 1)) ++stages;
     while (npb < 3 && fits(stages, npb + 1, 1)) ++npb;
-    while (stages < kMaxStages && fits(stages + 1, npb, 1)) ++stages;
-    while (npb < kMaxPatchBufs && fits(stages, npb + 1, 1)) ++npb;
+    while (stages < kMaxStages && fits(stages + 1, npb, 2)) ++stages;
+    while (npb < kMaxPatchBufs && fits(stages, npb + 1, 2)) ++npb;
   }
   P.nraw = fits(stages, npb, 2) ? 2 : 1;
   P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
@@ -1216,7 +1219,8 @@ Plan plan_variant(const ConvGeom &g, TcVariant v) {
   Plan single = make_plan(g, 0, false);
   if (single.ok && single.P.resident) return single;
   Plan pair = make_plan(g, 0, true);
-  if (pair.ok && (pair.P.resident || !single.ok)) return pair;
+  // neither resident: a pair pays when the slabs are wide (each CTA expands half the rows)
+  if (pair.ok && (pair.P.resident || !single.ok || pair.P.NT > 128)) return pair;
   return single;
 }
 
