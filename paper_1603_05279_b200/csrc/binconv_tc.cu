@@ -96,7 +96,7 @@ using namespace umma;
 
 constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
-constexpr int kWgtWarp0 = 5, kWgtWarps = 8, kWgtThreads = 32 * kWgtWarps;
+constexpr int kWgtWarp0 = 5, kWgtWarps = 8;
 constexpr int kPatWarp0 = 13, kPatWarps = 3;
 constexpr int kThreads = 32 * (kPatWarp0 + kPatWarps);     // 512: 16 warps, 128 registers each
 constexpr int kTileM = 128;          // stream positions per tile = tensor-memory lanes
@@ -108,6 +108,7 @@ constexpr int kMaxStages = 6;         // ring stages of the streaming schedule
 constexpr int kMaxBarStages = 32;    // stage barriers (the resident schedule has one stage per mps K-steps of a row)
 constexpr int kEpiSplitMax = 3;      // warps per lane quarter in the resident epilogue
 constexpr int kMaxPatchBufs = 4;
+constexpr int kMaxRaw = 6;            // raw buffers: up to 2 for each of up to 3 subgroups of patch warps
 constexpr int kMaxSteps = 800;       // K-steps (MMAs) per work item (< 1024: swap_mask)
 constexpr size_t kCtrlBytes = 1024;
 constexpr size_t kSmemMax = 232448 - 1024;
@@ -132,8 +133,11 @@ struct TcParams {
   uint32_t patch_bytes, stage_bytes;
   int rows_mod, grp_steps;     // weight-thread mapping (see weight producer)
   uint32_t off_ring, off_patch, off_raw;  // byte offsets in dynamic shared memory
-  int nraw;                    // raw buffers per patch warp (1 or 2)
-  uint32_t raw_bytes;          // size of one: the packed input rows a patch can touch
+  uint32_t raw_bytes;          // size of a raw buffer: the packed input rows a patch can touch
+  int nraw;                    // raw buffers per subgroup of patch warps (1 or 2)
+  int pat_group;               // warps that build patches: 3, or 7 with four of the weight warps
+  int pat_sub;                 // subgroups they form (each builds whole patches): 3 or 1
+  int wgt_warps;               // warps that expand weights: 8, or 4
   uint32_t idesc;
   uint32_t tail_mask;          // bits of real channels in the last word
   // Low word of the A-operand descriptor of every K-step (start address relative to the
@@ -286,7 +290,7 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m, int s) {
 }
 
 struct Smem {
-  uint32_t wfull, wempty, pfull, pempty, afull, aempty, rawfull;   // shared-space addresses of barrier arrays
+  uint32_t wfull, wempty, pfull, pempty, afull, aempty, rawfull, rawdone;   // shared-space addresses of barrier arrays
   uint32_t *tmem_slot;
   volatile int *abort_flag;
   uint32_t ring, patch, raw;                              // shared-space byte addresses
@@ -303,8 +307,9 @@ __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
   s.afull = s.pempty + 8u * kMaxPatchBufs;
   s.aempty = s.afull + 8u * kMaxAcc;
   s.rawfull = s.aempty + 8u * kMaxAcc;
+  s.rawdone = s.rawfull + 8u * kMaxRaw;
   s.tmem_slot = reinterpret_cast<uint32_t *>(
-      smem + 8 * (2 * kMaxBarStages + 2 * kMaxPatchBufs + 2 * kMaxAcc + 2 * kPatWarps));
+      smem + 8 * (2 * kMaxBarStages + 2 * kMaxPatchBufs + 2 * kMaxAcc + 2 * kMaxRaw));
   s.abort_flag = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
   s.ring = base + P.off_ring;
   s.patch = base + P.off_patch;
@@ -560,18 +565,21 @@ __device__ __forceinline__ bool weight_dispatch(const TcParams &P, const Smem &S
   return weight_role_swap<1>(P, S, nitems, slab0, wph0, wt, lane);
 }
 
-// ------------------------------------------------------------------ patch producers (3 warps)
-// Each warp builds whole patches on its own (warp p takes the CTA's patches p, p + active,
-// ...), so up to three patches are in the making; a patch's buffer is its index modulo the
-// number of buffers.  The packed pixels a patch touches are ONE contiguous range of x_packed:
-// input rows g0 .. g1 - 1 of the N*H rows (images follow one another in memory, the zero
-// rows and columns of the stream exist only in the patch).  Lane 0 brings that range into a
-// raw buffer of the warp with one bulk copy (an aligned superset inside the tensor; the
-// ragged last words of the tensor, if any, by plain loads), one patch ahead when the warp
-// has two raw buffers; the warp then expands from shared memory, a stream position per lane.
+// ------------------------------------------------------------------ patch producers
+// A group of P.pat_group warps (the three patch warps, in the resident schedule also four of
+// the weight warps) builds the CTA's patches one after the other, all warps on the same
+// patch: units of (32 stream positions, phase plane, up to 4 channel words) are dealt round
+// robin.  The packed pixels a patch touches are ONE contiguous range of x_packed: input rows
+// g0 .. g1 - 1 of the N*H rows (images follow one another in memory, the zero rows and
+// columns of the stream exist only in the patch).  Every patch buffer has a raw buffer; the
+// group's first warp brings a patch's range into it with one bulk copy (an aligned superset
+// inside the tensor; the ragged last words of the tensor, if any, by plain loads) as soon as
+// the group is done with the buffer's previous patch, so the rows of the next patches are on
+// their way while one is expanded.  Padding and the channel tail become the value 0 through
+// masks folded into the sign mask and the magnitude constants.
 // Streaming: one patch per tile of the CTA's range.  Resident (kRes): one patch per item.
 template <bool kRes>
-__device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long long i1, int pt,
+__device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long long i1, int pw,
                            int lane) {
   const int tile0 = kRes ? 0 : (int)(i0 / P.nslabs);
   const uint32_t npatches = kRes ? (uint32_t)(i1 - i0)
@@ -580,11 +588,6 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
   const int s = P.stride, phases = s * s;
   const uint32_t plane_bytes = (uint32_t)P.ppix * 16u;
   const bool vec = (P.Cw & 3) == 0;
-  const int pw = pt >> 5;                       // patch warp 0..2
-  // A barrier's parity tells apart only two consecutive uses of a buffer, so no warp may run
-  // more than one use ahead of the consumer: at most npb warps take part.
-  const int active = min(kPatWarps, P.npb);
-  if (pw >= active) return;
   // nibble masks of the channel tail, one per expanded register
   uint32_t tm[4];
 #pragma unroll
@@ -592,15 +595,16 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
   const bool tail = P.tail_mask != 0xFFFFFFFFu;
   const uint32_t row_bytes = (uint32_t)P.W * (uint32_t)P.Cw * 4u;
   const size_t tensor_bytes = (size_t)P.N * P.H * row_bytes;
-  const uint32_t raw0 = S.raw + (uint32_t)(pw * P.nraw) * P.raw_bytes;
-  const uint32_t rbar0 = S.rawfull + 8u * (uint32_t)(pw * 2);
+  // pairs: work tile t is stream tiles 2t (rank 0) and 2t + 1 (rank 1)
+  const uint32_t tmul = P.pair ? 2u : 1u;
+  const int ngrp = (P.Cw + 3) >> 2;                       // groups of 4 channel words
+  const int npass = (P.ppix + 31) >> 5;
+  const int nunits = npass * phases * ngrp;
 
   auto tile_of = [&](uint32_t seq) {
     return kRes ? (int)((tile_r0 + seq) % (uint32_t)P.ntiles) : tile0 + (int)seq;
   };
   // input rows [g0, g1) (of the N*H rows of the tensor) that the patch of a tile reads
-  // pairs: work tile t is stream tiles 2t (rank 0) and 2t + 1 (rank 1)
-  const uint32_t tmul = P.pair ? 2u : 1u;
   auto row_range = [&](int tile, int &g0, int &g1) {
     const uint32_t m0 = ((uint32_t)tile * tmul + S.rank) * kTileM;
     const uint32_t mlast = min(m0 + (uint32_t)P.ppix - 1u, (uint32_t)P.L - 1u);
@@ -614,12 +618,12 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     g0 = (int)n0 * P.H + t0;
     g1 = (int)n1 * P.H + t1;
   };
-  // lane 0: starts the copy of a patch's rows into raw buffer rb
-  auto start_copy = [&](uint32_t seq, int rb) {
+  // a subgroup's first warp, lane 0: starts the copy of a patch's rows into raw buffer rb
+  auto start_copy = [&](uint32_t seq, uint32_t rb) {
     int g0, g1;
     row_range(tile_of(seq), g0, g1);
-    const uint32_t bar = rbar0 + 8u * (uint32_t)rb;
-    const uint32_t dst = raw0 + (uint32_t)rb * P.raw_bytes;
+    const uint32_t bar = S.rawfull + 8u * rb;
+    const uint32_t dst = S.raw + rb * P.raw_bytes;
     if (g1 <= g0) { mbar_arrive(bar); return; }          // nothing but padding
     const size_t b0 = (size_t)g0 * row_bytes, b1 = (size_t)g1 * row_bytes;
     const size_t a0 = b0 & ~(size_t)15;
@@ -635,106 +639,110 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     }
   };
 
+  // The group works as `nsub` subgroups of equal size; subgroup sg builds patches sg,
+  // sg + nsub, ... (nsub <= npb: a barrier's parity tells apart only two consecutive uses of
+  // a buffer, so no subgroup may run more than one use ahead of the consumer).
+  const uint32_t nsub = (uint32_t)P.pat_sub, gsize = (uint32_t)P.pat_group / nsub;
+  const uint32_t sg = (uint32_t)pw % nsub, mi = (uint32_t)pw / nsub;
+  // The subgroup's k-th patch (patch sg + k nsub of the CTA) expands from the subgroup's raw
+  // buffer k % nraw; its rows are fetched as soon as the subgroup is done with patch k - nraw.
+  const uint32_t nraw = (uint32_t)P.nraw, rb0 = sg * nraw;
   bool ok = true;
-  bool pend[2] = {false, false};          // a copy into the raw buffer has not been consumed
-  uint32_t rph[2] = {0u, 0u};             // parity of the raw buffer's next completion
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    const uint32_t seq = (uint32_t)(pw + r * active);
-    if (r < P.nraw && seq < npatches) {
-      if (lane == 0) start_copy(seq, r);
-      pend[r] = true;
-    }
+  uint32_t kc = 0;                           // patches of the subgroup whose copy has been started
+  if (mi == 0) {
+    for (; kc < nraw && sg + kc * nsub < npatches; ++kc)
+      if (lane == 0) start_copy(sg + kc * nsub, rb0 + kc);
   }
-  int rb = 0;
-  TR_DECL(pt < 32);
+  TR_DECL(pw == 0);
   TR_T0;
+  uint32_t k = 0;
 #pragma unroll 1
-  for (uint32_t seq = (uint32_t)pw; seq < npatches && ok; seq += (uint32_t)active) {   // in order
+  for (uint32_t seq = sg; seq < npatches && ok; seq += nsub, ++k) {
     const int tile = tile_of(seq);
-    const int pb = (int)(seq % (uint32_t)P.npb);
-    const uint32_t pph = ((seq / (uint32_t)P.npb) & 1u) ^ 1u;
+    const uint32_t pb = seq % (uint32_t)P.npb;
+    const uint32_t use = seq / (uint32_t)P.npb;
+    const uint32_t rb = rb0 + k % nraw, ruse = k / nraw;
+    if (mi == 0 && k >= 1u && sg + kc * nsub < npatches) {
+      // kc = k - 1 + nraw: the raw buffer of patch k - 1 is free once every warp of the
+      // subgroup has expanded that patch
+      const uint32_t crb = rb0 + kc % nraw;
+      ok = mbar_wait_relaxed(S.rawdone + 8u * crb, (kc / nraw - 1u) & 1u, S.abort_flag,
+                             &g_status_tc, XNOR_SLEEP_PAT);
+      if (!ok) break;
+      fence_proxy_async();
+      if (lane == 0) start_copy(sg + kc * nsub, crb);
+      ++kc;
+    }
     int g0, g1;
     row_range(tile, g0, g1);
-    const uint32_t rbar = rbar0 + 8u * (uint32_t)rb;
-    ok = mbar_wait_relaxed(rbar, rb ? rph[1] : rph[0], S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
+    ok = mbar_wait_relaxed(S.rawfull + 8u * rb, ruse & 1u, S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
     if (!ok) break;
-    if (rb) { pend[1] = false; rph[1] ^= 1u; } else { pend[0] = false; rph[0] ^= 1u; }
-    ok = mbar_wait_relaxed(S.pempty + 8u * pb, pph, S.abort_flag, &g_status_tc, XNOR_SLEEP_PAT);
+    ok = mbar_wait_relaxed(S.pempty + 8u * pb, (use & 1u) ^ 1u, S.abort_flag, &g_status_tc,
+                           XNOR_SLEEP_PAT);
     TR_ADD(0);
     if (!ok) break;
-    const uint32_t patch = S.patch + (uint32_t)pb * P.patch_bytes;
+    const uint32_t patch = S.patch + pb * P.patch_bytes;
     const uint32_t m0 = ((uint32_t)tile * tmul + S.rank) * kTileM;
-    const uint32_t raw = raw0 + (uint32_t)rb * P.raw_bytes +
+    const uint32_t raw = S.raw + rb * P.raw_bytes +
                          (uint32_t)(((size_t)g0 * row_bytes) & 15u);   // where row g0 starts
-    // Two stream positions per lane and pass, their loads issued together.  Padding and the
-    // channel tail become the value 0 through the masks: keep (all or nothing) is folded into
-    // the sign mask and the magnitude constants, so a word costs a shift and one logic
-    // operation per register.
+    // two units per pass: their loads are issued together, then both are expanded
 #pragma unroll 1
-    for (int q0 = lane; q0 < P.ppix; q0 += 64) {
-      bool in[2];
-      int rrow[2], rcol[2], grow[2];
+    for (int u0 = (int)mi; u0 < nunits; u0 += 2 * (int)gsize) {
+      uint32_t src[2], dst[2], sm[2], mc[2][3], wv[2][4];
+      int w0[2];
+      bool on[2], real[2];
 #pragma unroll
       for (int b = 0; b < 2; ++b) {
-        const uint32_t sq = m0 + (uint32_t)(q0 + 32 * b);
+        const int u = u0 + b * (int)gsize;
+        const int pass = u / (phases * ngrp);
+        const int rem = u - pass * (phases * ngrp);
+        const int phase = rem / ngrp;
+        w0[b] = (rem - phase * ngrp) * 4;
+        const int q = pass * 32 + lane;
+        on[b] = u < nunits && q < P.ppix;
+        const uint32_t sq = m0 + (uint32_t)q;
         const uint32_t r = fast_div(sq, P.div_wq_m, P.div_wq_s);
         const int c = (int)(sq - r * (uint32_t)P.Wq);
         const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
         const int ry = (int)(r - n * (uint32_t)P.Hq);
-        in[b] = q0 + 32 * b < P.ppix && sq < (uint32_t)P.L && ry >= P.leadY && c >= P.leadX;
-        rrow[b] = (ry - P.leadY) * s;
-        rcol[b] = (c - P.leadX) * s;
-        grow[b] = (int)n * P.H + rrow[b] - g0;     // row inside the raw range (+ py)
-      }
-      const bool second = q0 + 32 < P.ppix;          // the lane has a second position
-#pragma unroll 1
-      for (int phase = 0; phase < phases; ++phase) {
         const int py = phase / s, px = phase - py * s;
-        uint32_t src[2], sm[2], mc[2][3];
-        bool real[2];
+        const int rrow = (ry - P.leadY) * s + py, rcol = (c - P.leadX) * s + px;
+        real[b] = on[b] && sq < (uint32_t)P.L && ry >= P.leadY && c >= P.leadX && rrow < P.H &&
+                  rcol < P.W;
+        const uint32_t keep = real[b] ? 0xFFFFFFFFu : 0u;        // padding expands to 0
+        sm[b] = 0x88888888u & keep;
+        mc[b][0] = 0xCCCCCCCCu & keep; mc[b][1] = 0xAAAAAAAAu & keep; mc[b][2] = 0x99999999u & keep;
+        src[b] = raw + (uint32_t)((((int)n * P.H + rrow - g0) * P.W + rcol) * P.Cw + w0[b]) * 4u;
+        dst[b] = patch + (uint32_t)(phase * P.Cw + w0[b]) * plane_bytes + (uint32_t)q * 16u;
+      }
 #pragma unroll
-        for (int b = 0; b < 2; ++b) {
-          real[b] = in[b] && rrow[b] + py < P.H && rcol[b] + px < P.W;
-          const uint32_t keep = real[b] ? 0xFFFFFFFFu : 0u;
-          src[b] = raw + (uint32_t)(((grow[b] + py) * P.W + rcol[b] + px) * P.Cw) * 4u;
-          sm[b] = 0x88888888u & keep;
-          mc[b][0] = 0xCCCCCCCCu & keep; mc[b][1] = 0xAAAAAAAAu & keep; mc[b][2] = 0x99999999u & keep;
-        }
-        const uint32_t dst = patch + (uint32_t)(phase * P.Cw) * plane_bytes + (uint32_t)q0 * 16u;
-#pragma unroll 1
-        for (int w0 = 0; w0 < P.Cw; w0 += 4) {
-          uint32_t wv[2][4];
+      for (int b = 0; b < 2; ++b) {
+        wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
+        if (real[b]) {
+          if (vec) {
+            lds128(src[b], wv[b]);
+          } else {
 #pragma unroll
-          for (int b = 0; b < 2; ++b) {
-            wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
-            if (real[b]) {
-              if (vec) {
-                lds128(src[b] + (uint32_t)w0 * 4u, wv[b]);
-              } else {
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  if (w0 + i < P.Cw) wv[b][i] = lds32(src[b] + (uint32_t)(w0 + i) * 4u);
-              }
-            }
+            for (int i = 0; i < 4; ++i)
+              if (w0[b] + i < P.Cw) wv[b][i] = lds32(src[b] + (uint32_t)i * 4u);
           }
+        }
+      }
 #pragma unroll
-          for (int b = 0; b < 2; ++b) {
-            if (b == 0 || second) {
+      for (int b = 0; b < 2; ++b) {
+        if (on[b]) {
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                if (w0 + i < P.Cw) {
-                  const uint32_t w = wv[b][i];
-                  uint32_t v0 = ((w << 3) & sm[b]) ^ mc[b][0];
-                  uint32_t v1 = ((w << 2) & sm[b]) ^ mc[b][1];
-                  uint32_t v2 = ((w << 1) & sm[b]) ^ mc[b][2];
-                  uint32_t v3 = (w & sm[b]) ^ mc[b][2];
-                  if (tail && w0 + i == P.Cw - 1) {       // channels beyond C_in are 0
-                    v0 &= tm[0]; v1 &= tm[1]; v2 &= tm[2]; v3 &= tm[3];
-                  }
-                  sts128(dst + (uint32_t)(w0 + i) * plane_bytes + (uint32_t)(b * 32 * 16), v0, v1, v2, v3);
-                }
+          for (int i = 0; i < 4; ++i) {
+            if (w0[b] + i < P.Cw) {
+              const uint32_t w = wv[b][i];
+              uint32_t v0 = ((w << 3) & sm[b]) ^ mc[b][0];
+              uint32_t v1 = ((w << 2) & sm[b]) ^ mc[b][1];
+              uint32_t v2 = ((w << 1) & sm[b]) ^ mc[b][2];
+              uint32_t v3 = (w & sm[b]) ^ mc[b][2];
+              if (tail && w0[b] + i == P.Cw - 1) {       // channels beyond C_in are 0
+                v0 &= tm[0]; v1 &= tm[1]; v2 &= tm[2]; v3 &= tm[3];
               }
+              sts128(dst[b] + (uint32_t)i * plane_bytes, v0, v1, v2, v3);
             }
           }
         }
@@ -743,22 +751,17 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     TR_ADD(1);
     fence_proxy_async();
     __syncwarp();
-    const uint32_t next = seq + (uint32_t)(P.nraw * active);   // reuses this raw buffer
     if (lane == 0) {
+      mbar_arrive(S.rawdone + 8u * rb);
       if (P.pair) mbar_arrive_cluster(S.pfull + 8u * pb, 0u); else mbar_arrive(S.pfull + 8u * pb);
-      if (next < npatches) start_copy(next, rb);
     }
-    if (next < npatches) { if (rb) pend[1] = true; else pend[0] = true; }
-    if (++rb == P.nraw) rb = 0;
   }
-  if (!ok) {
-    // gave up: a copy still in flight must land before the CTA's shared memory is released
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      if (pend[r]) {
-        const uint32_t bar = rbar0 + 8u * (uint32_t)r;
-        for (int i = 0; i < (1 << 20) && !mbar_try(bar, rph[r]); ++i) {}
-      }
+  if (!ok && mi == 0) {
+    // gave up: the copies this warp started last (one per buffer at most can still be in
+    // flight) must land before the CTA's shared memory is released
+    for (uint32_t back = 1; back <= nraw && back <= kc; ++back) {
+      const uint32_t c = kc - back;
+      for (int i = 0; i < (1 << 20) && !mbar_try(S.rawfull + 8u * (rb0 + c % nraw), (c / nraw) & 1u); ++i) {}
     }
   }
   TR_FLUSH(16);
@@ -939,14 +942,17 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     // waits for them); the MMA warp's commits reach the consumer barriers of both CTAs.
     constexpr uint32_t kCtas = kPair ? 2u : 1u;
     for (int i = 0; i < kMaxBarStages; ++i) {
-      mbar_init(S.wfull + 8u * i, kWgtWarps * kCtas);
+      mbar_init(S.wfull + 8u * i, (uint32_t)P.wgt_warps * kCtas);
       mbar_init(S.wempty + 8u * i, 1);
     }
     for (int i = 0; i < kMaxPatchBufs; ++i) {
-      mbar_init(S.pfull + 8u * i, kCtas);
+      mbar_init(S.pfull + 8u * i, (uint32_t)(P.pat_group / P.pat_sub) * kCtas);
       mbar_init(S.pempty + 8u * i, 1);
     }
-    for (int i = 0; i < 2 * kPatWarps; ++i) mbar_init(S.rawfull + 8u * i, 1);
+    for (int i = 0; i < kMaxRaw; ++i) {
+      mbar_init(S.rawfull + 8u * i, 1);
+      mbar_init(S.rawdone + 8u * i, (uint32_t)(P.pat_group / P.pat_sub));
+    }
     for (int i = 0; i < kMaxAcc; ++i) {
       mbar_init(S.afull + 8u * i, 1);
       mbar_init(S.aempty + 8u * i, (kRes ? kEpiWarps * P.epi_split : kEpiWarps) * kCtas);
@@ -1002,7 +1008,9 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   if (i0 < i1) {
     const int wt = tid - 32 * kWgtWarp0;
     if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base); }
-    else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, tid - 32 * kPatWarp0, lane);
+    else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, warp - kPatWarp0, lane);
+    else if (kRes && P.pat_group > kPatWarps && warp >= kWgtWarp0 + 4)
+      patch_role<kRes>(P, S, i0, i1, kPatWarps + warp - (kWgtWarp0 + 4), lane);   // helpers
     else if (!kRes) {
       if (warp < kEpiWarps) epilogue_role<false>(P, S, i0, i1, 0, tmem_base, warp, 0, lane);
       else weight_dispatch(P, S, i1 - i0, (int)(i0 % P.nslabs), 1u, wt, lane);
@@ -1060,9 +1068,10 @@ void plan_stage(TcParams &P) {
   int ntp = 16;
   while (ntp < P.NTh) ntp *= 2;                         // 16 .. 256
   P.rows_mod = ntp;
-  const int groups = kWgtThreads / P.rows_mod;          // 1 .. 16
+  const int groups = std::max(1, 32 * P.wgt_warps / P.rows_mod);   // 1 .. 16
   P.mps = std::max(2, std::min(8, 1024 / ntp));
   while (P.mps > 4 && P.nsteps < 3 * P.mps) P.mps /= 2;   // short items: smaller stages start sooner
+  if (P.mps > 4 * groups) P.mps = 4 * groups;           // a thread expands at most 4 K-steps of a stage
   P.grp_steps = std::max(1, P.mps / groups);            // 4, 4, 2, 1, 1
   P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NTh * 32u;
 }
@@ -1113,11 +1122,14 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
   // shared memory: control, weight stages, patch buffers
   P.off_ring = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
   const size_t avail = kSmemMax - P.off_ring;
-  // st weight stages, pb patch buffers, nraw raw buffers for each of the patch warps at work
+  // st weight stages, pb patch buffers, nraw raw buffers for each subgroup of patch warps
+  auto subgroups = [&](int pb) { return (P.pat_group == kPatWarps && pb >= kPatWarps) ? kPatWarps : 1; };
   auto fits = [&](int st, int pb, int nraw) {
     return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes +
-           (size_t)(std::min(kPatWarps, pb) * nraw) * P.raw_bytes <= avail;
+           (size_t)(subgroups(pb) * nraw) * P.raw_bytes <= avail;
   };
+  P.wgt_warps = kWgtWarps;
+  P.pat_group = kPatWarps;
   // as few slabs as fit two accumulators in the tensor-memory columns
   const int max_nt = pair ? 224 : 240;
   const int min_slabs = (g.Co + max_nt - 1) / max_nt;
@@ -1132,15 +1144,19 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
       P.NT = slab_width(g.Co, ns, pair);
       P.NTh = pair ? P.NT / 2 : P.NT;
       if (P.NT < 128 && ns > 1) break;
+      // The slab is expanded once per visit, so four weight warps are enough when a thread
+      // per row fits them; with many channel words per pixel (measured: from 12 on) the other
+      // four then build patches instead of draining accumulators.
+      const bool helpers = g.Cw >= 12 && P.NTh <= 128;
+      P.wgt_warps = helpers ? kWgtWarps / 2 : kWgtWarps;
+      P.pat_group = helpers ? kPatWarps + kWgtWarps / 2 : kPatWarps;
       plan_stage(P);
       const int nst = (P.nsteps + P.mps - 1) / P.mps;
       if (nst <= kMaxBarStages && fits(nst, 2, 1)) {
         P.resident = 1;
-        // three patches, then a second raw buffer per patch warp (a patch's rows are then on
-        // their way while the previous patch is expanded), then a fourth patch
         stages = nst; npb = 2;
         if (fits(stages, 3, 1)) npb = 3;
-        if (npb == 3 && fits(stages, 3, 2) && fits(stages, 4, 2)) npb = 4;
+        if (npb == 3 && fits(stages, 4, 2)) npb = 4;     // a second raw buffer comes first
       }
     }
   }
@@ -1148,6 +1164,8 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
     P.nslabs = min_slabs;
     P.NT = slab_width(g.Co, P.nslabs, pair);
     P.NTh = pair ? P.NT / 2 : P.NT;
+    P.wgt_warps = kWgtWarps;
+    P.pat_group = kPatWarps;
     plan_stage(P);
     if (!fits(2, 1, 1)) return pl;
     // at least 2 stages and 1 patch; then patches up to 3, stages up to 6, one more patch
@@ -1159,11 +1177,15 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
   }
   P.nraw = fits(stages, npb, 2) ? 2 : 1;
   P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
-  P.epi_split = std::min(kEpiSplitMax, P.NT / 16);
+  // worker warps per quarter of the lanes in the resident schedule: the four epilogue warps
+  // and the weight warps (all eight, or the four that are not patch helpers)
+  P.epi_split = std::min(P.pat_group > kPatWarps ? 2 : kEpiSplitMax, P.NT / 16);
   P.stages = stages; P.npb = npb;
+  // small patches: every patch warp builds whole patches on its own, three at a time
+  P.pat_sub = subgroups(npb);
   P.off_patch = P.off_ring + (uint32_t)stages * P.stage_bytes;
   P.off_raw = P.off_patch + (uint32_t)npb * P.patch_bytes;
-  pl.smem = (size_t)P.off_raw + (size_t)(std::min(kPatWarps, npb) * P.nraw) * P.raw_bytes;
+  pl.smem = (size_t)P.off_raw + (size_t)(P.pat_sub * P.nraw) * P.raw_bytes;
   // block-scaled instruction descriptor: e2m1 x e2m1, ue8m0 scales, M = 128 (256 for a
   // pair), N = NT
   P.idesc = (1u << 7) | (1u << 10) | ((uint32_t)(P.NT >> 3) << 17) | (1u << 23) |
