@@ -213,6 +213,47 @@ def test_alexnet_layers_at_full_batch(oracle, li):
     assert bool(torch.isfinite(out).all())
 
 
+@pytest.mark.parametrize("li,engine", [(0, B.XNOR_ENGINE_UMMA_STREAM), (0, B.XNOR_ENGINE_UMMA_PAIR),
+                                       (1, B.XNOR_ENGINE_UMMA_PAIR_STREAM), (2, B.XNOR_ENGINE_UMMA_SINGLE),
+                                       (2, B.XNOR_ENGINE_UMMA_PAIR), (3, B.XNOR_ENGINE_UMMA_PAIR_STREAM)])
+def test_alexnet_layers_at_full_batch_pinned_variants(oracle, li, engine):
+    """Every schedule of the tensor-core engine at the benchmark's size: CTAs whose item range
+    crosses a slab boundary (a second fill of the resident slab), many rounds of every barrier,
+    pairs with an odd number of stream tiles."""
+    s = wl.ALEXNET[li]
+    x, w, out, acc, K = _run_layer_full(s, wl.layer_seed("alexnet", li), engine)
+    _check_sampled_images(oracle, s, x, w, out, acc, [0, s.N // 2, s.N - 1])
+
+
+def test_engines_agree_bit_for_bit_on_odd_sizes():
+    """All engines compute the same integers and apply the same two fp32 roundings, so their
+    outputs are identical; shapes chosen for ragged tiles (odd pixel and filter counts, a
+    channel tail, stride 2, one stream tile for a pair)."""
+    for (N, C, H, W, Co, k, st, pad) in [(3, 70, 9, 7, 50, 3, 1, 1), (2, 40, 11, 11, 130, 5, 2, 2),
+                                         (1, 33, 6, 5, 17, 3, 1, 0), (5, 200, 14, 14, 272, 3, 1, 1)]:
+        g = rng(N * 1000 + C)
+        s = wl.ConvShape("t", N, C, H, W, Co, k, st, pad, 1.0)
+        x = g.standard_normal((N, C, H, W)).astype(np.float32)
+        w = g.standard_normal((Co, C, k, k)).astype(np.float32)
+        d = X.desc_of(s)
+        wp, alpha = X.alloc_weights(Co, C, k, k)
+        xp, A, K = X.alloc_binactiv(d)
+        X.xnor_binarize_weights(dev(w), wp, alpha)
+        X.xnor_binactiv(dev(x), None, None, d, xp, A, K)
+        outs = []
+        for engine in ENGINES:
+            out = X.alloc_out(d)
+            X.xnor_set_engine(engine)
+            try:
+                X.xnor_conv2d_forward(xp, wp, alpha, K, None, d, out, None)
+            finally:
+                X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
+            X.xnor_check_device()
+            outs.append(out)
+        for out in outs[1:]:
+            assert torch.equal(out, outs[0])
+
+
 @pytest.mark.parametrize("li", range(len(wl.RESNET18)))
 def test_resnet_layers_at_full_batch(oracle, li):
     s = wl.RESNET18[li]

@@ -45,10 +45,14 @@ def test_small_host_functions():
 def test_engine_switch():
     X.xnor_set_engine(B.XNOR_ENGINE_POPC)
     assert X.xnor_get_engine() == B.XNOR_ENGINE_POPC
-    X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
+    for e in (B.XNOR_ENGINE_UMMA, B.XNOR_ENGINE_UMMA_STREAM, B.XNOR_ENGINE_UMMA_SINGLE,
+              B.XNOR_ENGINE_UMMA_PAIR, B.XNOR_ENGINE_UMMA_PAIR_STREAM, B.XNOR_ENGINE_AUTO):
+        X.xnor_set_engine(e)
+        assert X.xnor_get_engine() == e
+    for bad in (-1, 7, 17):
+        with pytest.raises(X.XnorError):
+            X.xnor_set_engine(bad)
     assert X.xnor_get_engine() == B.XNOR_ENGINE_AUTO
-    with pytest.raises(X.XnorError):
-        X.xnor_set_engine(17)
 
 
 def test_arguments_are_rejected_before_any_launch():
