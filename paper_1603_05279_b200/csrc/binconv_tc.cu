@@ -62,13 +62,16 @@ namespace xnor {
 
 __device__ int g_status_tc = 0;
 #ifdef XNOR_TRACE
+#ifndef XNOR_TRACE_BLOCK
+#define XNOR_TRACE_BLOCK 1
+#endif
 // cycle totals of one warp per role of one CTA: [0..7] mma, [8..15] weights, [16..23] patch,
 // [24..31] epilogue
 __device__ long long g_tc_trace[64];
 // per CTA: clock at the start of the roles, at their end, SM id
 __device__ long long g_tc_cta[3 * 160];
 #define TR_DECL(first) long long tr_t = 0, tr_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}; \
-  const bool tr_on = blockIdx.x == 1 && (threadIdx.x & 31) == 0 && (first)
+  const bool tr_on = blockIdx.x == XNOR_TRACE_BLOCK && (threadIdx.x & 31) == 0 && (first)
 #define TR_T0 do { if (tr_on) tr_t = clock64(); } while (0)
 #define TR_ADD(i) do { if (tr_on) { const long long n_ = clock64(); tr_a[(i) & 7] += n_ - tr_t; tr_t = n_; } } while (0)
 #define TR_FLUSH(base) do { if (tr_on) { for (int q_ = 0; q_ < 8; ++q_) g_tc_trace[(base) + q_] += tr_a[q_]; } } while (0)
