@@ -290,11 +290,29 @@ class LayersJob:
             stream.wait_event(join)
 
     def e2e_step(self, stream):
+        """Host buffers in, host buffers out: the inputs of every layer go up on a copy stream,
+        a layer's kernels start when its inputs have landed, its output goes down on a third
+        stream while the next layer computes (the two directions of the link run together).
+        The step ends when the last output is on the host."""
+        torch = self.torch
+        if not hasattr(self, "_h2d"):
+            self._h2d, self._d2h = torch.cuda.Stream(), torch.cuda.Stream()
+            self._ev_in = [torch.cuda.Event() for _ in self.layers]
+            self._ev_out = [torch.cuda.Event() for _ in self.layers]
+        self._h2d.wait_stream(stream)          # the previous step is done with the device buffers
+        with torch.cuda.stream(self._h2d):
+            for li, L in enumerate(self.layers):
+                L.x.copy_(self.host_x[li], non_blocking=True)
+                L.w.copy_(self.host_w[li], non_blocking=True)
+                self._ev_in[li].record(self._h2d)
         for li, L in enumerate(self.layers):
-            L.x.copy_(self.host_x[li], non_blocking=True)
-            L.w.copy_(self.host_w[li], non_blocking=True)
+            stream.wait_event(self._ev_in[li])
             L.forward(stream)
-            self.host_out[li].copy_(L.out, non_blocking=True)
+            self._ev_out[li].record(stream)
+            self._d2h.wait_event(self._ev_out[li])
+            with torch.cuda.stream(self._d2h):
+                self.host_out[li].copy_(L.out, non_blocking=True)
+        stream.wait_stream(self._d2h)
 
     def parts(self, stream):
         for li, L in enumerate(self.layers):
