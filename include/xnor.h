@@ -231,6 +231,16 @@ xnor_engine xnor_get_engine(void);
  */
 xnor_status xnor_check_device(void *cuda_stream);
 
+/*
+ * Exercises that error path without touching any data: launches on
+ * `cuda_stream` one warp that waits, with a limit of about a millisecond, on
+ * a barrier that nothing signals.  The wait gives up by itself, so the next
+ * xnor_check_device returns XNOR_ERR_TIMEOUT once and the device stays
+ * usable.  No counterpart in the paper; meant for tests of the bounded waits.
+ * Returns XNOR_OK or XNOR_ERR_CUDA (launch failure).
+ */
+xnor_status xnor_selftest_wait_timeout(void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,7 @@ XNOR_ENGINE_UMMA_PAIR_STREAM = 6
 EXPORTS = [
     "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
     "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
-    "xnor_set_engine", "xnor_get_engine", "xnor_check_device",
+    "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
 ]
 
 
@@ -81,6 +81,8 @@ def load():
     lib.xnor_get_engine.restype = ci
     lib.xnor_check_device.restype = ci
     lib.xnor_check_device.argtypes = [vp]
+    lib.xnor_selftest_wait_timeout.restype = ci
+    lib.xnor_selftest_wait_timeout.argtypes = [vp]
     _lib = lib
     return lib
 
@@ -144,6 +146,11 @@ def xnor_get_engine():
 def xnor_check_device(stream=None):
     """Synchronises the stream and raises XnorError if a device-side wait expired."""
     _check(load().xnor_check_device(_stream(stream)), "xnor_check_device")
+
+
+def xnor_selftest_wait_timeout(stream=None):
+    """Launches the one-warp kernel whose bounded wait expires (see the header)."""
+    _check(load().xnor_selftest_wait_timeout(_stream(stream)), "xnor_selftest_wait_timeout")
 
 
 def xnor_binarize_weights(w, w_packed, alpha, stream=None):

@@ -119,6 +119,10 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
                                              acc_out, (cudaStream_t)cuda_stream));
 }
 
+xnor_status xnor_selftest_wait_timeout(void *cuda_stream) {
+  return from_cuda(xnor::launch_wait_timeout_selftest((cudaStream_t)cuda_stream));
+}
+
 xnor_status xnor_check_device(void *cuda_stream) {
   int st = 0;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess ||

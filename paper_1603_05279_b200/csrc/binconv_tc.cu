@@ -1321,6 +1321,29 @@ extern "C" int xnor_debug_trace_tc(long long *host64, int clear) {
 }
 #endif
 
+namespace {
+
+// One warp waits, with a limit of about a millisecond, on a barrier that nothing signals: the
+// wait must give up, raise the CTA's abort flag and record XNOR_ERR_TIMEOUT.
+__global__ void wait_timeout_selftest_kernel() {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ volatile int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  (void)mbar_wait_slow(smem_u32(&bar), 0u, &abort_flag, &g_status_tc, 1ll << 21);
+}
+
+}  // namespace
+
+cudaError_t launch_wait_timeout_selftest(cudaStream_t st) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, st>>>();
+  return cudaGetLastError();
+}
+
 cudaError_t read_status_tc(int *status) {
   cudaError_t e = cudaMemcpyFromSymbol(status, g_status_tc, sizeof(int));
   if (e == cudaSuccess && *status != 0) {

@@ -51,6 +51,8 @@ bool umma_tc_supported(const ConvGeom &g, TcVariant v);
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
                               float *out, int32_t *acc_out, TcVariant v, cudaStream_t st);
+// A one-warp kernel whose bounded wait expires (nothing signals its barrier).
+cudaError_t launch_wait_timeout_selftest(cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.
 cudaError_t read_status_tc(int *status);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,

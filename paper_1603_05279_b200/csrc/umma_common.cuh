@@ -85,14 +85,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // recorded in *status_word and the CTA-wide abort flag is raised) or when
 // another thread of the CTA already gave up.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity,
-                                            volatile int *abort_flag, int *status_word) {
+                                            volatile int *abort_flag, int *status_word,
+                                            long long limit = kWaitCycles) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 64; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicExch(status_word, (int)XNOR_ERR_TIMEOUT);
       return false;
