@@ -254,6 +254,62 @@ def test_engines_agree_bit_for_bit_on_odd_sizes():
             assert torch.equal(out, outs[0])
 
 
+def _random_shapes(count, seed):
+    """Seeded shapes that walk the planner's corners: few or many channel words (the patch
+    builders' cooperative mode starts at 12), filter counts around the slab widths, one or many
+    pixel tiles, both strides, with and without padding."""
+    g = rng(seed)
+    shapes = []
+    while len(shapes) < count:
+        C = int(g.choice([1, 31, 64, 96, 200, 384, 400, 520]))
+        Co = int(g.choice([1, 16, 40, 129, 224, 256, 300]))
+        k = int(g.choice([1, 2, 3, 5]))
+        st = int(g.choice([1, 2]))
+        pad = int(g.integers(0, k))
+        H = int(g.integers(max(1, k - 2 * pad), 23))
+        W = int(g.integers(max(1, k - 2 * pad), 23))
+        N = int(g.choice([1, 2, 5, 19]))
+        if C * k * k > 6000 and N * H * W > 2000:
+            N = 1                                     # keep the popcount reference quick
+        shapes.append((N, C, H, W, Co, k, st, pad))
+    return shapes
+
+
+@pytest.mark.parametrize("shape", _random_shapes(24, 20240607))
+def test_tensor_core_variants_match_the_popcount_engine(shape):
+    """The CUDA-core engine shares no code with the tensor-core kernels beyond the packed
+    operands; integers and the two fp32 roundings are the same, so outputs must be identical."""
+    N, C, H, W, Co, k, st, pad = shape
+    g = rng(sum(shape))
+    x = g.standard_normal((N, C, H, W)).astype(np.float32)
+    w = g.standard_normal((Co, C, k, k)).astype(np.float32)
+    res = g.standard_normal((N, Co, (H + 2 * pad - k) // st + 1, (W + 2 * pad - k) // st + 1)).astype(np.float32)
+    d = B.xnor_conv_desc(N, C, H, W, Co, k, k, st, pad)
+    wp, alpha = X.alloc_weights(Co, C, k, k)
+    xp, A, K = X.alloc_binactiv(d)
+    X.xnor_binarize_weights(dev(w), wp, alpha)
+    X.xnor_binactiv(dev(x), None, None, d, xp, A, K)
+    r = dev(res)
+    ref = None
+    for engine in ENGINES:
+        out = X.alloc_out(d)
+        acc = X.alloc_out(d, torch.int32)
+        X.xnor_set_engine(engine)
+        try:
+            X.xnor_conv2d_forward(xp, wp, alpha, K, r, d, out, acc)
+        except X.XnorError as e:
+            assert engine in TC_ENGINES and e.status == B.XNOR_ERR_UNSUPPORTED, (shape, engine)
+            continue
+        finally:
+            X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
+        X.xnor_check_device()
+        if ref is None:
+            ref = (out, acc)
+        else:
+            assert torch.equal(acc, ref[1]), (shape, engine)
+            assert torch.equal(out, ref[0]), (shape, engine)
+
+
 @pytest.mark.parametrize("li", range(len(wl.RESNET18)))
 def test_resnet_layers_at_full_batch(oracle, li):
     s = wl.RESNET18[li]
