@@ -543,7 +543,20 @@ def run_ours(args):
     def ordered(d):
         return [round(d[k], 4) for k in sorted(d)]
 
+    # per layer: the two floors of BinConv (fp32 output write at the measured copy bandwidth;
+    # 1-bit MACs at the tensor peak in use) and which of them binds
+    def conv_bytes(sh):
+        cw = (sh.C_in + 31) // 32
+        ho, wo = wl.out_hw(sh)
+        return 4 * (sh.N * sh.H * sh.W * cw + sh.C_out * sh.k * sh.k * cw + sh.N * ho * wo * (1 + sh.C_out)
+                    + sh.C_out)
+    hbm_floor = [conv_bytes(sh) / (peaks["hbm_gbs"] * 1e9) * 1e6 for sh in job.shapes]
+    pipe_floor = [2 * m / (roofline["peak"] * 1e12) * 1e6 for m in job.conv_macs]
     breakdown = {
+        "conv_floor_us": {"hbm": [round(v, 1) for v in hbm_floor],
+                          "pipe": [round(v, 1) for v in pipe_floor],
+                          "binding": ["hbm" if h > t else roofline["bound"]
+                                      for h, t in zip(hbm_floor, pipe_floor)]},
         "per_layer_ms": {n: ordered(per[n]) for n in job.part_names},
         "conv_TMACs": [round(job.conv_macs[i] / (per["conv"][k] / 1e3) / 1e12, 2)
                        for i, k in enumerate(sorted(per["conv"]))],
