@@ -154,7 +154,10 @@ def test_constant_magnitude_inputs_give_the_dense_convolution(oracle):
 
 def test_shortcut_conv_parity(oracle):
     g = rng(9)
-    for (N, C, H, W, Co, s) in [(2, 64, 56, 56, 128, 2), (3, 70, 9, 7, 33, 2), (1, 16, 5, 5, 8, 1)]:
+    # the ResNet shape; odd sizes (channel and filter tails, pixel tiles that straddle images,
+    # H_out*W_out not a multiple of 4); a 7x7 output at batch 40 (several tiles over many images)
+    for (N, C, H, W, Co, s) in [(2, 64, 56, 56, 128, 2), (3, 70, 9, 7, 33, 2), (1, 16, 5, 5, 8, 1),
+                                (40, 256, 14, 14, 130, 2), (5, 36, 6, 6, 64, 1), (7, 3, 1, 1, 2, 1)]:
         x = g.standard_normal((N, C, H, W)).astype(np.float32)
         w = (0.05 * g.standard_normal((Co, C))).astype(np.float32)
         out = torch.empty((N, Co, (H - 1) // s + 1, (W - 1) // s + 1), device="cuda")
