@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     scale_output,
     xnor_block,
     shortcut_conv1x1,
+    maxpool2d,
     speedup_model,
     out_extent,
 )

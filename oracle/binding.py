@@ -159,5 +159,14 @@ def shortcut_conv1x1(x, w, stride):
     return out
 
 
+def maxpool2d(x, k, stride, pad=0, relu=False):
+    """Max pooling (optionally after ReLU) of an NCHW fp32 tensor; padding taps take no part."""
+    x = _f32(x)
+    N, C, H, W = x.shape
+    out = np.empty((N, C, out_extent(H, k, stride, pad), out_extent(W, k, stride, pad)), np.float32)
+    _load().oracle_maxpool2d(_p(x), *_i(N, C, H, W, k, stride, pad, 1 if relu else 0), _p(out))
+    return out
+
+
 def speedup_model(c, n_w):
     return float(_load().oracle_speedup_model(float(c), float(n_w)))

@@ -208,6 +208,36 @@ void oracle_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H
         }
 }
 
+/* The last layer of the block of Section 3.2 ("Training XNOR-Networks": the
+ * order is BatchNorm, BinActiv, BinConv, Pool, with an optional non-binary
+ * activation such as ReLU after the binary convolution): max pooling over
+ * k x k windows at the given stride, on the real-valued output of BinConv.
+ * Readings where the paper is silent: a tap outside the image does not take
+ * part in the maximum (at least one tap is always inside since pad < k);
+ * Ho = (H + 2 pad - k) / stride + 1, rounded down; relu != 0 applies
+ * max(v, 0) to every input value before the maximum. */
+void oracle_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride,
+                      int pad, int relu, float *out) {
+  const int Ho = out_extent(H, k, stride, pad), Wo = out_extent(W, k, stride, pad);
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int c = 0; c < C; ++c)
+      for (int oy = 0; oy < Ho; ++oy)
+        for (int ox = 0; ox < Wo; ++ox) {
+          int first = 1;
+          float m = 0.0f;
+          for (int ky = 0; ky < k; ++ky)
+            for (int kx = 0; kx < k; ++kx) {
+              const int iy = oy * stride + ky - pad, ix = ox * stride + kx - pad;
+              if (iy < 0 || iy >= H || ix < 0 || ix >= W) continue;
+              float v = x[(((size_t)n * C + c) * H + iy) * W + ix];
+              if (relu && v < 0.0f) v = 0.0f;
+              if (first || v > m) { m = v; first = 0; }
+            }
+          out[(((size_t)n * C + c) * Ho + oy) * Wo + ox] = m;
+        }
+}
+
 /* Section 4.1: with 64 binary operations per clock, the ratio of the cost of
  * a standard convolution (c*N_W*N_I operations) to the binary one
  * (c*N_W*N_I/64 + N_I) is S = 64 c N_W / (c N_W + 64). */

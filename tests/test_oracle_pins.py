@@ -304,6 +304,42 @@ def test_shortcut_conv_matches_library(oracle):
 
 
 # ---------------------------------------------------------------- Section 4.1
+# ---------------------------------------------------------------- Pool (Section 3.2, block B-A-C-P)
+@pytest.mark.parametrize("case", [(2, 3, 9, 7, 3, 2, 0), (1, 4, 8, 11, 3, 2, 1), (2, 2, 6, 6, 2, 2, 0),
+                                  (1, 1, 5, 4, 5, 1, 2), (3, 2, 7, 7, 3, 1, 1)])
+def test_maxpool_matches_library_routine(oracle, case):
+    """torch's max_pool2d (fp64, floor mode, -inf padding) is an independent statement of the
+    same definition; maxima of fp32 values are exact, so the match is bit for bit."""
+    N, C, H, W, k, s, p = case
+    x = rng(sum(case)).standard_normal((N, C, H, W)).astype(np.float32)
+    want = F.max_pool2d(torch.from_numpy(x).double(), k, s, p).numpy()
+    assert np.array_equal(oracle.maxpool2d(x, k, s, p).astype(np.float64), want)
+    want_relu = F.max_pool2d(torch.relu(torch.from_numpy(x).double()), k, s, p).numpy()
+    assert np.array_equal(oracle.maxpool2d(x, k, s, p, relu=True).astype(np.float64), want_relu)
+
+
+def test_maxpool_special_cases(oracle):
+    g = rng(123)
+    x = g.standard_normal((2, 3, 6, 5)).astype(np.float32)
+    # a 1 x 1 window at stride 1 is the identity; with ReLU it is max(x, 0)
+    assert np.array_equal(oracle.maxpool2d(x, 1, 1), x)
+    assert np.array_equal(oracle.maxpool2d(x, 1, 1, relu=True), np.maximum(x, 0.0))
+    # ReLU commutes with the maximum (both are monotone)
+    assert np.array_equal(oracle.maxpool2d(x, 3, 2, 1, relu=True),
+                          np.maximum(oracle.maxpool2d(x, 3, 2, 1), 0.0))
+    # a window that covers the whole plane returns the plane's maximum, padding never wins
+    neg = -np.abs(x) - 1.0
+    full = oracle.maxpool2d(neg, 6, 6, 1)[:, :, 0, 0]
+    assert np.array_equal(full, neg[:, :, :5, :5].max(axis=(2, 3)))
+    # brute force over windows, written with slices only
+    k, s = 2, 2
+    got = oracle.maxpool2d(x, k, s)
+    for oy in range(got.shape[2]):
+        for ox in range(got.shape[3]):
+            assert np.array_equal(got[:, :, oy, ox],
+                                  x[:, :, oy * s:oy * s + k, ox * s:ox * s + k].max(axis=(2, 3)))
+
+
 def test_speedup_model_reproduces_printed_value(oracle):
     rows = [l.split() for l in open(os.path.join(GOLDEN, "efficiency_model.txt"))
             if l.strip() and not l.startswith("#")]
