@@ -187,6 +187,22 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
                                   int C_out, int stride, float *out, void *cuda_stream);
 
 /*
+ * The Pool layer that closes the block (Section 3.2, "Training XNOR-Networks":
+ * the order is BatchNorm, BinActiv, BinConv, Pool, with an optional ReLU after
+ * the binary convolution): max pooling of BinConv's output.
+ *   x     in   fp32  [N][C][H][W]           device, 16-byte aligned
+ *   out   out  fp32  [N][C][H_out][W_out]   H_out = (H + 2 pad - k) / stride + 1 rounded down
+ *   relu  != 0: max(v, 0) is applied to every input value first
+ * A tap outside the image takes no part in the maximum (0 <= pad < k, so every
+ * window holds at least one pixel).  Maxima of fp32 values are exact: results
+ * are bit-identical to the plain definition.  Asynchronous on `cuda_stream`.
+ * INVALID_ARG for null/misaligned pointers, non-positive sizes, pad outside
+ * [0, k), k larger than the padded image; UNSUPPORTED for k > 11.
+ */
+xnor_status xnor_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride, int pad,
+                           int relu, float *out, void *cuda_stream);
+
+/*
  * Which BinConv engine xnor_conv2d_forward uses.  XNOR_ENGINE_AUTO (default)
  * picks by shape: the tensor-core engine where it applies, else the CUDA-core
  * one.  Process-wide; meant for tests and measurements.  With an engine

@@ -31,6 +31,7 @@ EXPORTS = [
     "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
     "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
+    "xnor_maxpool2d",
 ]
 
 
@@ -81,6 +82,8 @@ def load():
     lib.xnor_get_engine.restype = ci
     lib.xnor_check_device.restype = ci
     lib.xnor_check_device.argtypes = [vp]
+    lib.xnor_maxpool2d.restype = ci
+    lib.xnor_maxpool2d.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
     lib.xnor_selftest_wait_timeout.restype = ci
     lib.xnor_selftest_wait_timeout.argtypes = [vp]
     _lib = lib
@@ -146,6 +149,13 @@ def xnor_get_engine():
 def xnor_check_device(stream=None):
     """Synchronises the stream and raises XnorError if a device-side wait expired."""
     _check(load().xnor_check_device(_stream(stream)), "xnor_check_device")
+
+
+def xnor_maxpool2d(x, k, stride, pad, relu, out, stream=None):
+    N, C, H, W = x.shape
+    _check(load().xnor_maxpool2d(_ptr(x, torch.float32), N, C, H, W, int(k), int(stride), int(pad),
+                                 1 if relu else 0, _ptr(out, torch.float32), _stream(stream)),
+           "xnor_maxpool2d")
 
 
 def xnor_selftest_wait_timeout(stream=None):

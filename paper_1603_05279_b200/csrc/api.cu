@@ -119,6 +119,17 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
                                              acc_out, (cudaStream_t)cuda_stream));
 }
 
+xnor_status xnor_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride, int pad,
+                           int relu, float *out, void *cuda_stream) {
+  if (bad_ptr(x) || bad_ptr(out)) return XNOR_ERR_INVALID_ARG;
+  if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || k < 1 || stride < 1 || pad < 0 || pad >= k ||
+      k > H + 2 * pad || k > W + 2 * pad)
+    return XNOR_ERR_INVALID_ARG;
+  if (k > 11) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_maxpool2d(x, N, C, H, W, k, stride, pad, relu != 0, out,
+                                          (cudaStream_t)cuda_stream));
+}
+
 xnor_status xnor_selftest_wait_timeout(void *cuda_stream) {
   return from_cuda(xnor::launch_wait_timeout_selftest((cudaStream_t)cuda_stream));
 }
