@@ -187,6 +187,36 @@ xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_i
                                   int C_out, int stride, float *out, void *cuda_stream);
 
 /*
+ * BinConv with the NEXT layer's BinActiv fused into its epilogue.  The block
+ * order of Section 3.2 makes the output of one BinConv (after the residual add,
+ * where there is one) the input of the next BatchNorm + BinActiv; the epilogue
+ * holds those fp32 values in registers, so it can emit what the next BinConv
+ * consumes without the fp32 tensor making a round trip through memory:
+ *   y = fmaf(next_scale[co], out[n][co][p], next_shift[co])   (identity if both NULL)
+ *   x_packed_next  u32 [N][H_out][W_out][ceil(C_out/32)]   bit = (y >= 0), along the filters
+ *   A_parts        fp32 [parts][N][H_out][W_out]           partial sums over filters of |y|
+ * `out` may be NULL (the fp32 tensor is then not written at all) or a buffer as
+ * in xnor_conv2d_forward; residual as there; no acc_out.  Values of out, and
+ * therefore the sign bits, are the ones xnor_conv2d_forward produces.
+ * xnor_conv2d_binactiv_parts(d) gives `parts` for the shape and the engine in
+ * force (set the engine before asking, do not change it in between); 0 means
+ * the fused kernel does not cover the shape (needs the tensor-core engine and
+ * C_out % 32 == 0): the call then returns UNSUPPORTED and the caller runs
+ * xnor_conv2d_forward + xnor_binactiv instead.
+ * xnor_binactiv_finish completes the next layer's BinActiv: A = (sum of the
+ * parts, in index order) / C_in of d_next, K = box filter of A for d_next's
+ * geometry (d_next: N, C_in = this C_out, H = H_out, W = W_out, its own k, stride, pad).
+ */
+int xnor_conv2d_binactiv_parts(const xnor_conv_desc *d);
+xnor_status xnor_conv2d_forward_binactiv(const uint32_t *x_packed, const uint32_t *w_packed,
+                                         const float *alpha, const float *K, const float *residual,
+                                         const xnor_conv_desc *d, float *out, const float *next_scale,
+                                         const float *next_shift, uint32_t *x_packed_next,
+                                         float *A_parts, void *cuda_stream);
+xnor_status xnor_binactiv_finish(const float *A_parts, int parts, const xnor_conv_desc *d_next,
+                                 float *A, float *K, void *cuda_stream);
+
+/*
  * The Pool layer that closes the block (Section 3.2, "Training XNOR-Networks":
  * the order is BatchNorm, BinActiv, BinConv, Pool, with an optional ReLU after
  * the binary convolution): max pooling of BinConv's output.

@@ -31,7 +31,7 @@ EXPORTS = [
     "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
     "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
-    "xnor_maxpool2d",
+    "xnor_maxpool2d", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
 ]
 
 
@@ -82,6 +82,13 @@ def load():
     lib.xnor_get_engine.restype = ci
     lib.xnor_check_device.restype = ci
     lib.xnor_check_device.argtypes = [vp]
+    lib.xnor_conv2d_binactiv_parts.restype = ci
+    lib.xnor_conv2d_binactiv_parts.argtypes = [ctypes.POINTER(xnor_conv_desc)]
+    lib.xnor_conv2d_forward_binactiv.restype = ci
+    lib.xnor_conv2d_forward_binactiv.argtypes = [vp, vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp,
+                                                 vp, vp, vp, vp, vp]
+    lib.xnor_binactiv_finish.restype = ci
+    lib.xnor_binactiv_finish.argtypes = [vp, ci, ctypes.POINTER(xnor_conv_desc), vp, vp, vp]
     lib.xnor_maxpool2d.restype = ci
     lib.xnor_maxpool2d.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
     lib.xnor_selftest_wait_timeout.restype = ci
@@ -149,6 +156,29 @@ def xnor_get_engine():
 def xnor_check_device(stream=None):
     """Synchronises the stream and raises XnorError if a device-side wait expired."""
     _check(load().xnor_check_device(_stream(stream)), "xnor_check_device")
+
+
+def xnor_conv2d_binactiv_parts(d):
+    """Partial planes the fused call writes for this shape (0: not covered)."""
+    return int(load().xnor_conv2d_binactiv_parts(ctypes.byref(d)))
+
+
+def xnor_conv2d_forward_binactiv(x_packed, w_packed, alpha, K, residual, d, out, next_scale,
+                                 next_shift, x_packed_next, A_parts, stream=None):
+    _check(load().xnor_conv2d_forward_binactiv(
+        _ptr(x_packed, torch.int32), _ptr(w_packed, torch.int32), _ptr(alpha, torch.float32),
+        _ptr(K, torch.float32), _ptr(residual, torch.float32) if residual is not None else None,
+        ctypes.byref(d), _ptr(out, torch.float32) if out is not None else None,
+        _ptr(next_scale, torch.float32) if next_scale is not None else None,
+        _ptr(next_shift, torch.float32) if next_shift is not None else None,
+        _ptr(x_packed_next, torch.int32), _ptr(A_parts, torch.float32), _stream(stream)),
+        "xnor_conv2d_forward_binactiv")
+
+
+def xnor_binactiv_finish(A_parts, parts, d_next, A, K, stream=None):
+    _check(load().xnor_binactiv_finish(_ptr(A_parts, torch.float32), int(parts), ctypes.byref(d_next),
+                                       _ptr(A, torch.float32), _ptr(K, torch.float32), _stream(stream)),
+           "xnor_binactiv_finish")
 
 
 def xnor_maxpool2d(x, k, stride, pad, relu, out, stream=None):

@@ -119,6 +119,59 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
                                              acc_out, (cudaStream_t)cuda_stream));
 }
 
+namespace {
+
+xnor::TcVariant current_variant() {
+  if (g_engine == XNOR_ENGINE_UMMA_STREAM) return xnor::kTcSingleStream;
+  if (g_engine == XNOR_ENGINE_UMMA_SINGLE) return xnor::kTcSingle;
+  if (g_engine == XNOR_ENGINE_UMMA_PAIR) return xnor::kTcPair;
+  if (g_engine == XNOR_ENGINE_UMMA_PAIR_STREAM) return xnor::kTcPairStream;
+  return xnor::kTcAuto;
+}
+
+bool good_desc(const xnor_conv_desc *d) {
+  return d && d->N > 0 && d->C_in > 0 && d->H > 0 && d->W > 0 && d->C_out > 0 && d->k_h > 0 &&
+         d->k_w > 0 && d->stride >= 1 && d->pad >= 0 && d->k_h <= d->H + 2 * d->pad &&
+         d->k_w <= d->W + 2 * d->pad;
+}
+
+}  // namespace
+
+int xnor_conv2d_binactiv_parts(const xnor_conv_desc *d) {
+  if (!good_desc(d) || g_engine == XNOR_ENGINE_POPC || d->k_h > 11 || d->k_w > 11 ||
+      (long long)d->C_in * d->k_h * d->k_w >= (1LL << 24))
+    return 0;
+  return xnor::tc_fused_parts(xnor::make_geom(*d), current_variant());
+}
+
+xnor_status xnor_conv2d_forward_binactiv(const uint32_t *x_packed, const uint32_t *w_packed,
+                                         const float *alpha, const float *K, const float *residual,
+                                         const xnor_conv_desc *d, float *out, const float *next_scale,
+                                         const float *next_shift, uint32_t *x_packed_next,
+                                         float *A_parts, void *cuda_stream) {
+  if (!good_desc(d)) return XNOR_ERR_INVALID_ARG;
+  if (bad_ptr(x_packed) || bad_ptr(w_packed) || bad_ptr(alpha) || bad_ptr(K) ||
+      bad_ptr(x_packed_next) || bad_ptr(A_parts))
+    return XNOR_ERR_INVALID_ARG;
+  if ((residual && misaligned(residual)) || (out && misaligned(out)) ||
+      (next_scale == nullptr) != (next_shift == nullptr) ||
+      (next_scale && (misaligned(next_scale) || misaligned(next_shift))))
+    return XNOR_ERR_INVALID_ARG;
+  if (xnor_conv2d_binactiv_parts(d) == 0) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_binconv_tc_fused(x_packed, w_packed, alpha, K, residual,
+                                                 xnor::make_geom(*d), out, next_scale, next_shift,
+                                                 x_packed_next, A_parts, current_variant(),
+                                                 (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_binactiv_finish(const float *A_parts, int parts, const xnor_conv_desc *d_next,
+                                 float *A, float *K, void *cuda_stream) {
+  if (!good_desc(d_next) || parts < 1 || bad_ptr(A_parts) || bad_ptr(A) || bad_ptr(K))
+    return XNOR_ERR_INVALID_ARG;
+  return from_cuda(xnor::launch_binactiv_finish(A_parts, parts, xnor::make_geom(*d_next), A, K,
+                                                (cudaStream_t)cuda_stream));
+}
+
 xnor_status xnor_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride, int pad,
                            int relu, float *out, void *cuda_stream) {
   if (bad_ptr(x) || bad_ptr(out)) return XNOR_ERR_INVALID_ARG;

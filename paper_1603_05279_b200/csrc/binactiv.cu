@@ -1,6 +1,8 @@
 // BatchNorm affine + BinActiv (Section 3.2): sign bits packed along channels,
 // A = channel mean of |y|, then K = box filter of zero-padded A at the
 // convolution's output positions.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace xnor {
@@ -219,6 +221,8 @@ box_filter_kernel(const float *__restrict__ A, int H, int W, int kh, int kw, int
 
 }  // namespace
 
+cudaError_t launch_box_filter(const float *A, const ConvGeom &g, float *K, cudaStream_t st);
+
 cudaError_t launch_binactiv(const float *x, const float *scale, const float *shift,
                             const ConvGeom &g, uint32_t *x_packed, float *A, float *K,
                             cudaStream_t st) {
@@ -264,6 +268,10 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
 #undef XNOR_PACK
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  return launch_box_filter(A, g, K, st);
+}
+
+cudaError_t launch_box_filter(const float *A, const ConvGeom &g, float *K, cudaStream_t st) {
   if (g.N > 65535) return cudaErrorInvalidValue;
   const dim3 kgrid((unsigned)((g.Ho * g.Wo + 255) / 256), (unsigned)g.N);
   const int ks = g.kh == g.kw ? g.kh : 0;
@@ -278,6 +286,30 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   return cudaGetLastError();
 }
 
+
+namespace {
+
+// A[i] = (part 0 + part 1 + ...)[i] / C, the parts added in index order.
+__global__ void __launch_bounds__(256)
+sum_parts_kernel(const float *__restrict__ parts, int nparts, size_t n, float C, float *__restrict__ A) {
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (size_t)gridDim.x * 256) {
+    float s = 0.0f;
+    for (int p = 0; p < nparts; ++p) s += __ldg(parts + (size_t)p * n + i);
+    A[i] = s / C;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_binactiv_finish(const float *A_part, int parts, const ConvGeom &g, float *A,
+                                   float *K, cudaStream_t st) {
+  const size_t n = (size_t)g.N * g.H * g.W;
+  const unsigned grid = (unsigned)std::min<size_t>((n + 255) / 256, 148 * 8);
+  sum_parts_kernel<<<grid, 256, 0, st>>>(A_part, parts, n, (float)g.C, A);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return launch_box_filter(A, g, K, st);
+}
 
 // ---------------------------------------------------------------------------
 // xnor_binactiv_static: the same two kernels, with the A plane kept in a

@@ -153,6 +153,13 @@ struct TcParams {
   int row_words;               // packed words per filter row = k_h*k_w*Cw
   int pair;                    // 1: two CTAs (a cluster) share every MMA: 256 pixels x NT filters
   int NTh;                     // filter rows of a slab that one CTA expands and holds: NT or NT/2
+  // Fused BinActiv of the next layer (kFuse kernels): the epilogue also applies the next
+  // BatchNorm affine to its output values, packs their signs along the filters (the next
+  // layer's channels) and sums |y| over the filters it handles.
+  const float *nscale, *nshift;      // [C_out], both null = identity
+  uint32_t *xp_next;                 // u32 [N][Ho][Wo][Cw_next]
+  float *A_part;                     // fp32 [nslabs * epi_split][N][Ho][Wo]: partial sums of |y|
+  int Cw_next;                       // ceil(C_out / 32)
   int resident;                // 1: resident schedule (stages = all stages of a slab)
   int epi_split;               // warps per lane quarter that drain an accumulator
   int any_swap;                // some bit of swap_mask is set
@@ -776,11 +783,20 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
 // run of the NCHW output row.
 // Drains items [i0, i1), the k0-th and following of the CTA.  Of every item this warp takes
 // the 16-column groups e, e + esplit, ... (esplit warps share a quarter of the lanes).
-template <bool kRes>
+// kFuse: the groups a warp takes come in pairs (32 consecutive filters = one packed word of the
+// next layer's input); see the fused emit below.
+template <bool kRes, bool kFuse>
 __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, long long i1,
                               long long k0, uint32_t tmem_base, int quarter, int e, int lane) {
   const int b_end = P.NT / 16;
   const int esplit = kRes ? P.epi_split : 1;
+  // the k-th group of this warp: groups e, e + esplit, ... or, fused, the two groups of the
+  // pairs e, e + esplit, ...
+  const int units = kFuse ? b_end / 2 : b_end;
+  const int nk = ((units - e + esplit - 1) / esplit) * (kFuse ? 2 : 1);
+  auto group_of = [&](int k) {
+    return kFuse ? 2 * (e + esplit * (k >> 1)) + (k & 1) : e + esplit * k;
+  };
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t howo = (uint32_t)HoWo;
   // the fast store paths: offsets of 16 consecutive filters fit 32 bits, no integer output
@@ -792,9 +808,9 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   else { tile = (int)(i0 / P.nslabs); slab = (int)(i0 - (long long)tile * P.nslabs); }
   bool ok = true;
   // this lane's output pixel in a tile: whether it exists, its K, offset of (image, filter 0, pixel)
-  struct Pix { bool valid; float kv; size_t obase; };
+  struct Pix { bool valid; float kv; size_t obase; size_t gpix; };   // gpix: pixel index over all images
   auto decode = [&](int t) {
-    Pix px{false, 0.0f, 0};
+    Pix px{false, 0.0f, 0, 0};
     const uint32_t m = ((uint32_t)t * (P.pair ? 2u : 1u) + S.rank) * kTileM + (uint32_t)(quarter * 32 + lane);
     if (m < (uint32_t)P.L) {
       const uint32_t r = fast_div(m, P.div_wq_m, P.div_wq_s);
@@ -806,6 +822,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         px.valid = true;
         px.kv = __ldg(P.K + (size_t)n * HoWo + pix);
         px.obase = (size_t)n * P.Co * HoWo + pix;
+        px.gpix = (size_t)n * HoWo + pix;
       }
     }
     return px;
@@ -820,6 +837,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     const bool valid = px.valid;
     const float kv = px.kv;
     const size_t obase = px.obase;
+    const size_t obase_pix = px.gpix;
     // the item after this one; its pixel is decoded (and its K loaded) while this one drains
     int ntile = tile, nslab = slab;
     bool next_new;
@@ -905,24 +923,68 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       }
     };
 
+    // Fused: out = D K alpha (+ residual) as above (stored only if the caller wants the fp32
+    // tensor), then y = fmaf(scale, out, shift) of the next layer's BatchNorm, the sign bit of
+    // y into the word of this pair of groups, |y| into this warp's partial sum for A.
+    uint32_t word = 0u;
+    float asum = 0.0f;
+    auto emit_fused = [&](int b, const int32_t r[16]) {
+      if (!valid) return;
+      const int co = co0 + b * 16;
+      const float *rp = P.residual + obase + (size_t)co * HoWo;
+      float *op = P.out + obase + (size_t)co * HoWo;
+#pragma unroll
+      for (int j4 = 0; j4 < 4; ++j4) {
+        const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
+        float4 sc = make_float4(1.0f, 1.0f, 1.0f, 1.0f), sh = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (P.nscale != nullptr) {
+          sc = __ldg(reinterpret_cast<const float4 *>(P.nscale + co) + j4);
+          sh = __ldg(reinterpret_cast<const float4 *>(P.nshift + co) + j4);
+        }
+        const float a4[4] = {al.x, al.y, al.z, al.w};
+        const float s4[4] = {sc.x, sc.y, sc.z, sc.w}, h4[4] = {sh.x, sh.y, sh.z, sh.w};
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const int j = j4 * 4 + jj;
+          float v = __fmul_rn(__fmul_rn(__int_as_float(r[j]), kv), a4[jj]);
+          if (P.residual != nullptr) v += rp[(uint32_t)j * howo];
+          if (P.out != nullptr) op[(uint32_t)j * howo] = v;
+          const float y = P.nscale != nullptr ? __fmaf_rn(s4[jj], v, h4[jj]) : v;
+          if (y >= 0.0f) word |= 1u << ((co + j) & 31);
+          asum += fabsf(y);
+        }
+      }
+    };
+
     // One copy of the code: the next 16 columns are being loaded into `nx` while the
     // current 16 (copied out to `cur`) are scaled and stored.
     int32_t nx[16], cur[16];
-    tmem_ld16(t_acc + (uint32_t)(e * 16), nx);
+    tmem_ld16(t_acc + (uint32_t)(group_of(0) * 16), nx);
 #pragma unroll 1
-    for (int b = e; b < b_end; b += esplit) {
+    for (int k = 0; k < nk; ++k) {
+      const int b = group_of(k);
       tmem_wait16(nx);
 #pragma unroll
       for (int j = 0; j < 16; ++j) cur[j] = nx[j];
-      if (b + esplit < b_end) {
-        tmem_ld16(t_acc + (uint32_t)((b + esplit) * 16), nx);
+      if (k + 1 < nk) {
+        tmem_ld16(t_acc + (uint32_t)(group_of(k + 1) * 16), nx);
       } else {                                   // that was the last load: release the buffer
         tc_fence_before();
         __syncwarp();
         if (lane == 0) { if (P.pair) mbar_arrive_cluster(S.aempty + 8u * ab, 0u); else mbar_arrive(S.aempty + 8u * ab); }
       }
-      emit(b, cur);
+      if (kFuse) {
+        emit_fused(b, cur);
+        if ((k & 1) && valid) {                  // the pair is complete: its word of the next input
+          P.xp_next[(obase_pix) * (size_t)P.Cw_next + (size_t)((co0 + b * 16) >> 5)] = word;
+          word = 0u;
+        }
+      } else {
+        emit(b, cur);
+      }
     }
+    if (kFuse && valid)
+      P.A_part[(size_t)(slab * esplit + e) * ((size_t)P.N * HoWo) + obase_pix] = asum;
     px = npx;
     tile = ntile;
     slab = nslab;
@@ -933,7 +995,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   return ok;
 }
 
-template <bool kRes, bool kPair>
+template <bool kRes, bool kPair, bool kFuse>
 __global__ void __launch_bounds__(kThreads, 1)
 binconv_tc_kernel(const __grid_constant__ TcParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -1015,7 +1077,7 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     else if (kRes && P.pat_group > kPatWarps && warp >= kWgtWarp0 + 4)
       patch_role<kRes>(P, S, i0, i1, kPatWarps + warp - (kWgtWarp0 + 4), lane);   // helpers
     else if (!kRes) {
-      if (warp < kEpiWarps) epilogue_role<false>(P, S, i0, i1, 0, tmem_base, warp, 0, lane);
+      if (warp < kEpiWarps) epilogue_role<false, kFuse>(P, S, i0, i1, 0, tmem_base, warp, 0, lane);
       else weight_dispatch(P, S, i1 - i0, (int)(i0 % P.nslabs), 1u, wt, lane);
     } else {
       // Slab visits of this CTA in order.  The weight warps expand the slab, then every
@@ -1030,7 +1092,7 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
         const long long vend = min(i1, (long long)(slab + 1) * P.ntiles);
         if (wgt) ok = weight_dispatch(P, S, 1, slab, (visit & 1u) ^ 1u, wt, lane);
         if (ok && e < P.epi_split)
-          ok = epilogue_role<true>(P, S, it, vend, it - i0, tmem_base, warp & 3, e, lane);
+          ok = epilogue_role<true, kFuse>(P, S, it, vend, it - i0, tmem_base, warp & 3, e, lane);
         it = vend;
         ++visit;
       }
@@ -1081,13 +1143,13 @@ void plan_stage(TcParams &P) {
 
 // Filters per slab for `ns` slabs.  A pair splits the rows of a slab between its two CTAs
 // (halves of a multiple of 16 rows each).
-int slab_width(int Co, int ns, bool pair) {
+int slab_width(int Co, int ns, bool pair) {     // pair: also set for the fused epilogue (32-filter words)
   const int q = pair ? 32 : 16;
   return ((Co + ns - 1) / ns + q - 1) / q * q;
 }
 
 // schedule: 0 = resident when the slab fits, 1 = streaming.  pair: CTA pairs (clusters of 2).
-Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
+Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   Plan pl{};
   pl.ok = false;
   TcParams &P = pl.P;
@@ -1144,7 +1206,7 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
     // (measured) slabs below 128 filters pay only when one slab holds all filters.
     for (int ns = min_slabs; ns <= 16 && !P.resident; ++ns) {
       P.nslabs = ns;
-      P.NT = slab_width(g.Co, ns, pair);
+      P.NT = slab_width(g.Co, ns, pair || fuse);
       P.NTh = pair ? P.NT / 2 : P.NT;
       if (P.NT < 128 && ns > 1) break;
       // The slab is expanded once per visit, so four weight warps are enough when a thread
@@ -1165,7 +1227,7 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
   }
   if (!P.resident) {
     P.nslabs = min_slabs;
-    P.NT = slab_width(g.Co, P.nslabs, pair);
+    P.NT = slab_width(g.Co, P.nslabs, pair || fuse);
     P.NTh = pair ? P.NT / 2 : P.NT;
     P.wgt_warps = kWgtWarps;
     P.pat_group = kPatWarps;
@@ -1182,7 +1244,8 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair) {
   P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
   // worker warps per quarter of the lanes in the resident schedule: the four epilogue warps
   // and the weight warps (all eight, or the four that are not patch helpers)
-  P.epi_split = std::min(P.pat_group > kPatWarps ? 2 : kEpiSplitMax, P.NT / 16);
+  P.epi_split = std::min(P.pat_group > kPatWarps ? 2 : kEpiSplitMax, P.NT / (fuse ? 32 : 16));
+  if (fuse && (g.Co & 31) != 0) return pl;          // whole words of the next layer's input
   P.stages = stages; P.npb = npb;
   // small patches: every patch warp builds whole patches on its own, three at a time
   P.pat_sub = subgroups(npb);
@@ -1233,23 +1296,23 @@ namespace {
 
 // The plan of a variant.  kTcAuto (measured on the AlexNet and ResNet-18 shapes): one CTA per
 // SM unless only a pair, each CTA holding half of a slab, can keep the filters resident.
-Plan plan_variant(const ConvGeom &g, TcVariant v) {
+Plan plan_variant(const ConvGeom &g, TcVariant v, bool fuse = false) {
   switch (v) {
-    case kTcSingle: return make_plan(g, 0, false);
-    case kTcSingleStream: return make_plan(g, 1, false);
-    case kTcPair: return make_plan(g, 0, true);
-    case kTcPairStream: return make_plan(g, 1, true);
+    case kTcSingle: return make_plan(g, 0, false, fuse);
+    case kTcSingleStream: return make_plan(g, 1, false, fuse);
+    case kTcPair: return make_plan(g, 0, true, fuse);
+    case kTcPairStream: return make_plan(g, 1, true, fuse);
     default: break;
   }
-  Plan single = make_plan(g, 0, false);
+  Plan single = make_plan(g, 0, false, fuse);
   if (single.ok && single.P.resident) return single;
-  Plan pair = make_plan(g, 0, true);
+  Plan pair = make_plan(g, 0, true, fuse);
   // neither resident: a pair pays when the slabs are wide (each CTA expands half the rows)
   if (pair.ok && (pair.P.resident || !single.ok || pair.P.NT > 128)) return pair;
   return single;
 }
 
-template <bool kRes, bool kPair>
+template <bool kRes, bool kPair, bool kFuse>
 cudaError_t launch_variant(const Plan &pl, unsigned units, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(kPair ? 2 * units : units);
@@ -1263,29 +1326,29 @@ cudaError_t launch_variant(const Plan &pl, unsigned units, cudaStream_t st) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, binconv_tc_kernel<kRes, kPair>, pl.P);
+  return cudaLaunchKernelEx(&cfg, binconv_tc_kernel<kRes, kPair, kFuse>, pl.P);
 }
 
 }  // namespace
 
 bool umma_tc_supported(const ConvGeom &g, TcVariant v) { return plan_variant(g, v).ok; }
 
-cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
-                              const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, TcVariant variant, cudaStream_t st) {
-  Plan pl = plan_variant(g, variant);
-  if (!pl.ok) return cudaErrorInvalidValue;
+namespace {
+
+cudaError_t launch_plan(Plan &pl, cudaStream_t st, bool fuse) {
   TcParams &P = pl.P;
-  P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
-  P.out = out; P.acc_out = acc_out;
   static bool attr_set = false;
   if (!attr_set) {
-    const void *kernels[4] = {(const void *)binconv_tc_kernel<false, false>,
-                              (const void *)binconv_tc_kernel<true, false>,
-                              (const void *)binconv_tc_kernel<false, true>,
-                              (const void *)binconv_tc_kernel<true, true>};
+    const void *kernels[8] = {(const void *)binconv_tc_kernel<false, false, false>,
+                              (const void *)binconv_tc_kernel<true, false, false>,
+                              (const void *)binconv_tc_kernel<false, true, false>,
+                              (const void *)binconv_tc_kernel<true, true, false>,
+                              (const void *)binconv_tc_kernel<false, false, true>,
+                              (const void *)binconv_tc_kernel<true, false, true>,
+                              (const void *)binconv_tc_kernel<false, true, true>,
+                              (const void *)binconv_tc_kernel<true, true, true>};
     cudaError_t e = cudaSuccess;
-    for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+    for (int i = 0; i < 8 && e == cudaSuccess; ++i)
       e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)kSmemMax);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
@@ -1296,8 +1359,13 @@ cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const floa
   // one CTA per SM, or one pair per two SMs
   const unsigned units = (unsigned)std::min<long long>(total, P.pair ? sms / 2 : sms);
   cudaError_t e_;
-  if (P.pair) e_ = P.resident ? launch_variant<true, true>(pl, units, st) : launch_variant<false, true>(pl, units, st);
-  else e_ = P.resident ? launch_variant<true, false>(pl, units, st) : launch_variant<false, false>(pl, units, st);
+  if (fuse) {
+    if (P.pair) e_ = P.resident ? launch_variant<true, true, true>(pl, units, st) : launch_variant<false, true, true>(pl, units, st);
+    else e_ = P.resident ? launch_variant<true, false, true>(pl, units, st) : launch_variant<false, false, true>(pl, units, st);
+  } else {
+    if (P.pair) e_ = P.resident ? launch_variant<true, true, false>(pl, units, st) : launch_variant<false, true, false>(pl, units, st);
+    else e_ = P.resident ? launch_variant<true, false, false>(pl, units, st) : launch_variant<false, false, false>(pl, units, st);
+  }
   if (e_ != cudaSuccess) {
     (void)cudaGetLastError();
     if (getenv("XNOR_DEBUG"))
@@ -1305,6 +1373,43 @@ cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const floa
               units, P.pair, pl.smem);
   }
   return e_;
+}
+
+}  // namespace
+
+cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                              const float *K, const float *residual, const ConvGeom &g,
+                              float *out, int32_t *acc_out, TcVariant variant, cudaStream_t st) {
+  Plan pl = plan_variant(g, variant);
+  if (!pl.ok) return cudaErrorInvalidValue;
+  TcParams &P = pl.P;
+  P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
+  P.out = out; P.acc_out = acc_out;
+  P.nscale = nullptr; P.nshift = nullptr; P.xp_next = nullptr; P.A_part = nullptr; P.Cw_next = 0;
+  return launch_plan(pl, st, false);
+}
+
+// Partial planes of |y| sums that the fused kernel writes for this shape: one per filter slab
+// and, in the resident schedule, per warp that shares a quarter of the lanes.  0: not supported.
+int tc_fused_parts(const ConvGeom &g, TcVariant variant) {
+  const Plan pl = plan_variant(g, variant, true);
+  if (!pl.ok) return 0;
+  return pl.P.nslabs * (pl.P.resident ? pl.P.epi_split : 1);
+}
+
+cudaError_t launch_binconv_tc_fused(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                                    const float *K, const float *residual, const ConvGeom &g,
+                                    float *out, const float *next_scale, const float *next_shift,
+                                    uint32_t *xp_next, float *A_part, TcVariant variant,
+                                    cudaStream_t st) {
+  Plan pl = plan_variant(g, variant, true);
+  if (!pl.ok) return cudaErrorInvalidValue;
+  TcParams &P = pl.P;
+  P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
+  P.out = out; P.acc_out = nullptr;
+  P.nscale = next_scale; P.nshift = next_shift; P.xp_next = xp_next; P.A_part = A_part;
+  P.Cw_next = (g.Co + 31) / 32;
+  return launch_plan(pl, st, true);
 }
 
 #ifdef XNOR_TRACE

@@ -51,6 +51,17 @@ bool umma_tc_supported(const ConvGeom &g, TcVariant v);
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
                               float *out, int32_t *acc_out, TcVariant v, cudaStream_t st);
+// BinConv with the next layer's BinActiv fused into its epilogue (sign bits packed along the
+// filters, partial sums of |y| per filter slab and epilogue warp); tc_fused_parts = number of
+// partial planes for the shape (0: the fused kernel does not cover it).
+int tc_fused_parts(const ConvGeom &g, TcVariant v);
+cudaError_t launch_binconv_tc_fused(const uint32_t *xp, const uint32_t *wp, const float *alpha,
+                                    const float *K, const float *residual, const ConvGeom &g,
+                                    float *out, const float *next_scale, const float *next_shift,
+                                    uint32_t *xp_next, float *A_part, TcVariant v, cudaStream_t st);
+// A = (sum of the partial planes) / C, then K = box filter of A for geometry g.
+cudaError_t launch_binactiv_finish(const float *A_part, int parts, const ConvGeom &g, float *A,
+                                   float *K, cudaStream_t st);
 // A one-warp kernel whose bounded wait expires (nothing signals its barrier).
 cudaError_t launch_wait_timeout_selftest(cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.
