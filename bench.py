@@ -324,12 +324,15 @@ class LayersJob:
 class ChainJob:
     """The 16-layer chain: weight binarisation, then 8 residual blocks."""
 
-    def __init__(self, batch, rank):
+    def __init__(self, batch, rank, fused=False):
         import torch
         from paper_1603_05279_b200 import binding as B
         from paper_1603_05279_b200.runner import ChainRunner
         self.torch, self.B = torch, B
+        self.fused = fused
         ch = ChainRunner(batch)
+        if fused:
+            ch.prepare_fused()
         self.ch = ch
         self.shapes = ch.shapes
         seed0 = du.rank_seed(wl.layer_seed("chain", 0), rank)
@@ -366,13 +369,18 @@ class ChainJob:
 
     def step(self, stream):
         self.ch.binarize_weights(stream)
-        self.ch.forward(stream)
+        if self.fused:
+            self.ch.forward_fused(stream)
+        else:
+            self.ch.forward(stream)
 
     def step_branches(self, stream):
         """The same step for graph capture.  The layers depend on one another, but the weight
         binarisations depend on nothing and a block's projection shortcut only on the block's
         input: both run on side branches and join where their results are consumed."""
         torch, B, ch = self.torch, self.B, self.ch
+        if self.fused:
+            return self.step(stream)
         if not hasattr(self, "_sw"):
             self._sw, self._sp = torch.cuda.Stream(), torch.cuda.Stream()
         fork = torch.cuda.Event()
@@ -456,7 +464,7 @@ def run_ours(args):
 
     # every rank has its own batch (weak scaling, no exchange on the data path)
     if args.workload == "chain":
-        job = ChainJob(args.batch, rank)
+        job = ChainJob(args.batch, rank, fused=args.fused)
     else:
         job = LayersJob(args.workload, args.layer_ids, args.batch, rank)
     torch.cuda.synchronize()
@@ -621,6 +629,7 @@ def run_ours(args):
         "config": {"workload": name if full else "subset of " + name,
                    "layers": [s.name for s in job.shapes],
                    "batch_per_gpu": job.images, "engine": engine,
+                   "fused_binactiv": bool(getattr(job, "fused", False)),
                    "l2": "step working set %d MB of inputs+outputs (L2 is 126 MB); no flush"
                          % ((job.h2d + job.d2h + (job.act_bytes if args.workload == "chain" else 0))
                             // 1000000),
@@ -652,6 +661,9 @@ def main():
     ap.add_argument("--ref-images", type=int, default=8,
                     help="images per layer per step of the reference (oracle) arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused", action="store_true",
+                    help="chain workload: every BinConv emits the next layer's BinActiv from its "
+                         "epilogue (the per-kernel breakdown still times the plain calls)")
     ap.add_argument("--no-branches", action="store_true",
                     help="capture the step as one chain of launches (no parallel branches)")
     ap.add_argument("--no-graph", action="store_true",

@@ -927,12 +927,18 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     // tensor), then y = fmaf(scale, out, shift) of the next layer's BatchNorm, the sign bit of
     // y into the word of this pair of groups, |y| into this warp's partial sum for A.
     uint32_t word = 0u;
-    float asum = 0.0f;
+    float as0 = 0.0f, as1 = 0.0f, as2 = 0.0f, as3 = 0.0f;     // four chains of the |y| sum
     auto emit_fused = [&](int b, const int32_t r[16]) {
       if (!valid) return;
       const int co = co0 + b * 16;
-      const float *rp = P.residual + obase + (size_t)co * HoWo;
+      uint32_t half = 0u;                     // the 16 sign bits of this group
       float *op = P.out + obase + (size_t)co * HoWo;
+      float res[16];                          // all 16 residual loads in flight together
+      if (P.residual != nullptr) {
+        const float *rp = P.residual + obase + (size_t)co * HoWo;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) res[j] = rp[(uint32_t)j * howo];
+      }
 #pragma unroll
       for (int j4 = 0; j4 < 4; ++j4) {
         const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
@@ -947,13 +953,17 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         for (int jj = 0; jj < 4; ++jj) {
           const int j = j4 * 4 + jj;
           float v = __fmul_rn(__fmul_rn(__int_as_float(r[j]), kv), a4[jj]);
-          if (P.residual != nullptr) v += rp[(uint32_t)j * howo];
+          if (P.residual != nullptr) v += res[j];
           if (P.out != nullptr) op[(uint32_t)j * howo] = v;
           const float y = P.nscale != nullptr ? __fmaf_rn(s4[jj], v, h4[jj]) : v;
-          if (y >= 0.0f) word |= 1u << ((co + j) & 31);
-          asum += fabsf(y);
+          half |= (y >= 0.0f ? 1u : 0u) << j;
+          if (jj == 0) as0 += fabsf(y);
+          else if (jj == 1) as1 += fabsf(y);
+          else if (jj == 2) as2 += fabsf(y);
+          else as3 += fabsf(y);
         }
       }
+      word |= half << (co & 16);              // C_out % 32 == 0: a group is the low or the high half
     };
 
     // One copy of the code: the next 16 columns are being loaded into `nx` while the
@@ -974,6 +984,9 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         if (lane == 0) { if (P.pair) mbar_arrive_cluster(S.aempty + 8u * ab, 0u); else mbar_arrive(S.aempty + 8u * ab); }
       }
       if (kFuse) {
+        // C_out is a multiple of 32, so a pair of groups lies inside the filters or (last slab)
+        // wholly beyond them
+        if (co0 + b * 16 >= P.Co) continue;
         emit_fused(b, cur);
         if ((k & 1) && valid) {                  // the pair is complete: its word of the next input
           P.xp_next[(obase_pix) * (size_t)P.Cw_next + (size_t)((co0 + b * 16) >> 5)] = word;
@@ -984,7 +997,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       }
     }
     if (kFuse && valid)
-      P.A_part[(size_t)(slab * esplit + e) * ((size_t)P.N * HoWo) + obase_pix] = asum;
+      P.A_part[(size_t)(slab * esplit + e) * ((size_t)P.N * HoWo) + obase_pix] = (as0 + as1) + (as2 + as3);
     px = npx;
     tile = ntile;
     slab = nslab;

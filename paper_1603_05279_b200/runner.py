@@ -138,6 +138,55 @@ class ChainRunner:
             self.run_layer(i, stream)
         return self.layers[-1]["out"]
 
+    def prepare_fused(self):
+        """Buffers of the fused forward: for every layer but the last, the partial |y| planes
+        its fused epilogue writes (0 parts: the shape is not covered and the layer runs the two
+        plain calls).  The engine in force now must be the one used by forward_fused."""
+        self.fused_parts = []
+        for i, L in enumerate(self.layers[:-1]):
+            parts = B.xnor_conv2d_binactiv_parts(L["desc"])
+            self.fused_parts.append(parts)
+            ho, wo = wl.out_hw(L["shape"])
+            L["A_parts"] = torch.empty((max(parts, 1), self.N, ho, wo), dtype=torch.float32,
+                                       device=self.device)
+        self.fused_parts.append(0)
+
+    def forward_fused(self, stream=None):
+        """The same chain with each BinConv emitting the next layer's BinActiv from its epilogue.
+        The output of a block's first convolution is consumed only by that BinActiv, so it is
+        never written as fp32; a block's output is (it is the next block's shortcut input)."""
+        n = len(self.layers)
+        L0 = self.layers[0]
+        B.xnor_binactiv(self.x0, L0["scale"], L0["shift"], L0["desc"], L0["x_packed"], L0["A"], L0["K"],
+                        stream)
+        for i, L in enumerate(self.layers):
+            residual = None
+            if i % 2 == 1:
+                b0 = i - 1
+                if b0 in self.proj:
+                    P = self.proj[b0]
+                    B.xnor_shortcut_conv1x1(self.layer_input(b0), P["w"], self.shapes[b0].stride,
+                                            P["out"], stream)
+                    residual = P["out"]
+                else:
+                    residual = self.layer_input(b0)
+            parts = self.fused_parts[i]
+            if parts > 0:
+                nxt = self.layers[i + 1]
+                out = L["out"] if i % 2 == 1 else None
+                B.xnor_conv2d_forward_binactiv(L["x_packed"], L["w_packed"], L["alpha"], L["K"],
+                                               residual, L["desc"], out, nxt["scale"], nxt["shift"],
+                                               nxt["x_packed"], L["A_parts"], stream)
+                B.xnor_binactiv_finish(L["A_parts"], parts, nxt["desc"], nxt["A"], nxt["K"], stream)
+            else:
+                B.xnor_conv2d_forward(L["x_packed"], L["w_packed"], L["alpha"], L["K"], residual,
+                                      L["desc"], L["out"], None, stream)
+                if i + 1 < n:
+                    nxt = self.layers[i + 1]
+                    B.xnor_binactiv(L["out"], nxt["scale"], nxt["shift"], nxt["desc"],
+                                    nxt["x_packed"], nxt["A"], nxt["K"], stream)
+        return self.layers[-1]["out"]
+
     def calibrate(self, eps=1e-5, stream=None):
         """Sets every BatchNorm to the statistics of its own input on the current batch
         (biased variance, gamma = 1, beta = 0), layer by layer.  Set-up, not the timed path:

@@ -77,3 +77,39 @@ def test_chain_benchmark_batch_sampled_images(oracle):
     for L in ch.layers:
         s = L["shape"]
         assert int(L["acc"].abs().max()) <= s.C_in * 9
+
+
+def test_fused_chain_is_consistent_with_the_plain_calls_layer_by_layer():
+    """The chain with BinActiv fused into every BinConv.  Parity of the fused call with the
+    oracle is established per layer elsewhere; here every fused layer of the running chain is
+    re-done with the two plain calls from the same inputs: the fp32 output (where the chain
+    keeps it) and the packed bits must be identical, A and K within the tolerance."""
+    N = 4
+    ch = ChainRunner(N)
+    g = np.random.Generator(np.random.Philox(2024))
+    ch.x0.copy_(torch.from_numpy(g.standard_normal(tuple(ch.x0.shape)).astype(np.float32)))
+    for L in ch.layers:
+        L["w"].copy_(torch.from_numpy((0.05 * g.standard_normal(tuple(L["w"].shape))).astype(np.float32)))
+    for P in ch.proj.values():
+        P["w"].copy_(torch.from_numpy((0.05 * g.standard_normal(tuple(P["w"].shape))).astype(np.float32)))
+    ch.binarize_weights()
+    ch.calibrate()
+    ch.prepare_fused()
+    assert sum(1 for p in ch.fused_parts if p > 0) == len(ch.layers) - 1
+    ch.forward_fused()
+    X.xnor_check_device()
+    for i, L in enumerate(ch.layers[:-1]):
+        nxt = ch.layers[i + 1]
+        residual = None
+        if i % 2 == 1:
+            b0 = i - 1
+            residual = ch.proj[b0]["out"] if b0 in ch.proj else ch.layer_input(b0)
+        out = torch.empty_like(L["out"])
+        X.xnor_conv2d_forward(L["x_packed"], L["w_packed"], L["alpha"], L["K"], residual, L["desc"], out, None)
+        if i % 2 == 1:
+            assert torch.equal(out, L["out"]), i
+        xp, A, K = X.alloc_binactiv(nxt["desc"])
+        X.xnor_binactiv(out, nxt["scale"], nxt["shift"], nxt["desc"], xp, A, K)
+        assert torch.equal(xp, nxt["x_packed"]), i
+        assert_close(host(nxt["A"]), host(A), "A of layer %d" % (i + 1))
+        assert_close(host(nxt["K"]), host(K), "K of layer %d" % (i + 1))

@@ -21,7 +21,9 @@ CASES = [(3, 64, 20, 20, 64, 3, 1, 1, 3, 1, 1, True),       # one slab of 64: tw
          (2, 96, 13, 13, 384, 3, 1, 1, 3, 1, 1, False),     # three slabs
          (2, 64, 18, 18, 128, 3, 2, 1, 3, 1, 1, False),     # stride 2
          (2, 40, 9, 11, 32, 5, 1, 2, 1, 1, 0, True),        # one pair only; channel tail in the input
-         (4, 128, 14, 14, 256, 3, 1, 1, 3, 2, 1, True)]
+         (4, 128, 14, 14, 256, 3, 1, 1, 3, 2, 1, True),
+         (2, 64, 10, 10, 512, 3, 2, 1, 3, 1, 1, False),     # slabs of 192: the last one holds 128 filters
+         (1, 32, 7, 7, 288, 1, 1, 0, 3, 1, 1, True)]
 
 
 def _run(case, engine, with_out, with_bn):
