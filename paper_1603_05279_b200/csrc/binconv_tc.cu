@@ -39,10 +39,20 @@
 //  tile, filter slab)): warps 0-3 epilogue (tensor memory -> registers ->
 //  coalesced NCHW stores of D * K * alpha (+ residual)), warp 4 issues the
 //  MMAs, warps 5-12 expand weights, warps 13-15 expand activation patches.
-//  Accumulators are double-buffered in tensor memory so the epilogue of one
+//  Accumulators are multi-buffered in tensor memory so the epilogue of one
 //  item overlaps the MMAs of the next.  Every wait is bounded: on expiry the
 //  CTA records XNOR_ERR_TIMEOUT in a device status word, stops, frees its
 //  tensor memory and exits.
+//
+//  CTA pairs (kPair kernels, clusters of 2).  One tcgen05.mma.cta_group::2
+//  drives the tensor cores of two SMs: M = 256 (each CTA's 128-position tile,
+//  patch and tensor memory) and each CTA expands and holds half of a slab's
+//  filter rows.  The producers of both CTAs arrive on the barriers of rank 0,
+//  whose MMA warp issues; its commits reach the consumer barriers of both.
+//
+//  Fused BinActiv (kFuse kernels).  The epilogue also applies the next layer's
+//  BatchNorm affine to its output values, packs their sign bits along the
+//  filters (the next layer's channels) and writes partial sums of |y|.
 //
 //  Two schedules.  "Resident": when the expanded rows of a filter slab fit in
 //  shared memory beside two patches, the slab is expanded ONCE per CTA and the
