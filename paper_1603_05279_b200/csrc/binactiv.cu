@@ -236,7 +236,8 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
                       (scale ? (size_t)g.Cw * 32 * sizeof(float2) : 0) +
                       (size_t)PG * kPix * g.Cw * sizeof(uint32_t) +
                       (size_t)PG * G * kPix * sizeof(float);
-  static bool attr_set = false;
+  static bool attr_flags[64] = {};
+  bool &attr_set = attr_done_for_current_device(attr_flags);
   if (!attr_set) {
     cudaError_t e = cudaSuccess;
     const void *kernels[4] = {(const void *)binactiv_pack_kernel<true, true>,

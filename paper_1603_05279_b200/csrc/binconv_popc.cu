@@ -139,7 +139,8 @@ cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const fl
   if (cwc > 8) cwc = 8;
   P.cwc = cwc;
   const size_t smem = words_per_cw * cwc * sizeof(uint32_t);
-  static bool attr_set = false;
+  static bool attr_flags[64] = {};
+  bool &attr_set = attr_done_for_current_device(attr_flags);
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(binconv_popc_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);

@@ -1360,7 +1360,8 @@ namespace {
 
 cudaError_t launch_plan(Plan &pl, cudaStream_t st, bool fuse) {
   TcParams &P = pl.P;
-  static bool attr_set = false;
+  static bool attr_flags[64] = {};
+  bool &attr_set = attr_done_for_current_device(attr_flags);
   if (!attr_set) {
     const void *kernels[8] = {(const void *)binconv_tc_kernel<false, false, false>,
                               (const void *)binconv_tc_kernel<true, false, false>,

@@ -43,6 +43,14 @@ cudaError_t launch_binactiv_static(const float *x, const float *scale, const flo
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
                                 float *out, int32_t *acc_out, cudaStream_t st);
+// Function attributes (dynamic shared-memory limits) belong to a device: a launcher sets them
+// once per device.  Returns the flag of the current device (out-of-range ids share the last).
+inline bool &attr_done_for_current_device(bool (&flags)[64]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); dev = 0; }
+  return flags[dev < 0 ? 0 : (dev > 63 ? 63 : dev)];
+}
+
 // Persistent tensor-core engine (strides 1 and 2).  Variants: one CTA per SM or CTA pairs
 // (one MMA drives two SMs), each with the filters of a slab resident in shared memory when
 // they fit or always streamed through a ring (re-expanded per work item).
