@@ -17,6 +17,13 @@ from .binding import (  # noqa: F401
     binconv_acc,
     scale_output,
     xnor_block,
+    xnor_block_ex,
+    box_filter_valid_taps,
+    relu,
+    quantize_k,
+    scale_output_k,
+    round_bf16,
+    bwn_conv,
     shortcut_conv1x1,
     maxpool2d,
     speedup_model,

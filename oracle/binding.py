@@ -149,6 +149,81 @@ def xnor_block(x, w, stride, pad, bn_scale=None, bn_shift=None, residual=None):
     return r
 
 
+def xnor_block_ex(x, w, stride, pad, bn_scale=None, bn_shift=None, residual=None, kbits=1,
+                  relu=False, k_valid_taps=False):
+    """The block with its options (k-bit activations, ReLU, border variant of K)."""
+    x, w = _f32(x), _f32(w)
+    bn_scale, bn_shift, residual = _f32(bn_scale), _f32(bn_shift), _f32(residual)
+    N, C, H, W = x.shape
+    Co, C2, kh, kw = w.shape
+    assert C == C2
+    Ho, Wo = out_extent(H, kh, stride, pad), out_extent(W, kw, stride, pad)
+    r = SimpleNamespace(
+        y=np.empty_like(x), H=np.empty(x.shape, np.int8), A=np.empty((N, H, W), np.float32),
+        K=np.empty((N, Ho, Wo), np.float32), B=np.empty(w.shape, np.int8),
+        alpha=np.empty((Co,), np.float32), acc=np.empty((N, Co, Ho, Wo), np.int32),
+        out=np.empty((N, Co, Ho, Wo), np.float32))
+    _load().oracle_xnor_block_ex(_p(x), _p(bn_scale), _p(bn_shift), _p(w), _p(residual),
+                                 *_i(N, C, H, W, Co, kh, kw, stride, pad, kbits,
+                                     1 if relu else 0, 1 if k_valid_taps else 0),
+                                 _p(r.y), _p(r.H), _p(r.A), _p(r.K), _p(r.B), _p(r.alpha),
+                                 _p(r.acc), _p(r.out))
+    return r
+
+
+def box_filter_valid_taps(A, kh, kw, stride, pad):
+    A = _f32(A)
+    N, H, W = A.shape
+    K = np.empty((N, out_extent(H, kh, stride, pad), out_extent(W, kw, stride, pad)),
+                 dtype=np.float32)
+    _load().oracle_box_filter_valid_taps(_p(A), *_i(N, H, W, kh, kw, stride, pad), _p(K))
+    return K
+
+
+def relu(v):
+    r = np.array(_f32(v), copy=True, order="C")
+    _load().oracle_relu(_p(r), ctypes.c_size_t(r.size))
+    return r
+
+
+def quantize_k(v, k):
+    """Level codes L of q_k (odd integers in [-(2^k-1), 2^k-1]); the level is L / (2^k - 1)."""
+    v = _f32(v)
+    L = np.empty(v.shape, dtype=np.int8)
+    _load().oracle_quantize_k(_p(v), ctypes.c_size_t(v.size), ctypes.c_int(int(k)), _p(L))
+    return L
+
+
+def scale_output_k(acc, k, K, alpha, residual=None):
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    K, alpha, residual = _f32(K), _f32(alpha), _f32(residual)
+    N, Co, Ho, Wo = acc.shape
+    out = np.empty(acc.shape, dtype=np.float32)
+    _load().oracle_scale_output_k(_p(acc), ctypes.c_int(int(k)), _p(K), _p(alpha), _p(residual),
+                                  *_i(N, Co, Ho, Wo), _p(out))
+    return out
+
+
+def round_bf16(v):
+    v = _f32(v)
+    r = np.empty_like(v)
+    _load().oracle_round_bf16(_p(v), ctypes.c_size_t(v.size), _p(r))
+    return r
+
+
+def bwn_conv(x, B, alpha, stride, pad, residual=None):
+    """Binary-Weight-Network convolution (I (+) B) alpha on real inputs x (Eq. 1)."""
+    x, alpha, residual = _f32(x), _f32(alpha), _f32(residual)
+    B = np.ascontiguousarray(B, dtype=np.int8)
+    N, C, H, W = x.shape
+    Co, C2, kh, kw = B.shape
+    assert C == C2
+    out = np.empty((N, Co, out_extent(H, kh, stride, pad), out_extent(W, kw, stride, pad)), np.float32)
+    _load().oracle_bwn_conv(_p(x), _p(B), _p(alpha), _p(residual),
+                            *_i(N, C, H, W, Co, kh, kw, stride, pad), _p(out))
+    return out
+
+
 def shortcut_conv1x1(x, w, stride):
     x, w = _f32(x), _f32(w)
     N, C, H, W = x.shape

@@ -20,6 +20,11 @@
  *   - real-valued sums (alpha, A, K, out) are accumulated in double and
  *     rounded to float once; the +/-1 convolution is exact int32.
  *
+ * Options beyond the main path (each a function of its own further down, all
+ * pinned by the CPU tests): the border variant of K that divides by the taps
+ * inside the image, ReLU on the block's output, k-bit activations q_k in place
+ * of sign(), and the Binary-Weight-Network convolution of Eq. 1 on real inputs.
+ *
  * The only parallelism is an OpenMP "parallel for" over independent outer
  * indices (images, filters); loop bodies are unchanged by it.
  */
@@ -189,6 +194,38 @@ void oracle_xnor_block(const float *x, const float *bn_scale, const float *bn_sh
   oracle_scale_output(acc, K, alpha, residual, N, Co, Ho, Wo, out);
 }
 
+/* The same block with the options the paper mentions around it: kbits > 1
+ * quantises the normalised input with q_k instead of sign() (Hs then holds the
+ * level codes, and the sums are divided by 2^k - 1); k_valid_taps selects the
+ * border variant of K; relu applies max(., 0) to the block's output.  With
+ * kbits = 1 and both flags 0 it is oracle_xnor_block.  Forward declarations:
+ * the option functions are defined further down. */
+void oracle_box_filter_valid_taps(const float *A, int N, int H, int W, int kh, int kw,
+                                  int stride, int pad, float *K);
+void oracle_relu(float *v, size_t count);
+void oracle_quantize_k(const float *v, size_t count, int k, int8_t *L);
+void oracle_scale_output_k(const int32_t *acc, int k, const float *K, const float *alpha,
+                           const float *residual, int N, int Co, int Ho, int Wo, float *out);
+
+void oracle_xnor_block_ex(const float *x, const float *bn_scale, const float *bn_shift,
+                          const float *w, const float *residual, int N, int C, int H,
+                          int W, int Co, int kh, int kw, int stride, int pad, int kbits,
+                          int relu, int k_valid_taps, float *y, int8_t *Hs, float *A,
+                          float *K, int8_t *B, float *alpha, int32_t *acc, float *out) {
+  const int Ho = out_extent(H, kh, stride, pad), Wo = out_extent(W, kw, stride, pad);
+  oracle_bn_affine(x, bn_scale, bn_shift, N, C, H, W, y);
+  if (kbits == 1) oracle_sign(y, (size_t)N * C * H * W, Hs);
+  else oracle_quantize_k(y, (size_t)N * C * H * W, kbits, Hs);
+  oracle_channel_abs_mean(y, N, C, H, W, A);
+  if (k_valid_taps) oracle_box_filter_valid_taps(A, N, H, W, kh, kw, stride, pad, K);
+  else oracle_box_filter(A, N, H, W, kh, kw, stride, pad, K);
+  oracle_binarize_weights(w, Co, C, kh, kw, B, alpha);
+  oracle_binconv_acc(Hs, B, N, C, H, W, Co, kh, kw, stride, pad, acc);
+  if (kbits == 1) oracle_scale_output(acc, K, alpha, residual, N, Co, Ho, Wo, out);
+  else oracle_scale_output_k(acc, kbits, K, alpha, residual, N, Co, Ho, Wo, out);
+  if (relu) oracle_relu(out, (size_t)N * Co * Ho * Wo);
+}
+
 /* Full-precision 1x1 strided convolution without bias: the projection
  * shortcut ("type B") of the ResNet-18 variant in Section 4.2.  Plain
  * definition, double accumulation. */
@@ -235,6 +272,137 @@ void oracle_maxpool2d(const float *x, int N, int C, int H, int W, int k, int str
               if (first || v > m) { m = v; first = 0; }
             }
           out[(((size_t)n * C + c) * Ho + oy) * Wo + ox] = m;
+        }
+}
+
+/* Variant of the box filter for the border: the paper writes K = A * k without
+ * saying how A is padded.  The main reading (oracle_box_filter) pads with zeros
+ * and always divides by kh*kw.  This one averages over the taps that lie
+ * inside the image only (divisor = their number), so that K is the mean of |I|
+ * over exactly the input values the window sees; in the interior the two agree. */
+void oracle_box_filter_valid_taps(const float *A, int N, int H, int W, int kh, int kw,
+                                  int stride, int pad, float *K) {
+  const int Ho = out_extent(H, kh, stride, pad), Wo = out_extent(W, kw, stride, pad);
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int oy = 0; oy < Ho; ++oy)
+      for (int ox = 0; ox < Wo; ++ox) {
+        double s = 0.0;
+        int count = 0;
+        for (int ky = 0; ky < kh; ++ky)
+          for (int kx = 0; kx < kw; ++kx) {
+            const int iy = oy * stride + ky - pad, ix = ox * stride + kx - pad;
+            if (iy < 0 || iy >= H || ix < 0 || ix >= W) continue;
+            s += (double)A[((size_t)n * H + iy) * W + ix];
+            ++count;
+          }
+        /* a window wholly inside the padding sees nothing: K = 0 there */
+        K[((size_t)n * Ho + oy) * Wo + ox] = count ? (float)(s / (double)count) : 0.0f;
+      }
+}
+
+/* Section 3.2, "Training XNOR-Networks": a non-binary activation such as ReLU
+ * may follow the binary convolution.  Reading: it is applied to the value the
+ * block writes, i.e. after the scaling by K alpha and after the shortcut add
+ * where there is one.  In place on fp32 values (max with 0 is exact). */
+void oracle_relu(float *v, size_t count) {
+#pragma omp parallel for schedule(static)
+  for (size_t i = 0; i < count; ++i)
+    if (!(v[i] > 0.0f)) v[i] = (v[i] != v[i]) ? v[i] : 0.0f; /* NaN stays NaN */
+}
+
+/* Section 3.2, "k-bit Quantization": q_k(x) = 2([(2^k-1)(x+1)/2]/(2^k-1) - 1/2)
+ * replaces sign(); [.] rounds to the nearest integer and x lies in [-1, 1].
+ * The result is one of 2^k evenly spaced levels; written as an odd integer
+ * code L = 2 i - (2^k - 1), i = [.] in 0 .. 2^k - 1, the level is L/(2^k - 1).
+ * Readings: values outside [-1, 1] are clipped first; ties round up, which
+ * makes k = 1 the sign() of Eq. 4 (+1 at zero).  The rounding decision is
+ * taken in fp32, the precision of the data: [t] >= j exactly when
+ * x >= tau_j = (2j - 1)/(2^k - 1) - 1, and x is compared with tau_j rounded to
+ * float (tau_1 = 0 for k = 1).  1 <= k <= 7 (codes fit int8). */
+void oracle_quantize_k(const float *v, size_t count, int k, int8_t *L) {
+  const int levels = (1 << k) - 1; /* 2^k - 1 */
+#pragma omp parallel for schedule(static)
+  for (size_t i = 0; i < count; ++i) {
+    float x = v[i];
+    if (x > 1.0f) x = 1.0f;
+    if (x < -1.0f) x = -1.0f;
+    int idx = 0;
+    for (int j = 1; j <= levels; ++j) {
+      const float tau = (float)((double)(2 * j - 1) / (double)levels - 1.0);
+      if (x >= tau) idx = j;
+    }
+    L[i] = (int8_t)(2 * idx - levels);
+  }
+}
+
+/* Eq. 11 with q_k in place of sign(I): the integer sums of
+ * oracle_binconv_acc over level codes are sums of L * (+-1); dividing by
+ * 2^k - 1 turns codes into levels.  K, alpha and the residual as in
+ * oracle_scale_output. */
+void oracle_scale_output_k(const int32_t *acc, int k, const float *K, const float *alpha,
+                           const float *residual, int N, int Co, int Ho, int Wo,
+                           float *out) {
+  const size_t hw = (size_t)Ho * Wo;
+  const double levels = (double)((1 << k) - 1);
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < Co; ++co)
+      for (size_t i = 0; i < hw; ++i) {
+        const size_t o = ((size_t)n * Co + co) * hw + i;
+        double v = (double)acc[o] / levels * (double)K[(size_t)n * hw + i] * (double)alpha[co];
+        if (residual) v += (double)residual[o];
+        out[o] = (float)v;
+      }
+}
+
+/* Rounds fp32 values to bfloat16 (8 significand bits, round to nearest, ties
+ * to even) and returns them as fp32: the activation format of the
+ * Binary-Weight-Network convolution below.  Written on the bit pattern:
+ * keep the upper 16 bits, round on the lower 16.  NaN and infinity pass. */
+void oracle_round_bf16(const float *v, size_t count, float *r) {
+  for (size_t i = 0; i < count; ++i) {
+    union { float f; uint32_t u; } a;
+    a.f = v[i];
+    if ((a.u & 0x7F800000u) != 0x7F800000u) {
+      const uint32_t lower = a.u & 0xFFFFu, upper = a.u >> 16;
+      uint32_t up = upper;
+      if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u))) up = upper + 1u;
+      a.u = up << 16;
+    }
+    r[i] = a.f;
+  }
+}
+
+/* Binary-Weight-Network convolution, Section 3.1, Eq. 1:
+ * I * W ~ (I (+) B) alpha, where (+) is a convolution that only adds and
+ * subtracts the real-valued inputs according to B = sign(W), and alpha is the
+ * filter's scale (Eq. 6).  x holds the real inputs (the caller rounds them to
+ * the format the convolution consumes), B and alpha come from
+ * oracle_binarize_weights.  Zero padding; residual (nullable) added last. */
+void oracle_bwn_conv(const float *x, const int8_t *B, const float *alpha,
+                     const float *residual, int N, int C, int H, int W, int Co, int kh,
+                     int kw, int stride, int pad, float *out) {
+  const int Ho = out_extent(H, kh, stride, pad), Wo = out_extent(W, kw, stride, pad);
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < Co; ++co)
+      for (int oy = 0; oy < Ho; ++oy)
+        for (int ox = 0; ox < Wo; ++ox) {
+          double s = 0.0;
+          for (int c = 0; c < C; ++c)
+            for (int ky = 0; ky < kh; ++ky)
+              for (int kx = 0; kx < kw; ++kx) {
+                const int iy = oy * stride + ky - pad, ix = ox * stride + kx - pad;
+                if (iy < 0 || iy >= H || ix < 0 || ix >= W) continue;
+                const double xv = (double)x[(((size_t)n * C + c) * H + iy) * W + ix];
+                if (B[(((size_t)co * C + c) * kh + ky) * kw + kx] > 0) s += xv;
+                else s -= xv;
+              }
+          const size_t o = (((size_t)n * Co + co) * Ho + oy) * Wo + ox;
+          double v = s * (double)alpha[co];
+          if (residual) v += (double)residual[o];
+          out[o] = (float)v;
         }
 }
 
