@@ -51,12 +51,28 @@ typedef enum {
 } xnor_status;
 
 /* Geometry of one convolution layer.  Square or rectangular filters, one
- * stride and one zero-padding amount for both axes, no groups, no dilation. */
+ * stride and one zero-padding amount for both axes, no groups, no dilation.
+ * `flags` selects two options the paper mentions around the block (Section
+ * 3.2, "Training XNOR-Networks"); 0 is the block as Eq. 11 states it, and a
+ * descriptor initialised with nine values (C aggregate initialisation) has
+ * flags = 0.  Unknown bits give INVALID_ARG. */
 typedef struct {
   int N, C_in, H, W;
   int C_out, k_h, k_w;
   int stride, pad;
+  int flags;
 } xnor_conv_desc;
+
+/* "We can insert a non-binary activation (e.g. ReLU) after binary
+ * convolution": the BinConv calls write max(v, 0) instead of v, where v is the
+ * value after the K alpha scaling and after the shortcut add, if any (NaN
+ * gives 0).  Ignored by the BinActiv calls. */
+#define XNOR_FLAG_RELU 1
+/* Border variant of K = A * k: the box filter divides by the number of taps
+ * that lie inside the image instead of k_h*k_w, so K is the mean of A over the
+ * input values the window really sees (0 for a window wholly in the padding).
+ * Read by the BinActiv calls (they make K); ignored by the BinConv calls. */
+#define XNOR_FLAG_K_VALID_TAPS 2
 
 /* Library version: major*10000 + minor*100 + patch. */
 int xnor_version(void);
@@ -108,10 +124,14 @@ xnor_status xnor_binarize_weights(const float *w, int C_out, int C_in, int k_h, 
  *                                           K kernel reads, so it must not be NULL
  *   K         out  fp32 [N][H_out][W_out]   box filter of zero-padded A at the
  *                                           convolution's own output positions, divisor
- *                                           always k_h*k_w
+ *                                           always k_h*k_w (XNOR_FLAG_K_VALID_TAPS:
+ *                                           the number of in-image taps)
  *
  * INVALID_ARG: null/misaligned pointer (bn_* may both be NULL, not just one),
  * non-positive size, stride < 1, pad < 0, filter larger than the padded image.
+ * UNSUPPORTED (checked before anything is launched): N > 65535; C_in > 2976
+ * with a BatchNorm affine or C_in > 8960 without (the packed words of a group
+ * of pixels are staged in shared memory).
  */
 xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn_shift,
                           const xnor_conv_desc *d, uint32_t *x_packed, float *A, float *K,
@@ -166,13 +186,49 @@ xnor_status xnor_binactiv_static(const float *x, const float *bn_scale, const fl
  *                  sign(I) (*) sign(W) (sum over in-image taps of +-1 products), for
  *                  verification
  *
+ * d->flags & XNOR_FLAG_RELU: out = max(., 0) of the above (after the residual add).
+ *
  * INVALID_ARG as above.  UNSUPPORTED: k_h or k_w > 11, C_in*k_h*k_w >= 2^24
- * (the integer result must be exact in fp32).
+ * (the integer result must be exact in fp32), or a shape no engine covers
+ * (strides above 2 with an input patch larger than the CUDA-core kernel's
+ * shared memory).
  */
 xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_packed,
                                 const float *alpha, const float *K, const float *residual,
                                 const xnor_conv_desc *d, float *out, int32_t *acc_out,
                                 void *cuda_stream);
+
+/*
+ * k-bit activations -- Section 3.2, "k-bit Quantization": the block with
+ *   q_k(y) = 2([(2^k - 1)(y + 1)/2]/(2^k - 1) - 1/2)
+ * in place of sign(y); [.] rounds to the nearest integer, y in [-1, 1].  Everything
+ * else of the block (A, K, alpha, Eq. 11's scaling) stays as it is.
+ * Readings where the paper is silent: y outside [-1, 1] is clipped; ties round up,
+ * which makes k = 1 exactly sign() (+1 at zero); the rounding decision is a
+ * comparison in fp32: [.] >= j exactly when y >= fp32((2j - 1)/(2^k - 1) - 1).
+ *
+ * xnor_binactiv_kbit is xnor_binactiv with
+ *   x_planes  out  u32 [kbits][N][H][W][Cw]   plane p holds bit p of the index
+ *                  i = [.] in 0 .. 2^k - 1 of every value (the level is
+ *                  (2i - (2^k - 1))/(2^k - 1) = sum_p 2^p (2 b_p - 1) / (2^k - 1));
+ *                  for kbits = 1 the one plane is xnor_binactiv's x_packed.
+ * xnor_conv2d_forward_kbit is xnor_conv2d_forward on those planes:
+ *   out = (q_k(I) (*) sign(W)) (.) K alpha (+ residual), one pass of the binary
+ *   convolution per plane, each adding D_p K alpha 2^p/(2^k - 1) to the output;
+ *   acc_out (nullable) receives the exact integer sum over level codes,
+ *   sum_p 2^p D_p = (2^k - 1) (q_k(I) (*) sign(W)).
+ * 1 <= kbits <= 7 (INVALID_ARG otherwise); other errors as for the 1-bit calls;
+ * for kbits > 1 the convolution needs N*H*W*Cw to be a multiple of 4 (planes
+ * stay 16-byte aligned; UNSUPPORTED otherwise) and, with a residual that is not
+ * `out` itself, reads it in the first pass only.
+ */
+xnor_status xnor_binactiv_kbit(const float *x, const float *bn_scale, const float *bn_shift,
+                               const xnor_conv_desc *d, int kbits, uint32_t *x_planes, float *A,
+                               float *K, void *cuda_stream);
+xnor_status xnor_conv2d_forward_kbit(const uint32_t *x_planes, int kbits, const uint32_t *w_packed,
+                                     const float *alpha, const float *K, const float *residual,
+                                     const xnor_conv_desc *d, float *out, int32_t *acc_out,
+                                     void *cuda_stream);
 
 /*
  * Full-precision 1x1 strided convolution without bias: the projection
@@ -235,9 +291,13 @@ xnor_status xnor_maxpool2d(const float *x, int N, int C, int H, int W, int k, in
 /*
  * Which BinConv engine xnor_conv2d_forward uses.  XNOR_ENGINE_AUTO (default)
  * picks by shape: the tensor-core engine where it applies, else the CUDA-core
- * one.  Process-wide; meant for tests and measurements.  With an engine
- * forced, xnor_conv2d_forward returns UNSUPPORTED for shapes that engine does
- * not cover.
+ * one.  Meant for tests and measurements.  This is the library's only
+ * process-wide setting: an atomic that every BinConv call reads once at its
+ * start, so a call uses one engine throughout and a change made by another
+ * thread applies to the calls that start after it; a program that wants
+ * different engines in different threads must order those calls itself.
+ * With an engine forced, xnor_conv2d_forward returns UNSUPPORTED for shapes
+ * that engine does not cover.
  *   XNOR_ENGINE_POPC   CUDA-core XOR + population count, any supported shape
  *   XNOR_ENGINE_UMMA   5th-generation tensor cores (tcgen05), 4-bit (e2m1)
  *                      operands built from the sign bits, exact fp32

@@ -19,6 +19,9 @@ XNOR_ERR_UNSUPPORTED = 2
 XNOR_ERR_CUDA = 3
 XNOR_ERR_TIMEOUT = 4
 
+XNOR_FLAG_RELU = 1
+XNOR_FLAG_K_VALID_TAPS = 2
+
 XNOR_ENGINE_AUTO = 0
 XNOR_ENGINE_POPC = 1
 XNOR_ENGINE_UMMA = 2
@@ -32,12 +35,13 @@ EXPORTS = [
     "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
     "xnor_maxpool2d", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
+    "xnor_binactiv_kbit", "xnor_conv2d_forward_kbit",
 ]
 
 
 class xnor_conv_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
-                ("N", "C_in", "H", "W", "C_out", "k_h", "k_w", "stride", "pad")]
+                ("N", "C_in", "H", "W", "C_out", "k_h", "k_w", "stride", "pad", "flags")]
 
 
 class XnorError(RuntimeError):
@@ -93,6 +97,11 @@ def load():
     lib.xnor_maxpool2d.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
     lib.xnor_selftest_wait_timeout.restype = ci
     lib.xnor_selftest_wait_timeout.argtypes = [vp]
+    lib.xnor_binactiv_kbit.restype = ci
+    lib.xnor_binactiv_kbit.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), ci, vp, vp, vp, vp]
+    lib.xnor_conv2d_forward_kbit.restype = ci
+    lib.xnor_conv2d_forward_kbit.argtypes = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc),
+                                             vp, vp, vp]
     _lib = lib
     return lib
 
@@ -120,13 +129,13 @@ def _check(status, where):
         raise XnorError(status, where)
 
 
-def make_desc(N, C_in, H, W, C_out, k_h, k_w, stride, pad):
-    return xnor_conv_desc(N, C_in, H, W, C_out, k_h, k_w, stride, pad)
+def make_desc(N, C_in, H, W, C_out, k_h, k_w, stride, pad, flags=0):
+    return xnor_conv_desc(N, C_in, H, W, C_out, k_h, k_w, stride, pad, flags)
 
 
 def desc_of(s):
     """xnor_conv_desc of a workloads.ConvShape."""
-    return xnor_conv_desc(s.N, s.C_in, s.H, s.W, s.C_out, s.k, s.k, s.stride, s.pad)
+    return xnor_conv_desc(s.N, s.C_in, s.H, s.W, s.C_out, s.k, s.k, s.stride, s.pad, 0)
 
 
 def xnor_version():
@@ -205,6 +214,23 @@ def xnor_binactiv(x, bn_scale, bn_shift, d, x_packed, A, K, stream=None):
                                 _ptr(bn_shift, torch.float32), ctypes.byref(d),
                                 _ptr(x_packed, torch.int32), _ptr(A, torch.float32),
                                 _ptr(K, torch.float32), _stream(stream)), "xnor_binactiv")
+
+
+def xnor_binactiv_kbit(x, bn_scale, bn_shift, d, kbits, x_planes, A, K, stream=None):
+    _check(load().xnor_binactiv_kbit(_ptr(x, torch.float32), _ptr(bn_scale, torch.float32),
+                                     _ptr(bn_shift, torch.float32), ctypes.byref(d), int(kbits),
+                                     _ptr(x_planes, torch.int32), _ptr(A, torch.float32),
+                                     _ptr(K, torch.float32), _stream(stream)), "xnor_binactiv_kbit")
+
+
+def xnor_conv2d_forward_kbit(x_planes, kbits, w_packed, alpha, K, residual, d, out, acc_out=None,
+                             stream=None):
+    _check(load().xnor_conv2d_forward_kbit(_ptr(x_planes, torch.int32), int(kbits),
+                                           _ptr(w_packed, torch.int32), _ptr(alpha, torch.float32),
+                                           _ptr(K, torch.float32), _ptr(residual, torch.float32),
+                                           ctypes.byref(d), _ptr(out, torch.float32),
+                                           _ptr(acc_out, torch.int32), _stream(stream)),
+           "xnor_conv2d_forward_kbit")
 
 
 BINACTIV_STATIC_MAX_PIXELS = 1 << 20

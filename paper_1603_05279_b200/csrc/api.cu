@@ -1,9 +1,16 @@
 // C-ABI entry points of libxnor: argument checks and dispatch.  No kernel code.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
 
-xnor_engine g_engine = XNOR_ENGINE_AUTO;
+// The one piece of process-wide state: which BinConv engine the calls use.  An atomic, read
+// once per call, so that a change from another thread is seen whole by the calls after it.
+std::atomic<int> g_engine_state{(int)XNOR_ENGINE_AUTO};
+inline xnor_engine current_engine() {
+  return (xnor_engine)g_engine_state.load(std::memory_order_relaxed);
+}
 
 inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 inline bool bad_ptr(const void *p) { return p == nullptr || misaligned(p); }
@@ -15,6 +22,7 @@ xnor_status check_desc(const xnor_conv_desc *d, bool need_cout) {
   if (need_cout && d->C_out <= 0) return XNOR_ERR_INVALID_ARG;
   if (d->stride < 1 || d->pad < 0) return XNOR_ERR_INVALID_ARG;
   if (d->k_h > d->H + 2 * d->pad || d->k_w > d->W + 2 * d->pad) return XNOR_ERR_INVALID_ARG;
+  if (d->flags & ~(XNOR_FLAG_RELU | XNOR_FLAG_K_VALID_TAPS)) return XNOR_ERR_INVALID_ARG;
   return XNOR_OK;
 }
 
@@ -47,11 +55,11 @@ int xnor_out_extent(int in, int k, int stride, int pad) {
 xnor_status xnor_set_engine(xnor_engine e) {
   if ((int)e < (int)XNOR_ENGINE_AUTO || (int)e > (int)XNOR_ENGINE_UMMA_PAIR_STREAM)
     return XNOR_ERR_INVALID_ARG;
-  g_engine = e;
+  g_engine_state.store((int)e, std::memory_order_relaxed);
   return XNOR_OK;
 }
 
-xnor_engine xnor_get_engine(void) { return g_engine; }
+xnor_engine xnor_get_engine(void) { return current_engine(); }
 
 xnor_status xnor_binarize_weights(const float *w, int C_out, int C_in, int k_h, int k_w,
                                   uint32_t *w_packed, float *alpha, void *cuda_stream) {
@@ -71,6 +79,7 @@ xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn
   if ((bn_scale == nullptr) != (bn_shift == nullptr)) return XNOR_ERR_INVALID_ARG;
   if (bn_scale && (misaligned(bn_scale) || misaligned(bn_shift))) return XNOR_ERR_INVALID_ARG;
   const xnor::ConvGeom g = xnor::make_geom(*d);
+  if (!xnor::binactiv_supported(g, bn_scale != nullptr)) return XNOR_ERR_UNSUPPORTED;
   return from_cuda(xnor::launch_binactiv(x, bn_scale, bn_shift, g, x_packed, A, K,
                                          (cudaStream_t)cuda_stream));
 }
@@ -86,14 +95,32 @@ xnor_status xnor_binactiv_static(const float *x, const float *bn_scale, const fl
   if ((unsigned long long)d->N * d->H * d->W > XNOR_BINACTIV_STATIC_MAX_PIXELS)
     return XNOR_ERR_UNSUPPORTED;
   const xnor::ConvGeom g = xnor::make_geom(*d);
+  if (!xnor::binactiv_supported(g, bn_scale != nullptr)) return XNOR_ERR_UNSUPPORTED;
   return from_cuda(xnor::launch_binactiv_static(x, bn_scale, bn_shift, g, x_packed, K,
                                                 (cudaStream_t)cuda_stream));
 }
 
-xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_packed,
-                                const float *alpha, const float *K, const float *residual,
-                                const xnor_conv_desc *d, float *out, int32_t *acc_out,
-                                void *cuda_stream) {
+namespace {
+
+xnor::TcVariant variant_of(xnor_engine e) {
+  if (e == XNOR_ENGINE_UMMA_STREAM) return xnor::kTcSingleStream;
+  if (e == XNOR_ENGINE_UMMA_SINGLE) return xnor::kTcSingle;
+  if (e == XNOR_ENGINE_UMMA_PAIR) return xnor::kTcPair;
+  if (e == XNOR_ENGINE_UMMA_PAIR_STREAM) return xnor::kTcPairStream;
+  return xnor::kTcAuto;
+}
+
+// Which engine runs shape g under engine choice e: 1 tensor cores, 0 CUDA cores, -1 neither.
+int pick_engine(const xnor::ConvGeom &g, xnor_engine e) {
+  const bool tc_ok = e != XNOR_ENGINE_POPC && xnor::umma_tc_supported(g, variant_of(e));
+  if (tc_ok) return 1;
+  if (e != XNOR_ENGINE_AUTO && e != XNOR_ENGINE_POPC) return -1;
+  return xnor::binconv_popc_supported(g) ? 0 : -1;
+}
+
+xnor_status check_conv_args(const uint32_t *x_packed, const uint32_t *w_packed, const float *alpha,
+                            const float *K, const float *residual, const xnor_conv_desc *d,
+                            const float *out, const int32_t *acc_out) {
   xnor_status s = check_desc(d, true);
   if (s != XNOR_OK) return s;
   if (bad_ptr(x_packed) || bad_ptr(w_packed) || bad_ptr(alpha) || bad_ptr(K) || bad_ptr(out))
@@ -102,43 +129,94 @@ xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_pack
     return XNOR_ERR_INVALID_ARG;
   if (d->k_h > 11 || d->k_w > 11) return XNOR_ERR_UNSUPPORTED;
   if ((long long)d->C_in * d->k_h * d->k_w >= (1LL << 24)) return XNOR_ERR_UNSUPPORTED;
+  return XNOR_OK;
+}
+
+xnor_status run_conv(int engine, xnor_engine choice, const uint32_t *x_packed,
+                     const uint32_t *w_packed, const float *alpha, const float *K,
+                     const float *residual, const xnor::ConvGeom &g, const xnor::EpiOpts &epi,
+                     float *out, int32_t *acc_out, cudaStream_t st) {
+  if (engine == 1)
+    return from_cuda(xnor::launch_binconv_tc(x_packed, w_packed, alpha, K, residual, g, epi, out,
+                                             acc_out, variant_of(choice), st));
+  return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, epi, out,
+                                             acc_out, st));
+}
+
+}  // namespace
+
+xnor_status xnor_conv2d_forward(const uint32_t *x_packed, const uint32_t *w_packed,
+                                const float *alpha, const float *K, const float *residual,
+                                const xnor_conv_desc *d, float *out, int32_t *acc_out,
+                                void *cuda_stream) {
+  xnor_status s = check_conv_args(x_packed, w_packed, alpha, K, residual, d, out, acc_out);
+  if (s != XNOR_OK) return s;
   const xnor::ConvGeom g = xnor::make_geom(*d);
-  const cudaStream_t st = (cudaStream_t)cuda_stream;
-  xnor::TcVariant variant = xnor::kTcAuto;
-  if (g_engine == XNOR_ENGINE_UMMA_STREAM) variant = xnor::kTcSingleStream;
-  else if (g_engine == XNOR_ENGINE_UMMA_SINGLE) variant = xnor::kTcSingle;
-  else if (g_engine == XNOR_ENGINE_UMMA_PAIR) variant = xnor::kTcPair;
-  else if (g_engine == XNOR_ENGINE_UMMA_PAIR_STREAM) variant = xnor::kTcPairStream;
-  const bool tc_ok = xnor::umma_tc_supported(g, variant);
-  if (g_engine != XNOR_ENGINE_AUTO && g_engine != XNOR_ENGINE_POPC && !tc_ok)
-    return XNOR_ERR_UNSUPPORTED;
-  if (g_engine != XNOR_ENGINE_POPC && tc_ok)
-    return from_cuda(xnor::launch_binconv_tc(x_packed, w_packed, alpha, K, residual, g, out,
-                                             acc_out, variant, st));
-  return from_cuda(xnor::launch_binconv_popc(x_packed, w_packed, alpha, K, residual, g, out,
-                                             acc_out, (cudaStream_t)cuda_stream));
+  const xnor_engine choice = current_engine();
+  const int engine = pick_engine(g, choice);
+  if (engine < 0) return XNOR_ERR_UNSUPPORTED;
+  return run_conv(engine, choice, x_packed, w_packed, alpha, K, residual, g, xnor::default_epi(g),
+                  out, acc_out, (cudaStream_t)cuda_stream);
+}
+
+xnor_status xnor_binactiv_kbit(const float *x, const float *bn_scale, const float *bn_shift,
+                               const xnor_conv_desc *d, int kbits, uint32_t *x_planes, float *A,
+                               float *K, void *cuda_stream) {
+  xnor_status s = check_desc(d, false);
+  if (s != XNOR_OK) return s;
+  if (kbits < 1 || kbits > 7) return XNOR_ERR_INVALID_ARG;
+  if (bad_ptr(x) || bad_ptr(x_planes) || bad_ptr(A) || bad_ptr(K)) return XNOR_ERR_INVALID_ARG;
+  if ((bn_scale == nullptr) != (bn_shift == nullptr)) return XNOR_ERR_INVALID_ARG;
+  if (bn_scale && (misaligned(bn_scale) || misaligned(bn_shift))) return XNOR_ERR_INVALID_ARG;
+  if (d->N > 65535) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_binactiv_kbit(x, bn_scale, bn_shift, xnor::make_geom(*d), kbits,
+                                              x_planes, A, K, (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_conv2d_forward_kbit(const uint32_t *x_planes, int kbits, const uint32_t *w_packed,
+                                     const float *alpha, const float *K, const float *residual,
+                                     const xnor_conv_desc *d, float *out, int32_t *acc_out,
+                                     void *cuda_stream) {
+  xnor_status s = check_conv_args(x_planes, w_packed, alpha, K, residual, d, out, acc_out);
+  if (s != XNOR_OK) return s;
+  if (kbits < 1 || kbits > 7) return XNOR_ERR_INVALID_ARG;
+  const size_t plane_words = (size_t)d->N * d->H * d->W * ((d->C_in + 31) / 32);
+  if (kbits > 1 && (plane_words & 3u)) return XNOR_ERR_UNSUPPORTED;   // planes stay 16-byte aligned
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  const xnor_engine choice = current_engine();
+  const int engine = pick_engine(g, choice);
+  if (engine < 0) return XNOR_ERR_UNSUPPORTED;
+  // One pass per bit plane: with index bits b_p the level code is sum_p 2^p (2 b_p - 1), so the
+  // sum over codes is sum_p 2^p (sum over plane p); pass p adds D_p K alpha 2^p / (2^k - 1) to
+  // what the passes before it wrote (the output is its own residual).
+  const double levels = (double)((1 << kbits) - 1);
+  for (int p = 0; p < kbits; ++p) {
+    xnor::EpiOpts epi = xnor::default_epi(g);
+    epi.relu = epi.relu && p == kbits - 1;
+    epi.out_scale = (float)((double)(1 << p) / levels);
+    epi.acc_shift = p;
+    epi.acc_accum = p > 0;
+    s = run_conv(engine, choice, x_planes + (size_t)p * plane_words, w_packed, alpha, K,
+                 p == 0 ? residual : out, g, epi, out, acc_out, (cudaStream_t)cuda_stream);
+    if (s != XNOR_OK) return s;
+  }
+  return XNOR_OK;
 }
 
 namespace {
 
-xnor::TcVariant current_variant() {
-  if (g_engine == XNOR_ENGINE_UMMA_STREAM) return xnor::kTcSingleStream;
-  if (g_engine == XNOR_ENGINE_UMMA_SINGLE) return xnor::kTcSingle;
-  if (g_engine == XNOR_ENGINE_UMMA_PAIR) return xnor::kTcPair;
-  if (g_engine == XNOR_ENGINE_UMMA_PAIR_STREAM) return xnor::kTcPairStream;
-  return xnor::kTcAuto;
-}
+xnor::TcVariant current_variant() { return variant_of(current_engine()); }
 
 bool good_desc(const xnor_conv_desc *d) {
   return d && d->N > 0 && d->C_in > 0 && d->H > 0 && d->W > 0 && d->C_out > 0 && d->k_h > 0 &&
          d->k_w > 0 && d->stride >= 1 && d->pad >= 0 && d->k_h <= d->H + 2 * d->pad &&
-         d->k_w <= d->W + 2 * d->pad;
+         d->k_w <= d->W + 2 * d->pad && !(d->flags & ~(XNOR_FLAG_RELU | XNOR_FLAG_K_VALID_TAPS));
 }
 
 }  // namespace
 
 int xnor_conv2d_binactiv_parts(const xnor_conv_desc *d) {
-  if (!good_desc(d) || g_engine == XNOR_ENGINE_POPC || d->k_h > 11 || d->k_w > 11 ||
+  if (!good_desc(d) || current_engine() == XNOR_ENGINE_POPC || d->k_h > 11 || d->k_w > 11 ||
       (long long)d->C_in * d->k_h * d->k_w >= (1LL << 24))
     return 0;
   return xnor::tc_fused_parts(xnor::make_geom(*d), current_variant());
@@ -168,6 +246,7 @@ xnor_status xnor_binactiv_finish(const float *A_parts, int parts, const xnor_con
                                  float *A, float *K, void *cuda_stream) {
   if (!good_desc(d_next) || parts < 1 || bad_ptr(A_parts) || bad_ptr(A) || bad_ptr(K))
     return XNOR_ERR_INVALID_ARG;
+  if (d_next->N > 65535) return XNOR_ERR_UNSUPPORTED;
   return from_cuda(xnor::launch_binactiv_finish(A_parts, parts, xnor::make_geom(*d_next), A, K,
                                                 (cudaStream_t)cuda_stream));
 }
@@ -179,6 +258,8 @@ xnor_status xnor_maxpool2d(const float *x, int N, int C, int H, int W, int k, in
       k > H + 2 * pad || k > W + 2 * pad)
     return XNOR_ERR_INVALID_ARG;
   if (k > 11) return XNOR_ERR_UNSUPPORTED;
+  if ((long long)((H + 2 * pad - k) / stride + 1) * ((W + 2 * pad - k) / stride + 1) >= (1ll << 30))
+    return XNOR_ERR_UNSUPPORTED;
   return from_cuda(xnor::launch_maxpool2d(x, N, C, H, W, k, stride, pad, relu != 0, out,
                                           (cudaStream_t)cuda_stream));
 }

@@ -113,6 +113,7 @@ binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scal
     float asum = 0.0f;
     for (int k = 0; k < nw; ++k) {
       asm volatile("cp.async.wait_group 1;" ::: "memory");   // the older of the two tiles landed
+      __syncwarp();                      // ... for every lane: a lane reads what other lanes copied
       const int cw = g + k * G;
       const int c0 = cw * 32;
       const float *t = my_stage + buf * kTileFloats + lane;
@@ -147,6 +148,7 @@ binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scal
       }
       asum += part;
       words[(pgl * kPix + lane) * Cw + cw] = word;
+      __syncwarp();                      // every lane is done reading the tile before it is refilled
       issue(fb, fk, buf); advance_fetch();                   // refill the tile just consumed
       buf ^= 1;
     }
@@ -189,7 +191,7 @@ binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scal
 template <int KS>
 __global__ void __launch_bounds__(256)
 box_filter_kernel(const float *__restrict__ A, int H, int W, int kh, int kw, int stride, int pad,
-                  int Ho, int Wo, float *__restrict__ K) {
+                  int Ho, int Wo, int valid_taps, float *__restrict__ K) {
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= Ho * Wo) return;
   const int oy = i / Wo, ox = i - oy * Wo;
@@ -216,26 +218,63 @@ box_filter_kernel(const float *__restrict__ A, int H, int W, int kh, int kw, int
       for (int kx = kx0; kx < kx1; ++kx) s += __ldg(row + kx);
     }
   }
-  K[(size_t)blockIdx.y * Ho * Wo + i] = s / (float)(kh * kw);
+  // divisor: k_h k_w (zero-padded A), or the number of taps inside the image
+  int div = kh * kw;
+  if (valid_taps) {
+    const int ny = min(kh, H - y0) - max(0, -y0), nx = min(kw, W - x0) - max(0, -x0);
+    div = (ny > 0 && nx > 0) ? ny * nx : 0;
+  }
+  K[(size_t)blockIdx.y * Ho * Wo + i] = div > 0 ? s / (float)div : 0.0f;
 }
 
 }  // namespace
 
 cudaError_t launch_box_filter(const float *A, const ConvGeom &g, float *K, cudaStream_t st);
 
+namespace {
+
+constexpr size_t kPackSmemMax = 100 * 1024;      // three blocks per SM
+
+struct PackPlan { int G, PG; size_t smem; };
+
+size_t pack_smem(int Cw, bool bn, int G, int PG) {
+  return (size_t)kWarps * kBufsPerWarp * kTileFloats * sizeof(float) +
+         (bn ? (size_t)Cw * 32 * sizeof(float2) : 0) + (size_t)PG * kPix * Cw * sizeof(uint32_t) +
+         (size_t)PG * G * kPix * sizeof(float);
+}
+
+// With enough pixel groups to fill the GPU every warp packs whole pixel groups on its own
+// (G = 1); otherwise, or when the staged words of eight pixel groups do not fit shared
+// memory (many channels), the channel words of a pixel group are spread over the warps.
+bool pack_plan(const ConvGeom &g, bool bn, PackPlan *pl) {
+  const long long total_pix = (long long)g.N * g.H * g.W;
+  const long long ngroups = (total_pix + kPix - 1) / kPix;
+  const int Gs = g.Cw < kWarps ? g.Cw : kWarps;
+  int G = ngroups >= 2048 ? 1 : Gs;
+  if (pack_smem(g.Cw, bn, G, kWarps / G) > kPackSmemMax) G = Gs;
+  pl->G = G;
+  pl->PG = kWarps / G;
+  pl->smem = pack_smem(g.Cw, bn, G, pl->PG);
+  return pl->smem <= kPackSmemMax;
+}
+
+}  // namespace
+
+// Shapes the BinActiv kernels cover: the staged words fit shared memory (C_in <= 2976 with a
+// BatchNorm affine, more without) and one grid row per image.
+bool binactiv_supported(const ConvGeom &g, bool has_bn) {
+  PackPlan pl;
+  return g.N <= 65535 && pack_plan(g, has_bn, &pl);
+}
+
 cudaError_t launch_binactiv(const float *x, const float *scale, const float *shift,
                             const ConvGeom &g, uint32_t *x_packed, float *A, float *K,
                             cudaStream_t st) {
   const long long total_pix = (long long)g.N * g.H * g.W;
-  // with enough pixel groups to fill the GPU every warp packs whole pixel groups on its own;
-  // otherwise the channel words of a pixel group are spread over the warps of a block
-  const long long ngroups = (total_pix + kPix - 1) / kPix;
-  const int G = ngroups >= 2048 ? 1 : (g.Cw < kWarps ? g.Cw : kWarps);
-  const int PG = kWarps / G;
-  const size_t smem = (size_t)kWarps * kBufsPerWarp * kTileFloats * sizeof(float) +
-                      (scale ? (size_t)g.Cw * 32 * sizeof(float2) : 0) +
-                      (size_t)PG * kPix * g.Cw * sizeof(uint32_t) +
-                      (size_t)PG * G * kPix * sizeof(float);
+  PackPlan pl;
+  if (g.N > 65535 || !pack_plan(g, scale != nullptr, &pl)) return cudaErrorInvalidValue;
+  const int G = pl.G, PG = pl.PG;
+  const size_t smem = pl.smem;
   static bool attr_flags[64] = {};
   bool &attr_set = attr_done_for_current_device(attr_flags);
   if (!attr_set) {
@@ -245,20 +284,11 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
                               (const void *)binactiv_pack_kernel<false, true>,
                               (const void *)binactiv_pack_kernel<false, false>};
     for (int i = 0; i < 4 && e == cudaSuccess; ++i)
-      e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPackSmemMax);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
     attr_set = true;
   }
-  if (smem > 100 * 1024) return cudaErrorInvalidValue;
-  int sms = 148;
-  {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-      (void)cudaGetLastError();
-      sms = 148;
-    }
-  }
+  const int sms = sm_count_of_current_device();
   const long long nbatches = ((total_pix + kPix - 1) / kPix + PG - 1) / PG;
   const unsigned grid = (unsigned)(nbatches < 3ll * sms ? nbatches : 3ll * sms);   // 3 blocks fit an SM
   const bool v16 = ((g.H * g.W) & 3) == 0;
@@ -276,8 +306,9 @@ cudaError_t launch_box_filter(const float *A, const ConvGeom &g, float *K, cudaS
   if (g.N > 65535) return cudaErrorInvalidValue;
   const dim3 kgrid((unsigned)((g.Ho * g.Wo + 255) / 256), (unsigned)g.N);
   const int ks = g.kh == g.kw ? g.kh : 0;
+  const int valid = (g.flags & XNOR_FLAG_K_VALID_TAPS) ? 1 : 0;
 #define XNOR_BOX(KS) box_filter_kernel<KS><<<kgrid, 256, 0, st>>>(A, g.H, g.W, g.kh, g.kw, g.stride, \
-                                                                g.pad, g.Ho, g.Wo, K)
+                                                                g.pad, g.Ho, g.Wo, valid, K)
   if (ks == 1) XNOR_BOX(1);
   else if (ks == 3) XNOR_BOX(3);
   else if (ks == 5) XNOR_BOX(5);
@@ -305,8 +336,81 @@ sum_parts_kernel(const float *__restrict__ parts, int nparts, size_t n, float C,
 cudaError_t launch_binactiv_finish(const float *A_part, int parts, const ConvGeom &g, float *A,
                                    float *K, cudaStream_t st) {
   const size_t n = (size_t)g.N * g.H * g.W;
-  const unsigned grid = (unsigned)std::min<size_t>((n + 255) / 256, 148 * 8);
+  const unsigned grid = (unsigned)std::min<size_t>((n + 255) / 256, (size_t)sm_count_of_current_device() * 8);
   sum_parts_kernel<<<grid, 256, 0, st>>>(A_part, parts, n, (float)g.C, A);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return launch_box_filter(A, g, K, st);
+}
+
+// ---------------------------------------------------------------------------
+// BinActiv with k-bit activations (Section 3.2, "k-bit Quantization"):
+//   q_k(x) = 2([(2^k - 1)(x + 1)/2]/(2^k - 1) - 1/2),  x in [-1, 1]
+// replaces sign().  With i = [.] in 0 .. 2^k - 1 the level is (2i - (2^k-1))/(2^k-1); the
+// kernel stores the index i as k bit planes (plane p, bit c % 32 of word c / 32 = bit p of i),
+// so that the level code is sum_p 2^p (2 b_p - 1): a weighted sum of k ordinary +-1 planes.
+// Values outside [-1, 1] are clipped; ties round up (k = 1 is then sign() with +1 at zero).
+// The rounding decision is a comparison in fp32: i >= j exactly when
+// y >= tau_j = fp32((2j - 1)/(2^k - 1) - 1).  A (and K) are those of the 1-bit block.
+namespace {
+
+__global__ void __launch_bounds__(256)
+binactiv_pack_kbit_kernel(const float *__restrict__ x, const float *__restrict__ scale,
+                          const float *__restrict__ shift, long long total_pix, int C, int HW, int Cw,
+                          int kbits, uint32_t *__restrict__ x_planes, float *__restrict__ A) {
+  __shared__ float tau[128];                 // tau[j], j = 1 .. 2^k - 1; tau[0] unused
+  const int levels = (1 << kbits) - 1;
+  for (int j = 1 + threadIdx.x; j <= levels; j += blockDim.x)
+    tau[j] = (float)((double)(2 * j - 1) / (double)levels - 1.0);
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const long long ngroups = (total_pix + 31) / 32;
+  const long long warp0 = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long grp = warp0; grp < ngroups; grp += nwarps) {
+    const long long gp = grp * 32 + lane;          // this lane's pixel
+    if (gp >= total_pix) continue;
+    const long long n = gp / HW;
+    const int p = (int)(gp - n * HW);
+    const float *src = x + (size_t)n * C * HW + p;
+    float asum = 0.0f;
+    for (int cw = 0; cw < Cw; ++cw) {
+      uint32_t words[7] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
+      float p0 = 0.0f, p1 = 0.0f;
+      const int c0 = cw * 32, nc = min(32, C - c0);
+      for (int j = 0; j < nc; ++j) {
+        float y = __ldg(src + (size_t)(c0 + j) * HW);
+        if (scale != nullptr) y = __fmaf_rn(__ldg(scale + c0 + j), y, __ldg(shift + c0 + j));
+        if (j & 1) p1 += fabsf(y); else p0 += fabsf(y);
+        // largest index whose decision point is <= y, by bisection over the sorted tau
+        int idx = 0;
+        for (int b = kbits - 1; b >= 0; --b) {
+          const int cand = idx + (1 << b);
+          if (y >= tau[cand]) idx = cand;
+        }
+#pragma unroll
+        for (int b = 0; b < 7; ++b)
+          if (b < kbits) words[b] |= (uint32_t)((idx >> b) & 1) << j;
+      }
+      asum += p0 + p1;
+#pragma unroll
+      for (int b = 0; b < 7; ++b)
+        if (b < kbits) x_planes[((size_t)b * total_pix + gp) * Cw + cw] = words[b];
+    }
+    A[gp] = asum / (float)C;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_binactiv_kbit(const float *x, const float *scale, const float *shift,
+                                 const ConvGeom &g, int kbits, uint32_t *x_planes, float *A, float *K,
+                                 cudaStream_t st) {
+  const long long total_pix = (long long)g.N * g.H * g.W;
+  const long long nblocks = ((total_pix + 31) / 32 + 7) / 8;
+  const unsigned grid = (unsigned)std::min<long long>(nblocks, 8ll * sm_count_of_current_device());
+  binactiv_pack_kbit_kernel<<<grid, 256, 0, st>>>(x, scale, shift, total_pix, g.C, g.H * g.W, g.Cw,
+                                                  kbits, x_planes, A);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   return launch_box_filter(A, g, K, st);

@@ -24,7 +24,7 @@ struct PopcParams {
 __global__ void __launch_bounds__(kThreads)
 binconv_popc_kernel(const uint32_t *__restrict__ xp, const uint32_t *__restrict__ wp,
                     const float *__restrict__ alpha, const float *__restrict__ K,
-                    const float *residual, PopcParams P, float *out, int32_t *acc_out) {
+                    const float *residual, PopcParams P, EpiOpts epi, float *out, int32_t *acc_out) {
   extern __shared__ uint32_t smem[];
   const int taps = P.kh * P.kw;
   uint32_t *patch = smem;                       // [cwc][PP]
@@ -109,17 +109,31 @@ binconv_popc_kernel(const uint32_t *__restrict__ xp, const uint32_t *__restrict_
     const int acc = nvalid * P.C - 2 * pops[f];
     const size_t o = ((size_t)n * P.Co + co) * HoWo + op;
     float v = __fmul_rn(__fmul_rn((float)acc, kv), __ldg(alpha + co));
+    if (epi.out_scale != 1.0f) v = __fmul_rn(v, epi.out_scale);
     if (residual) v += residual[o];
+    if (epi.relu) v = fmaxf(v, 0.0f);
     out[o] = v;
-    if (acc_out) acc_out[o] = acc;
+    if (acc_out) acc_out[o] = (epi.acc_accum ? acc_out[o] : 0) + (acc << epi.acc_shift);
   }
 }
 
 }  // namespace
 
+// Shapes the CUDA-core engine covers: one channel word of the input patch and of the filter
+// tile must fit its 96 KB of shared memory.
+bool binconv_popc_supported(const ConvGeom &g) {
+  const long long PW = (long long)(g.Wo - 1) * g.stride + g.kw;
+  long long rows = (TP - 1 + g.Wo - 1) / g.Wo + 1;
+  if (rows > g.Ho) rows = g.Ho;
+  const long long PP = ((rows - 1) * g.stride + g.kh) * PW;
+  const long long words_per_cw = PP + (long long)TF * g.kh * g.kw;
+  return words_per_cw <= (long long)(96 * 1024 / sizeof(uint32_t)) &&
+         (long long)g.N * ((g.Ho * g.Wo + TP - 1) / TP) < (1ll << 31) && (g.Co + TF - 1) / TF <= 65535;
+}
+
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
-                                float *out, int32_t *acc_out, cudaStream_t st) {
+                                const EpiOpts &epi, float *out, int32_t *acc_out, cudaStream_t st) {
   PopcParams P;
   P.C = g.C; P.H = g.H; P.W = g.W; P.Co = g.Co; P.kh = g.kh; P.kw = g.kw;
   P.stride = g.stride; P.pad = g.pad; P.Ho = g.Ho; P.Wo = g.Wo; P.Cw = g.Cw;
@@ -148,7 +162,7 @@ cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const fl
     attr_set = true;
   }
   const dim3 grid((unsigned)(g.N * P.tiles_per_image), (unsigned)((g.Co + TF - 1) / TF));
-  binconv_popc_kernel<<<grid, kThreads, smem, st>>>(xp, wp, alpha, K, residual, P, out, acc_out);
+  binconv_popc_kernel<<<grid, kThreads, smem, st>>>(xp, wp, alpha, K, residual, P, epi, out, acc_out);
   return cudaGetLastError();
 }
 

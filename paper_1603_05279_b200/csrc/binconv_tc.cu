@@ -62,8 +62,6 @@
 //  otherwise the weights of every item pass through a ring of stages (items in
 //  tile-major order, so that a patch serves all slabs of its tile).
 #include <algorithm>
-#include <cstdio>
-#include <cstdlib>
 
 #include "common.cuh"
 #include "umma_common.cuh"
@@ -71,26 +69,6 @@
 namespace xnor {
 
 __device__ int g_status_tc = 0;
-#ifdef XNOR_TRACE
-#ifndef XNOR_TRACE_BLOCK
-#define XNOR_TRACE_BLOCK 1
-#endif
-// cycle totals of one warp per role of one CTA: [0..7] mma, [8..15] weights, [16..23] patch,
-// [24..31] epilogue
-__device__ long long g_tc_trace[64];
-// per CTA: clock at the start of the roles, at their end, SM id
-__device__ long long g_tc_cta[3 * 160];
-#define TR_DECL(first) long long tr_t = 0, tr_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}; \
-  const bool tr_on = blockIdx.x == XNOR_TRACE_BLOCK && (threadIdx.x & 31) == 0 && (first)
-#define TR_T0 do { if (tr_on) tr_t = clock64(); } while (0)
-#define TR_ADD(i) do { if (tr_on) { const long long n_ = clock64(); tr_a[(i) & 7] += n_ - tr_t; tr_t = n_; } } while (0)
-#define TR_FLUSH(base) do { if (tr_on) { for (int q_ = 0; q_ < 8; ++q_) g_tc_trace[(base) + q_] += tr_a[q_]; } } while (0)
-#else
-#define TR_DECL(first)
-#define TR_T0 do {} while (0)
-#define TR_ADD(i) do {} while (0)
-#define TR_FLUSH(base) do {} while (0)
-#endif
 
 namespace {
 
@@ -131,6 +109,9 @@ struct TcParams {
   const float *alpha, *K, *residual;
   float *out;
   int32_t *acc_out;
+  int relu;                    // max(v, 0) on every stored value
+  float out_scale;             // extra factor of D K alpha (1 unless several calls build one output)
+  int acc_shift, acc_accum;    // acc_out receives D << acc_shift, stored or added to its content
   int N, C, H, W, Co, kh, kw, stride, pad, Ho, Wo, Cw;
   int Hq, Wq, leadY, leadX;    // stream geometry of every phase plane
   int dymin, dxmin;
@@ -380,20 +361,16 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
   int tile = kRes ? (int)(i0 % P.ntiles) : 0;
   bool ok = true, new_tile = true;
   uint32_t patch_lo = 0;                 // patch address in descriptor units
-  TR_DECL(true);
-  TR_T0;
   const uint32_t nitems = (uint32_t)(i1 - i0);
   for (uint32_t it = 0; it < nitems && ok; ++it) {
     if (new_tile) {
       ok = mbar_wait_warp(S.pfull + 8u * pb, pph, S.abort_flag);
-      TR_ADD(0);
       if (!ok) break;
       patch_lo = ((S.patch + (uint32_t)pb * P.patch_bytes) & 0x3FFFFu) >> 4;
     }
     const bool visit_first = !kRes || it == 0 || tile == 0;
     const bool visit_last = !kRes || it + 1 == nitems || tile + 1 == P.ntiles;
     ok = mbar_wait_warp(S.aempty + 8u * ab, aph, S.abort_flag);
-    TR_ADD(1);
     if (!ok) break;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.NT);
@@ -404,11 +381,9 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
       const uint32_t first = st == 0 ? 0u : 1u;     // the first MMA of an item overwrites
       if (visit_first) {
         ok = mbar_wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
-        TR_ADD(2);
         if (!ok) break;
         tc_fence_after();
       }
-      TR_ADD(3);
       if (nj == 4) issue_stage<4, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
       else if (nj == 2) issue_stage<2, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
       else if (nj == 8) issue_stage<8, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
@@ -418,9 +393,7 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
                             b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc, tmem_sf,
                             jj == 0 ? first : 1u, el);
       }
-      TR_ADD(4);
       if (visit_last) umma_commit_to<kPair>(S.wempty + 8u * ws, el);
-      TR_ADD(5);
       if (++ws == P.stages) { ws = 0; if (!kRes) wph ^= 1u; }
     }
     if (!ok) break;
@@ -440,9 +413,7 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
       if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
     }
     if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
-    TR_ADD(6);
   }
-  TR_FLUSH(0);
 }
 
 // ------------------------------------------------------------------ weight producers (8 warps)
@@ -500,8 +471,6 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
                                            : make_uint2(0u, 0u);
     }
   };
-  TR_DECL(wt < 32);
-  TR_T0;
 #pragma unroll
   for (int d = 0; d < kPrefetch; ++d) { fetch(pf[d], fc); advance(fc); }
   int ws = 0;
@@ -511,7 +480,6 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
 #pragma unroll 1
   while (cc.item < i1 && ok) {
     ok = mbar_wait_relaxed(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc, XNOR_SLEEP_WGT);
-    TR_ADD(0);
     if (!ok) break;
     const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + row_off;
     const int co = cc.slab * P.NT + row_co;
@@ -551,7 +519,6 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
         }
       }
     }
-    TR_ADD(1);
     fence_proxy_async();
     __syncwarp();
     if (lane == 0) { if (P.pair) mbar_arrive_cluster(S.wfull + 8u * ws, 0u); else mbar_arrive(S.wfull + 8u * ws); }
@@ -564,9 +531,7 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
       for (int u = 0; u < kUnits; ++u) pf[d][u] = pf[d + 1][u];
     fetch(pf[kPrefetch - 1], fc);
     advance(fc);
-    TR_ADD(2);
   }
-  TR_FLUSH(8);
   return ok;
 }
 
@@ -673,8 +638,6 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     for (; kc < nraw && sg + kc * nsub < npatches; ++kc)
       if (lane == 0) start_copy(sg + kc * nsub, rb0 + kc);
   }
-  TR_DECL(pw == 0);
-  TR_T0;
   uint32_t k = 0;
 #pragma unroll 1
   for (uint32_t seq = sg; seq < npatches && ok; seq += nsub, ++k) {
@@ -699,7 +662,6 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     if (!ok) break;
     ok = mbar_wait_relaxed(S.pempty + 8u * pb, (use & 1u) ^ 1u, S.abort_flag, &g_status_tc,
                            XNOR_SLEEP_PAT);
-    TR_ADD(0);
     if (!ok) break;
     const uint32_t patch = S.patch + pb * P.patch_bytes;
     const uint32_t m0 = ((uint32_t)tile * tmul + S.rank) * kTileM;
@@ -768,7 +730,6 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
         }
       }
     }
-    TR_ADD(1);
     fence_proxy_async();
     __syncwarp();
     if (lane == 0) {
@@ -784,7 +745,6 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
       for (int i = 0; i < (1 << 20) && !mbar_try(S.rawfull + 8u * (rb0 + c % nraw), (c / nraw) & 1u); ++i) {}
     }
   }
-  TR_FLUSH(16);
 }
 
 // ------------------------------------------------------------------ epilogue (4 warps)
@@ -810,7 +770,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t howo = (uint32_t)HoWo;
   // the fast store paths: offsets of 16 consecutive filters fit 32 bits, no integer output
-  const bool small = HoWo < ((size_t)1 << 27) && P.acc_out == nullptr;
+  const bool small = HoWo < ((size_t)1 << 27) && P.acc_out == nullptr && P.out_scale == 1.0f;
+  const bool relu = P.relu != 0;
   const bool plain = small && P.residual == nullptr, with_res = small && P.residual != nullptr;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tile, slab;
@@ -840,8 +801,6 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   Pix px = decode(tile);
   int ab = (int)(k0 % P.nacc);            // accumulator buffer of the next item and the parity
   uint32_t fph = (uint32_t)(k0 / P.nacc) & 1u;   // of its full barrier
-  TR_DECL(quarter == 0 && e == 0);
-  TR_T0;
   const uint32_t nitems = (uint32_t)(i1 - i0);
   for (uint32_t it = 0; it < nitems && ok; ++it) {
     const bool valid = px.valid;
@@ -868,9 +827,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         rp += HoWo;
       }
     }
-    TR_ADD(0);
     ok = mbar_wait_relaxed(S.afull + 8u * ab, fph, S.abort_flag, &g_status_tc, XNOR_SLEEP_EPI);
-    TR_ADD(1);
     if (!ok) break;
     tc_fence_after();
     const uint32_t t_acc = t_lane + (uint32_t)(ab * P.NT);
@@ -894,8 +851,10 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
           const float a4[4] = {al[j4].x, al[j4].y, al[j4].z, al[j4].w};
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj)
-            op[(uint32_t)(j4 * 4 + jj) * howo] =
-                __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
+          {
+            const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
+            op[(uint32_t)(j4 * 4 + jj) * howo] = relu ? fmaxf(v, 0.0f) : v;
+          }
         }
       } else if (co + 16 <= P.Co && with_res) {
         const float *rp = P.residual + obase + (size_t)co * HoWo;
@@ -908,7 +867,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
           const float a4[4] = {al.x, al.y, al.z, al.w};
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
-            *op = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]) + res[j4 * 4 + jj];
+            const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]) + res[j4 * 4 + jj];
+            *op = relu ? fmaxf(v, 0.0f) : v;
             op += HoWo;
           }
         }
@@ -925,9 +885,14 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
           if (co + j < P.Co) {
             const float d = __int_as_float(r[j]);
             float v = __fmul_rn(__fmul_rn(d, kv), __ldg(P.alpha + co + j));
+            if (P.out_scale != 1.0f) v = __fmul_rn(v, P.out_scale);
             if (P.residual) v += res[j];
+            if (relu) v = fmaxf(v, 0.0f);
             P.out[o0 + (size_t)j * HoWo] = v;
-            if (P.acc_out) P.acc_out[o0 + (size_t)j * HoWo] = __float2int_rn(d);
+            if (P.acc_out) {
+              int32_t *ap = P.acc_out + o0 + (size_t)j * HoWo;
+              *ap = (P.acc_accum ? *ap : 0) + (__float2int_rn(d) << P.acc_shift);
+            }
           }
         }
       }
@@ -964,6 +929,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
           const int j = j4 * 4 + jj;
           float v = __fmul_rn(__fmul_rn(__int_as_float(r[j]), kv), a4[jj]);
           if (P.residual != nullptr) v += res[j];
+          if (relu) v = fmaxf(v, 0.0f);
           if (P.out != nullptr) op[(uint32_t)j * howo] = v;
           const float y = P.nscale != nullptr ? __fmaf_rn(s4[jj], v, h4[jj]) : v;
           half |= (y >= 0.0f ? 1u : 0u) << j;
@@ -1012,9 +978,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     tile = ntile;
     slab = nslab;
     if (++ab == P.nacc) { ab = 0; fph ^= 1u; }
-    TR_ADD(2);
   }
-  TR_FLUSH(24);
   return ok;
 }
 
@@ -1086,13 +1050,6 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   const unsigned unit = kPair ? blockIdx.x >> 1 : blockIdx.x, units = kPair ? gridDim.x >> 1 : gridDim.x;
   const long long i0 = total * unit / units;
   const long long i1 = total * (unit + 1) / units;
-#ifdef XNOR_TRACE
-  if (tid == 0 && blockIdx.x < 160) {
-    long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));
-    uint32_t sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_));
-    g_tc_cta[3 * blockIdx.x] = t_; g_tc_cta[3 * blockIdx.x + 2] = sm_;
-  }
-#endif
   if (i0 < i1) {
     const int wt = tid - 32 * kWgtWarp0;
     if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base); }
@@ -1123,12 +1080,6 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   }
   tc_fence_before();
   __syncthreads();
-#ifdef XNOR_TRACE
-  if (tid == 0 && blockIdx.x < 160) {
-    long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));
-    g_tc_cta[3 * blockIdx.x + 1] = t_;
-  }
-#endif
   // both CTAs of a pair are done with each other's barriers and tensor memory
   if (kPair) cluster_sync();
   if (warp == kMmaWarp) {
@@ -1300,19 +1251,6 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   return pl;
 }
 
-int sm_count_cached() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-      (void)cudaGetLastError();
-      n = 148;
-    }
-  }
-  return n;
-}
-
 }  // namespace
 
 namespace {
@@ -1379,7 +1317,7 @@ cudaError_t launch_plan(Plan &pl, cudaStream_t st, bool fuse) {
     attr_set = true;
   }
   const long long total = (long long)P.ntiles * P.nslabs;
-  const int sms = sm_count_cached();
+  const int sms = sm_count_of_current_device();
   // one CTA per SM, or one pair per two SMs
   const unsigned units = (unsigned)std::min<long long>(total, P.pair ? sms / 2 : sms);
   cudaError_t e_;
@@ -1390,12 +1328,7 @@ cudaError_t launch_plan(Plan &pl, cudaStream_t st, bool fuse) {
     if (P.pair) e_ = P.resident ? launch_variant<true, true, false>(pl, units, st) : launch_variant<false, true, false>(pl, units, st);
     else e_ = P.resident ? launch_variant<true, false, false>(pl, units, st) : launch_variant<false, false, false>(pl, units, st);
   }
-  if (e_ != cudaSuccess) {
-    (void)cudaGetLastError();
-    if (getenv("XNOR_DEBUG"))
-      fprintf(stderr, "binconv_tc launch: %s (units %u, pair %d, smem %zu)\n", cudaGetErrorString(e_),
-              units, P.pair, pl.smem);
-  }
+  if (e_ != cudaSuccess) (void)cudaGetLastError();
   return e_;
 }
 
@@ -1403,12 +1336,14 @@ cudaError_t launch_plan(Plan &pl, cudaStream_t st, bool fuse) {
 
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, TcVariant variant, cudaStream_t st) {
+                              const EpiOpts &epi, float *out, int32_t *acc_out, TcVariant variant,
+                              cudaStream_t st) {
   Plan pl = plan_variant(g, variant);
   if (!pl.ok) return cudaErrorInvalidValue;
   TcParams &P = pl.P;
   P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
   P.out = out; P.acc_out = acc_out;
+  P.relu = epi.relu; P.out_scale = epi.out_scale; P.acc_shift = epi.acc_shift; P.acc_accum = epi.acc_accum;
   P.nscale = nullptr; P.nshift = nullptr; P.xp_next = nullptr; P.A_part = nullptr; P.Cw_next = 0;
   return launch_plan(pl, st, false);
 }
@@ -1431,24 +1366,12 @@ cudaError_t launch_binconv_tc_fused(const uint32_t *xp, const uint32_t *wp, cons
   TcParams &P = pl.P;
   P.xp = xp; P.wp = wp; P.alpha = alpha; P.K = K; P.residual = residual;
   P.out = out; P.acc_out = nullptr;
+  P.relu = (g.flags & XNOR_FLAG_RELU) ? 1 : 0; P.out_scale = 1.0f; P.acc_shift = 0; P.acc_accum = 0;
   P.nscale = next_scale; P.nshift = next_shift; P.xp_next = xp_next; P.A_part = A_part;
   P.Cw_next = (g.Co + 31) / 32;
   return launch_plan(pl, st, true);
 }
 
-#ifdef XNOR_TRACE
-extern "C" int xnor_debug_trace_cta(long long *host480) {
-  return (int)cudaMemcpyFromSymbol(host480, g_tc_cta, sizeof(long long) * 480);
-}
-extern "C" int xnor_debug_trace_tc(long long *host64, int clear) {
-  cudaError_t e = cudaMemcpyFromSymbol(host64, g_tc_trace, sizeof(long long) * 64);
-  if (clear) {
-    long long z[64] = {};
-    cudaMemcpyToSymbol(g_tc_trace, z, sizeof(z));
-  }
-  return (int)e;
-}
-#endif
 
 namespace {
 

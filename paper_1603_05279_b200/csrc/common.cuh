@@ -9,7 +9,24 @@ namespace xnor {
 
 struct ConvGeom {
   int N, C, H, W, Co, kh, kw, stride, pad, Ho, Wo, Cw;
+  int flags;      // XNOR_FLAG_* of the descriptor
 };
+
+// What the BinConv epilogues do beyond Eq. 11's D K alpha (+ residual).
+struct EpiOpts {
+  int relu;          // max(v, 0) on the stored value
+  float out_scale;   // v = D K alpha out_scale (1: as Eq. 11; other values take the general path)
+  int acc_shift;     // acc_out receives D << acc_shift ...
+  int acc_accum;     // ... added to what acc_out holds (1) or stored (0)
+};
+inline EpiOpts default_epi(const ConvGeom &g) {
+  EpiOpts e;
+  e.relu = (g.flags & XNOR_FLAG_RELU) ? 1 : 0;
+  e.out_scale = 1.0f;
+  e.acc_shift = 0;
+  e.acc_accum = 0;
+  return e;
+}
 
 inline ConvGeom make_geom(const xnor_conv_desc &d) {
   ConvGeom g;
@@ -18,6 +35,7 @@ inline ConvGeom make_geom(const xnor_conv_desc &d) {
   g.Ho = (d.H + 2 * d.pad - d.k_h) / d.stride + 1;
   g.Wo = (d.W + 2 * d.pad - d.k_w) / d.stride + 1;
   g.Cw = (d.C_in + 31) / 32;
+  g.flags = d.flags;
   return g;
 }
 
@@ -40,15 +58,39 @@ size_t binactiv_static_max_pixels();
 cudaError_t launch_binactiv_static(const float *x, const float *scale, const float *shift,
                                    const ConvGeom &g, uint32_t *x_packed, float *K,
                                    cudaStream_t st);
+bool binactiv_supported(const ConvGeom &g, bool has_bn);
+// BinActiv with q_k in place of sign(): kbits planes of index bits, [kbits][N][H][W][Cw].
+cudaError_t launch_binactiv_kbit(const float *x, const float *scale, const float *shift,
+                                 const ConvGeom &g, int kbits, uint32_t *x_planes, float *A, float *K,
+                                 cudaStream_t st);
+bool binconv_popc_supported(const ConvGeom &g);
 cudaError_t launch_binconv_popc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                                 const float *K, const float *residual, const ConvGeom &g,
-                                float *out, int32_t *acc_out, cudaStream_t st);
+                                const EpiOpts &epi, float *out, int32_t *acc_out, cudaStream_t st);
 // Function attributes (dynamic shared-memory limits) belong to a device: a launcher sets them
 // once per device.  Returns the flag of the current device (out-of-range ids share the last).
 inline bool &attr_done_for_current_device(bool (&flags)[64]) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); dev = 0; }
   return flags[dev < 0 ? 0 : (dev > 63 ? 63 : dev)];
+}
+
+// Number of SMs of the current device, looked up once per device (persistent kernels size
+// their grids by it).  148 if the query fails.
+inline int sm_count_of_current_device() {
+  static int counts[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 148; }
+  const int slot = dev < 0 ? 0 : (dev > 63 ? 63 : dev);
+  if (counts[slot] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      n = 148;
+    }
+    counts[slot] = n;
+  }
+  return counts[slot];
 }
 
 // Persistent tensor-core engine (strides 1 and 2).  Variants: one CTA per SM or CTA pairs
@@ -58,7 +100,8 @@ enum TcVariant { kTcAuto = 0, kTcSingle, kTcSingleStream, kTcPair, kTcPairStream
 bool umma_tc_supported(const ConvGeom &g, TcVariant v);
 cudaError_t launch_binconv_tc(const uint32_t *xp, const uint32_t *wp, const float *alpha,
                               const float *K, const float *residual, const ConvGeom &g,
-                              float *out, int32_t *acc_out, TcVariant v, cudaStream_t st);
+                              const EpiOpts &epi, float *out, int32_t *acc_out, TcVariant v,
+                              cudaStream_t st);
 // BinConv with the next layer's BinActiv fused into its epilogue (sign bits packed along the
 // filters, partial sums of |y| per filter slab and epilogue warp); tc_fused_parts = number of
 // partial planes for the shape (0: the fused kernel does not cover it).

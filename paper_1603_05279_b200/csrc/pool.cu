@@ -55,12 +55,7 @@ cudaError_t launch_maxpool2d(const float *x, int N, int C, int H, int W, int k, 
   const int Ho = (H + 2 * pad - k) / stride + 1, Wo = (W + 2 * pad - k) / stride + 1;
   if ((long long)Ho * Wo >= (1ll << 30)) return cudaErrorInvalidValue;
   const long long total = (long long)N * C * Ho * Wo;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-    (void)cudaGetLastError();
-    sms = 148;
-  }
+  const int sms = sm_count_of_current_device();
   auto magic = [](uint32_t d) {
     Magic g;
     g.s = 0;

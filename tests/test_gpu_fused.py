@@ -10,7 +10,7 @@ import torch
 
 import paper_1603_05279_b200 as X
 from paper_1603_05279_b200 import binding as B
-from util import assert_close, dev, host, unpack_activations
+from util import GuardSet, assert_close, dev, host, unpack_activations
 
 pytestmark = pytest.mark.gpu
 
@@ -47,9 +47,10 @@ def _run(case, engine, with_out, with_bn):
         X.xnor_conv2d_forward(xp, wp, alpha, K, res, d, out_ref, None)
         parts = X.xnor_conv2d_binactiv_parts(d)
         assert parts >= 1, (case, engine)
-        xp2, A2, K2 = X.alloc_binactiv(d2)
-        A_parts = torch.empty((parts, N, Ho, Wo), dtype=torch.float32, device="cuda")
-        out = X.alloc_out(d) if with_out else None
+        gs = GuardSet()
+        xp2, A2, K2 = (gs.like(n, t) for n, t in zip(("x_packed_next", "A", "K"), X.alloc_binactiv(d2)))
+        A_parts = gs.new("A_parts", (parts, N, Ho, Wo))
+        out = gs.like("out", X.alloc_out(d)) if with_out else None
         X.xnor_conv2d_forward_binactiv(xp, wp, alpha, K, res, d, out,
                                        dev(scale) if with_bn else None, dev(shift) if with_bn else None,
                                        xp2, A_parts)
@@ -57,6 +58,7 @@ def _run(case, engine, with_out, with_bn):
     finally:
         X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
     X.xnor_check_device()
+    gs.check()
     return out_ref, out, xp2, A2, K2, scale, shift, (k2, s2, p2)
 
 

@@ -8,7 +8,7 @@ import torch
 import paper_1603_05279_b200 as X
 from paper_1603_05279_b200 import binding as B
 from paper_1603_05279_b200 import workloads as wl
-from util import REL_TOL, assert_close, dev, host, unpack_activations, unpack_weights
+from util import REL_TOL, GuardSet, assert_close, dev, host, unpack_activations, unpack_weights
 
 pytestmark = pytest.mark.gpu
 
@@ -28,10 +28,14 @@ def gpu_block(x, w, stride, pad, scale=None, shift=None, residual=None, engine=B
     N, C, H, W = x.shape
     Co, _, kh, kw = w.shape
     d = X.make_desc(N, C, H, W, Co, kh, kw, stride, pad)
-    wp, alpha = X.alloc_weights(Co, C, kh, kw)
-    xp, A, K = X.alloc_binactiv(d)
-    out = X.alloc_out(d)
-    acc = X.alloc_out(d, torch.int32)
+    # every output lies between guard words that must survive the calls
+    gs = GuardSet()
+    wp0, alpha0 = X.alloc_weights(Co, C, kh, kw)
+    xp0, A0, K0 = X.alloc_binactiv(d)
+    wp, alpha = gs.like("w_packed", wp0), gs.like("alpha", alpha0)
+    xp, A, K = gs.like("x_packed", xp0), gs.like("A", A0), gs.like("K", K0)
+    out = gs.like("out", X.alloc_out(d))
+    acc = gs.like("acc_out", X.alloc_out(d, torch.int32))
     X.xnor_binarize_weights(dev(w), wp, alpha)
     X.xnor_binactiv(dev(x), None if scale is None else dev(scale),
                     None if shift is None else dev(shift), d, xp, A, K)
@@ -48,7 +52,7 @@ def gpu_block(x, w, stride, pad, scale=None, shift=None, residual=None, engine=B
     finally:
         X.xnor_set_engine(B.XNOR_ENGINE_AUTO)
     X.xnor_check_device()
-    torch.cuda.synchronize()
+    gs.check()
     return dict(wp=host(wp), alpha=host(alpha), xp=host(xp), A=host(A), K=host(K),
                 out=host(out), acc=host(acc))
 

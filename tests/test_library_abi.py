@@ -85,6 +85,24 @@ def test_arguments_are_rejected_before_any_launch():
         B.XNOR_ERR_UNSUPPORTED
     assert lib.xnor_shortcut_conv1x1(p, null, 1, 4, 4, 4, 4, 2, p, null) == inv
     assert lib.xnor_shortcut_conv1x1(p, p, 1, 4, 4, 4, 4, 0, p, null) == inv
+    # option flags: unknown bits are an error
+    badflag = X.make_desc(1, 8, 5, 5, 4, 3, 3, 1, 1, 8)
+    assert lib.xnor_binactiv(p, null, null, ctypes.byref(badflag), p, p, p, null) == inv
+    assert lib.xnor_conv2d_forward(p, p, p, p, null, ctypes.byref(badflag), p, null, null) == inv
+    # shapes the BinActiv kernels do not cover are refused before any launch
+    wide = X.make_desc(1, 4000, 5, 5, 4, 3, 3, 1, 1)
+    assert lib.xnor_binactiv(p, p, p, ctypes.byref(wide), p, p, p, null) == B.XNOR_ERR_UNSUPPORTED
+    many = X.make_desc(70000, 8, 2, 2, 4, 1, 1, 1, 0)
+    assert lib.xnor_binactiv(p, null, null, ctypes.byref(many), p, p, p, null) == B.XNOR_ERR_UNSUPPORTED
+    # k-bit calls: the number of bits is checked, then the same rules as the 1-bit calls
+    for kb in (0, 8, -1):
+        assert lib.xnor_binactiv_kbit(p, null, null, ctypes.byref(d), kb, p, p, p, null) == inv
+        assert lib.xnor_conv2d_forward_kbit(p, kb, p, p, p, null, ctypes.byref(d), p, null, null) == inv
+    assert lib.xnor_binactiv_kbit(p, null, null, ctypes.byref(d), 2, null, p, p, null) == inv
+    assert lib.xnor_conv2d_forward_kbit(null, 2, p, p, p, null, ctypes.byref(d), p, null, null) == inv
+    odd_planes = X.make_desc(1, 8, 5, 5, 4, 3, 3, 1, 1)          # 25 words per plane: not 16-byte aligned
+    assert lib.xnor_conv2d_forward_kbit(p, 2, p, p, p, null, ctypes.byref(odd_planes), p, null, null) == \
+        B.XNOR_ERR_UNSUPPORTED
 
 
 def test_binding_refuses_host_tensors():

@@ -4,8 +4,9 @@ The ordinary xnor_binactiv wants a caller buffer for the A plane.  A caller that
 lives inside a fixed memory plan (or a plug-in that is handed only its inputs
 and outputs) has none to give, so this entry point keeps A in a fixed array
 inside the library.  These tests call it through the C ABI and compare it with
-xnor_binactiv on the same inputs, twice in a row with different shapes, so that
-what the first call leaves in the shared array is seen not to leak into the second.
+xnor_binactiv and with the CPU oracle on the same inputs, twice in a row with
+different shapes, so that what the first call leaves in the shared array is seen
+not to leak into the second; a last case fills the array to its last element.
 Collected last on purpose: a run that stops at the first failure has then
 already run every other test.
 """
@@ -17,7 +18,7 @@ import torch
 
 import paper_1603_05279_b200 as X
 from paper_1603_05279_b200 import binding as B
-from util import assert_close, dev, host
+from util import assert_close, dev, host, unpack_activations
 
 
 def _both(x, scale, shift, d):
@@ -31,7 +32,7 @@ def _both(x, scale, shift, d):
 
 
 @pytest.mark.gpu
-def test_static_scratch_matches_binactiv_on_two_calls_in_a_row():
+def test_static_scratch_matches_binactiv_on_two_calls_in_a_row(oracle):
     g = np.random.Generator(np.random.Philox(77))
     # first a larger problem, then a smaller one with another geometry: stale A values
     # of the first call lie beyond and between what the second call writes
@@ -44,6 +45,29 @@ def test_static_scratch_matches_binactiv_on_two_calls_in_a_row():
         assert np.array_equal(xp, xp_ref), "packed sign bits"
         assert_close(K, K_ref, "K")          # the tolerance every fp32 comparison here uses
         assert np.array_equal(K, K_ref)      # and in fact the same kernels: identical
+        # and against the oracle directly, not only through xnor_binactiv
+        y = oracle.bn_affine(x, scale, shift)
+        assert np.array_equal(unpack_activations(xp, C), oracle.sign(y).reshape(y.shape))
+        assert_close(K, oracle.box_filter(oracle.channel_abs_mean(y), k, k, s, p), "K against the oracle")
+
+
+@pytest.mark.gpu
+def test_static_scratch_at_exactly_its_capacity(oracle):
+    """N*H*W equal to the array's size: the last element of the array is used, and with this
+    many pixels the pack kernel runs in its one-warp-per-pixel-group mode."""
+    N, C, H, W = 256, 8, 64, 64
+    assert N * H * W == B.BINACTIV_STATIC_MAX_PIXELS
+    g = np.random.Generator(np.random.Philox(78))
+    x = g.standard_normal((N, C, H, W), dtype=np.float32)
+    scale = (1.0 + 0.1 * g.standard_normal(C)).astype(np.float32)
+    shift = (0.1 * g.standard_normal(C)).astype(np.float32)
+    d = X.make_desc(N, C, H, W, 8, 3, 3, 1, 1)
+    xp_ref, K_ref, xp, K = _both(x, scale, shift, d)
+    assert np.array_equal(xp, xp_ref) and np.array_equal(K, K_ref)
+    for n in (0, N - 1):                       # the last image's A sits at the end of the array
+        y = oracle.bn_affine(x[n:n + 1], scale, shift)
+        assert np.array_equal(unpack_activations(xp[n:n + 1], C), oracle.sign(y).reshape(y.shape))
+        assert_close(K[n:n + 1], oracle.box_filter(oracle.channel_abs_mean(y), 3, 3, 1, 1), "K")
 
 
 def test_static_scratch_rejects_sizes_beyond_its_array():
