@@ -88,7 +88,8 @@ using namespace umma;
 constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
 constexpr int kWgtWarp0 = 5, kWgtWarps = 8;
-constexpr int kPatWarp0 = 13, kPatWarps = 3;
+constexpr int kPatWarp0 = 13, kPatWarps = 3;               // warps 13-15 build patches; where a second
+constexpr int kMma2Warp = 15;                              // MMA issuer pays, warp 15 is that instead
 constexpr int kThreads = 32 * (kPatWarp0 + kPatWarps);     // 512: 16 warps, 128 registers each
 constexpr int kTileM = 128;          // stream positions per tile = tensor-memory lanes
 constexpr int kTmemCols = 512;
@@ -127,9 +128,12 @@ struct TcParams {
   uint32_t patch_bytes, stage_bytes;
   int rows_mod, grp_steps;     // weight-thread mapping (see weight producer)
   uint32_t off_ring, off_patch, off_raw;  // byte offsets in dynamic shared memory
+  uint32_t off_vec;            // per-filter vectors staged for the epilogue: alpha, then (fused)
+  int vec_len;                 // the next layer's scale and shift; vec_len floats each
   uint32_t raw_bytes;          // size of a raw buffer: the packed input rows a patch can touch
   int nraw;                    // raw buffers per subgroup of patch warps (1 or 2)
-  int pat_group;               // warps that build patches: 3, or 7 with four of the weight warps
+  int pat_base;                // dedicated patch warps: 3, or 2 when warp 15 is the second MMA issuer
+  int pat_group;               // warps that build patches: pat_base, or pat_base + 4 with four of the weight warps
   int pat_sub;                 // subgroups they form (each builds whole patches): 3 or 1
   int wgt_warps;               // warps that expand weights: 8, or 4
   uint32_t idesc;
@@ -252,6 +256,18 @@ __device__ __forceinline__ void expand_signs(uint32_t w, uint32_t v[4]) {
   v[3] = (w & 0x88888888u) ^ m3;
 }
 
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float lds_f(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+
 // Shift of a filter tap inside a phase plane, and the plane it reads.
 inline void tap_geometry(const TcParams &P, int tap, int &phase, int &shift) {
   const int ky = tap / P.kw, kx = tap - ky * P.kw;
@@ -290,11 +306,50 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m, int s) {
   return (uint32_t)(((uint64_t)n * m) >> (31 + s));
 }
 
+// Resident schedule: which pixel tiles a CTA (a pair) takes.  The U units of the grid are
+// split into one group per filter slab (so a CTA expands one slab, once); inside its group of
+// G units, unit g takes tiles g, g + G, g + 2G, ... of the slab: at any moment the CTAs of a
+// group write neighbouring runs of every output plane, so the lines that leave the L2
+// together lie together in memory (measured on 27x27 planes: 3.9 TB/s of stores against
+// 2.85 TB/s when every CTA owns a contiguous range of tiles).
+struct ResSched {
+  uint32_t ntiles, nslabs;
+  uint32_t slab, g, G;           // this unit's slab, its index in the slab's group, the group's size
+  __device__ __forceinline__ uint32_t first(uint32_t s) const { return g; }
+  __device__ __forceinline__ uint32_t step() const { return G; }
+  __device__ __forceinline__ uint32_t count(uint32_t s) const {
+    return (s == slab && g < ntiles) ? (ntiles - g + G - 1u) / G : 0u;
+  }
+  __device__ __forceinline__ uint32_t total() const { return count(slab); }
+  // the seq-th item of the unit (seq < total()): its slab and tile
+  __device__ __forceinline__ void item(uint32_t seq, uint32_t &sl, uint32_t &tile) const {
+    sl = slab;
+    tile = g + seq * G;
+  }
+};
+
+__device__ __forceinline__ ResSched res_sched(int ntiles, int nslabs, bool pair) {
+  ResSched R;
+  const uint32_t unit = pair ? blockIdx.x >> 1 : blockIdx.x;
+  const uint32_t units = pair ? gridDim.x >> 1 : gridDim.x;    // >= nslabs (host)
+  R.ntiles = (uint32_t)ntiles;
+  R.nslabs = (uint32_t)nslabs;
+  // group s = units [s U / nslabs, (s + 1) U / nslabs)
+  R.slab = unit * R.nslabs / units;
+  while ((R.slab + 1u) * units / R.nslabs <= unit) ++R.slab;
+  while (R.slab * units / R.nslabs > unit) --R.slab;
+  const uint32_t g0 = R.slab * units / R.nslabs;
+  R.g = unit - g0;
+  R.G = (R.slab + 1u) * units / R.nslabs - g0;
+  return R;
+}
+
 struct Smem {
   uint32_t wfull, wempty, pfull, pempty, afull, aempty, rawfull, rawdone;   // shared-space addresses of barrier arrays
   uint32_t *tmem_slot;
   volatile int *abort_flag;
   uint32_t ring, patch, raw;                              // shared-space byte addresses
+  uint32_t alpha, nscale, nshift;                         // staged per-filter vectors
   uint32_t rank;                                          // CTA rank in its pair (0 = issues the MMAs)
 };
 
@@ -315,6 +370,9 @@ __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
   s.ring = base + P.off_ring;
   s.patch = base + P.off_patch;
   s.raw = base + P.off_raw;
+  s.alpha = base + P.off_vec;
+  s.nscale = s.alpha + 4u * (uint32_t)P.vec_len;
+  s.nshift = s.nscale + 4u * (uint32_t)P.vec_len;
   s.rank = P.pair ? cluster_ctarank() : 0u;
   return s;
 }
@@ -339,11 +397,17 @@ __device__ __forceinline__ void issue_stage(const TcParams &P, int j0, uint32_t 
                       b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u, el);
 }
 
-// kRes: resident schedule.  The stage barriers are then waited for only on the first item of
-// a slab visit (the slab stays in shared memory afterwards) and released only on the last.
+// kRes: resident schedule.  The stage barriers are then waited for only before an issuer's
+// first item (the slab stays in shared memory afterwards) and never released.
+// Resident schedule: two warps issue (`which` = 0, 1 of `nissue` = 2), taking alternate items.
+// One warp issues an MMA of 128 x 128 x 64 every ~95 cycles (measured; ~105 beside busy
+// epilogue warps) while the tensor core needs 64: two issuers keep it fed.  Each item has its own
+// patch and accumulator buffer, and a CTA stays on one slab (no stage is ever released), so the
+// two streams of MMAs depend on nothing of each other.  Streaming: one issuer (the stages of the
+// weight ring are handed from item to item in order).
 template <bool kRes, bool kPair>
 __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long long i1,
-                         uint32_t tmem_base) {
+                         uint32_t tmem_base, uint32_t which, uint32_t nissue) {
   const uint32_t tmem_sf = tmem_base + (uint32_t)kSfCol;
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const uint32_t b_lbo = (uint32_t)P.NTh * 16u;
@@ -356,20 +420,29 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
   int ws = 0, pb = 0, ab = 0;
   uint32_t wph = 0, pph = 0;
   uint32_t aph = 1u;                     // parity to wait for on the accumulator's empty barrier
-  // streaming: item = tile * nslabs + slab; resident: item = slab * ntiles + tile
+  // streaming: items [i0, i1), item = tile * nslabs + slab; resident: the unit's own tiles of
+  // its slab (see ResSched), one patch per item
+  const ResSched R = res_sched(P.ntiles, P.nslabs, kPair);
   int slab = kRes ? 0 : (int)(i0 % P.nslabs);
-  int tile = kRes ? (int)(i0 % P.ntiles) : 0;
   bool ok = true, new_tile = true;
   uint32_t patch_lo = 0;                 // patch address in descriptor units
-  const uint32_t nitems = (uint32_t)(i1 - i0);
-  for (uint32_t it = 0; it < nitems && ok; ++it) {
+  const uint32_t nitems = kRes ? R.total() : (uint32_t)(i1 - i0);
+  for (uint32_t it = which; it < nitems && ok; it += nissue) {
+    if (kRes) {
+      // buffers and barrier phases of the it-th item of the CTA
+      pb = (int)(it % (uint32_t)P.npb);
+      pph = (it / (uint32_t)P.npb) & 1u;
+      ab = (int)(it % (uint32_t)P.nacc);
+      aph = ((it / (uint32_t)P.nacc) & 1u) ^ 1u;
+      ws = 0;
+    }
     if (new_tile) {
       ok = mbar_wait_warp(S.pfull + 8u * pb, pph, S.abort_flag);
       if (!ok) break;
       patch_lo = ((S.patch + (uint32_t)pb * P.patch_bytes) & 0x3FFFFu) >> 4;
     }
-    const bool visit_first = !kRes || it == 0 || tile == 0;
-    const bool visit_last = !kRes || it + 1 == nitems || tile + 1 == P.ntiles;
+    // resident: the slab is expanded once; an issuer waits for its stages before its first item
+    const bool wait_stages = !kRes || it == which;
     ok = mbar_wait_warp(S.aempty + 8u * ab, aph, S.abort_flag);
     if (!ok) break;
     tc_fence_after();
@@ -379,7 +452,7 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
       const int nj = min(P.mps, P.nsteps - j0);
       const uint32_t b_lo = b_lo0 + (uint32_t)ws * stage_step;
       const uint32_t first = st == 0 ? 0u : 1u;     // the first MMA of an item overwrites
-      if (visit_first) {
+      if (wait_stages) {
         ok = mbar_wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -393,17 +466,13 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
                             b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc, tmem_sf,
                             jj == 0 ? first : 1u, el);
       }
-      if (visit_last) umma_commit_to<kPair>(S.wempty + 8u * ws, el);
+      if (!kRes) umma_commit_to<kPair>(S.wempty + 8u * ws, el);
       if (++ws == P.stages) { ws = 0; if (!kRes) wph ^= 1u; }
     }
     if (!ok) break;
     if (kRes) {
-      // every item has its own patch; the barrier phase of the slab flips with the visit
-      if (visit_last) wph ^= 1u;
-      if (++tile == P.ntiles) tile = 0;
       umma_commit_to<kPair>(S.afull + 8u * ab, el);
       umma_commit_to<kPair>(S.pempty + 8u * pb, el);
-      if (++pb == P.npb) { pb = 0; pph ^= 1u; }
     } else {
       // next item: same tile (next slab) or the next tile
       new_tile = false;
@@ -411,8 +480,8 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
       umma_commit_to<kPair>(S.afull + 8u * ab, el);
       if (new_tile || it + 1 == nitems) umma_commit_to<kPair>(S.pempty + 8u * pb, el);
       if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
+      if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
     }
-    if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
   }
 }
 
@@ -566,10 +635,10 @@ __device__ __forceinline__ bool weight_dispatch(const TcParams &P, const Smem &S
 template <bool kRes>
 __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long long i1, int pw,
                            int lane) {
+  const ResSched R = res_sched(P.ntiles, P.nslabs, P.pair != 0);
   const int tile0 = kRes ? 0 : (int)(i0 / P.nslabs);
-  const uint32_t npatches = kRes ? (uint32_t)(i1 - i0)
+  const uint32_t npatches = kRes ? R.total()
                                  : (uint32_t)((i1 - 1) / P.nslabs) - (uint32_t)tile0 + 1u;
-  const uint32_t tile_r0 = kRes ? (uint32_t)(i0 % P.ntiles) : 0u;   // resident: tile of the first item
   const int s = P.stride, phases = s * s;
   const uint32_t plane_bytes = (uint32_t)P.ppix * 16u;
   const bool vec = (P.Cw & 3) == 0;
@@ -587,7 +656,10 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
   const int nunits = npass * phases * ngrp;
 
   auto tile_of = [&](uint32_t seq) {
-    return kRes ? (int)((tile_r0 + seq) % (uint32_t)P.ntiles) : tile0 + (int)seq;
+    if (!kRes) return tile0 + (int)seq;
+    uint32_t sl, t;
+    R.item(seq, sl, t);
+    return (int)t;
   };
   // input rows [g0, g1) (of the N*H rows of the tensor) that the patch of a tile reads
   auto row_range = [&](int tile, int &g0, int &g1) {
@@ -751,13 +823,16 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
 // Warp w reads tensor-memory lanes 32 w .. +31 (pixels), all the slab's columns (filters).
 // Lane = pixel, so for one filter a warp stores 32 consecutive stream pixels: a contiguous
 // run of the NCHW output row.
-// Drains items [i0, i1), the k0-th and following of the CTA.  Of every item this warp takes
+// Drains `nitems` items, the k0-th and following of the CTA: streaming, items i0, i0 + 1, ...
+// (item = tile * nslabs + slab); resident, tiles tile0, tile0 + tstep, ... of slab `slab0`.
+// Of every item this warp takes
 // the 16-column groups e, e + esplit, ... (esplit warps share a quarter of the lanes).
 // kFuse: the groups a warp takes come in pairs (32 consecutive filters = one packed word of the
 // next layer's input); see the fused emit below.
 template <bool kRes, bool kFuse>
-__device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, long long i1,
-                              long long k0, uint32_t tmem_base, int quarter, int e, int lane) {
+__device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, int slab0, int tile0,
+                              int tstep, uint32_t nitems, long long k0, uint32_t tmem_base,
+                              int quarter, int e, int lane) {
   const int b_end = P.NT / 16;
   const int esplit = kRes ? P.epi_split : 1;
   // the k-th group of this warp: groups e, e + esplit, ... or, fused, the two groups of the
@@ -775,7 +850,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   const bool plain = small && P.residual == nullptr, with_res = small && P.residual != nullptr;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tile, slab;
-  if (kRes) { slab = (int)(i0 / P.ntiles); tile = (int)(i0 - (long long)slab * P.ntiles); }
+  if (kRes) { slab = slab0; tile = tile0; }
   else { tile = (int)(i0 / P.nslabs); slab = (int)(i0 - (long long)tile * P.nslabs); }
   bool ok = true;
   // this lane's output pixel in a tile: whether it exists, its K, offset of (image, filter 0, pixel)
@@ -801,7 +876,6 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
   Pix px = decode(tile);
   int ab = (int)(k0 % P.nacc);            // accumulator buffer of the next item and the parity
   uint32_t fph = (uint32_t)(k0 / P.nacc) & 1u;   // of its full barrier
-  const uint32_t nitems = (uint32_t)(i1 - i0);
   for (uint32_t it = 0; it < nitems && ok; ++it) {
     const bool valid = px.valid;
     const float kv = px.kv;
@@ -812,7 +886,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
     bool next_new;
     if (kRes) {
       next_new = true;
-      if (++ntile == P.ntiles) { ntile = 0; ++nslab; }
+      ntile += tstep;
     } else {
       next_new = false;
       if (++nslab == P.nslabs) { nslab = 0; ++ntile; next_new = true; }
@@ -845,7 +919,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         float4 al[4];
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4)
-          al[j4] = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
+          al[j4] = lds_f4(S.alpha + (uint32_t)(co * 4 + j4 * 16));
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
           const float a4[4] = {al[j4].x, al[j4].y, al[j4].z, al[j4].w};
@@ -863,7 +937,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         for (int j = 0; j < 16; ++j) res[j] = rp[(size_t)j * HoWo];
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
-          const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
+          const float4 al = lds_f4(S.alpha + (uint32_t)(co * 4 + j4 * 16));
           const float a4[4] = {al.x, al.y, al.z, al.w};
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
@@ -884,7 +958,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
         for (int j = 0; j < 16; ++j) {
           if (co + j < P.Co) {
             const float d = __int_as_float(r[j]);
-            float v = __fmul_rn(__fmul_rn(d, kv), __ldg(P.alpha + co + j));
+            float v = __fmul_rn(__fmul_rn(d, kv), lds_f(S.alpha + (uint32_t)((co + j) * 4)));
             if (P.out_scale != 1.0f) v = __fmul_rn(v, P.out_scale);
             if (P.residual) v += res[j];
             if (relu) v = fmaxf(v, 0.0f);
@@ -916,11 +990,11 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, lo
       }
 #pragma unroll
       for (int j4 = 0; j4 < 4; ++j4) {
-        const float4 al = __ldg(reinterpret_cast<const float4 *>(P.alpha + co) + j4);
+        const float4 al = lds_f4(S.alpha + (uint32_t)(co * 4 + j4 * 16));
         float4 sc = make_float4(1.0f, 1.0f, 1.0f, 1.0f), sh = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         if (P.nscale != nullptr) {
-          sc = __ldg(reinterpret_cast<const float4 *>(P.nscale + co) + j4);
-          sh = __ldg(reinterpret_cast<const float4 *>(P.nshift + co) + j4);
+          sc = lds_f4(S.nscale + (uint32_t)(co * 4 + j4 * 16));
+          sh = lds_f4(S.nshift + (uint32_t)(co * 4 + j4 * 16));
         }
         const float a4[4] = {al.x, al.y, al.z, al.w};
         const float s4[4] = {sc.x, sc.y, sc.z, sc.w}, h4[4] = {sh.x, sh.y, sh.z, sh.w};
@@ -1012,6 +1086,15 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     *S.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // per-filter vectors of the epilogue, zero beyond C_out (one global round trip per CTA
+  // instead of one per 16 columns drained)
+  for (int i = tid; i < P.vec_len; i += kThreads) {
+    reinterpret_cast<float *>(smem + P.off_vec)[i] = i < P.Co ? __ldg(P.alpha + i) : 0.0f;
+    if (kFuse && P.nscale != nullptr) {
+      reinterpret_cast<float *>(smem + P.off_vec)[P.vec_len + i] = i < P.Co ? __ldg(P.nscale + i) : 0.0f;
+      reinterpret_cast<float *>(smem + P.off_vec)[2 * P.vec_len + i] = i < P.Co ? __ldg(P.nshift + i) : 0.0f;
+    }
+  }
   if (warp == kMmaWarp) {
     if (kPair) {
       // the same warp of both CTAs of the pair allocates, at the same shared-memory offset
@@ -1050,30 +1133,34 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   const unsigned unit = kPair ? blockIdx.x >> 1 : blockIdx.x, units = kPair ? gridDim.x >> 1 : gridDim.x;
   const long long i0 = total * unit / units;
   const long long i1 = total * (unit + 1) / units;
-  if (i0 < i1) {
+  const ResSched R = res_sched(P.ntiles, P.nslabs, kPair);
+  if (kRes ? R.total() > 0u : i0 < i1) {
     const int wt = tid - 32 * kWgtWarp0;
-    if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base); }
+    const uint32_t nissue = P.pat_base < kPatWarps ? 2u : 1u;
+    if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base, 0u, nissue); }
+    else if (warp == kMma2Warp && nissue == 2u) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base, 1u, 2u); }
     else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, warp - kPatWarp0, lane);
-    else if (kRes && P.pat_group > kPatWarps && warp >= kWgtWarp0 + 4)
-      patch_role<kRes>(P, S, i0, i1, kPatWarps + warp - (kWgtWarp0 + 4), lane);   // helpers
+    else if (kRes && P.pat_group > P.pat_base && warp >= kWgtWarp0 + 4)
+      patch_role<kRes>(P, S, i0, i1, P.pat_base + warp - (kWgtWarp0 + 4), lane);   // helpers
     else if (!kRes) {
-      if (warp < kEpiWarps) epilogue_role<false, kFuse>(P, S, i0, i1, 0, tmem_base, warp, 0, lane);
+      if (warp < kEpiWarps)
+        epilogue_role<false, kFuse>(P, S, i0, 0, 0, 0, (uint32_t)(i1 - i0), 0, tmem_base, warp, 0, lane);
       else weight_dispatch(P, S, i1 - i0, (int)(i0 % P.nslabs), 1u, wt, lane);
     } else {
       // Slab visits of this CTA in order.  The weight warps expand the slab, then every
       // worker warp drains its share of the visit's items.
       const bool wgt = warp >= kWgtWarp0;
       const int e = wgt ? 1 + (warp - kWgtWarp0) / 4 : 0;
-      long long it = i0;
-      uint32_t visit = 0;
+      uint32_t visit = 0, done = 0;
       bool ok = true;
-      while (it < i1 && ok) {
-        const int slab = (int)(it / P.ntiles);
-        const long long vend = min(i1, (long long)(slab + 1) * P.ntiles);
-        if (wgt) ok = weight_dispatch(P, S, 1, slab, (visit & 1u) ^ 1u, wt, lane);
+      for (uint32_t slab = 0; slab < R.nslabs && ok; ++slab) {
+        const uint32_t n = R.count(slab);
+        if (n == 0u) continue;
+        if (wgt) ok = weight_dispatch(P, S, 1, (int)slab, (visit & 1u) ^ 1u, wt, lane);
         if (ok && e < P.epi_split)
-          ok = epilogue_role<true, kFuse>(P, S, it, vend, it - i0, tmem_base, warp & 3, e, lane);
-        it = vend;
+          ok = epilogue_role<true, kFuse>(P, S, 0, (int)slab, (int)R.first(slab), (int)R.step(), n,
+                                          done, tmem_base, warp & 3, e, lane);
+        done += n;
         ++visit;
       }
     }
@@ -1159,15 +1246,20 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   P.nsteps = (P.row_words + 1) / 2;
   if (P.nsteps > kMaxSteps) return pl;
   // shared memory: control, weight stages, patch buffers
-  P.off_ring = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
+  // per-filter vectors (alpha; fused: also the next scale and shift), padded to whole slabs
+  P.off_vec = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
+  P.vec_len = (g.Co + 15) / 16 * 16 + 512;          // every slab of any width ends inside it
+  P.off_ring = (uint32_t)((P.off_vec + (size_t)(fuse ? 3 : 1) * P.vec_len * 4 + 127) / 128 * 128);
+  if (P.off_ring + 4096 > kSmemMax) return pl;
   const size_t avail = kSmemMax - P.off_ring;
   // st weight stages, pb patch buffers, nraw raw buffers for each subgroup of patch warps
-  auto subgroups = [&](int pb) { return (P.pat_group == kPatWarps && pb >= kPatWarps) ? kPatWarps : 1; };
+  auto subgroups = [&](int pb) { return (P.pat_group == P.pat_base && pb >= P.pat_base) ? P.pat_base : 1; };
   auto fits = [&](int st, int pb, int nraw) {
     return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes +
            (size_t)(subgroups(pb) * nraw) * P.raw_bytes <= avail;
   };
   P.wgt_warps = kWgtWarps;
+  P.pat_base = kPatWarps;
   P.pat_group = kPatWarps;
   // as few slabs as fit two accumulators in the tensor-memory columns
   const int max_nt = pair ? 224 : 240;
@@ -1187,8 +1279,12 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
       // per row fits them; with many channel words per pixel (measured: from 12 on) the other
       // four then build patches instead of draining accumulators.
       const bool helpers = g.Cw >= 12 && P.NTh <= 128;
+      // Many MMAs per item on a small patch (few channel words, a large filter): one warp
+      // cannot issue the MMAs as fast as the tensor core runs them (~95 cycles against 64 for
+      // 128 x 128 x 64), and two patch warps keep up; so the third patch warp issues too.
+      P.pat_base = (!helpers && P.nsteps >= 10 * g.Cw && P.NT <= 160) ? kPatWarps - 1 : kPatWarps;
       P.wgt_warps = helpers ? kWgtWarps / 2 : kWgtWarps;
-      P.pat_group = helpers ? kPatWarps + kWgtWarps / 2 : kPatWarps;
+      P.pat_group = helpers ? P.pat_base + kWgtWarps / 2 : P.pat_base;
       plan_stage(P);
       const int nst = (P.nsteps + P.mps - 1) / P.mps;
       if (nst <= kMaxBarStages && fits(nst, 2, 1)) {
@@ -1204,6 +1300,7 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
     P.NT = slab_width(g.Co, P.nslabs, pair || fuse);
     P.NTh = pair ? P.NT / 2 : P.NT;
     P.wgt_warps = kWgtWarps;
+    P.pat_base = kPatWarps;
     P.pat_group = kPatWarps;
     plan_stage(P);
     if (!fits(2, 1, 1)) return pl;
@@ -1218,7 +1315,7 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
   // worker warps per quarter of the lanes in the resident schedule: the four epilogue warps
   // and the weight warps (all eight, or the four that are not patch helpers)
-  P.epi_split = std::min(P.pat_group > kPatWarps ? 2 : kEpiSplitMax, P.NT / (fuse ? 32 : 16));
+  P.epi_split = std::min(P.pat_group > P.pat_base ? 2 : kEpiSplitMax, P.NT / (fuse ? 32 : 16));
   if (fuse && (g.Co & 31) != 0) return pl;          // whole words of the next layer's input
   P.stages = stages; P.npb = npb;
   // small patches: every patch warp builds whole patches on its own, three at a time
