@@ -231,6 +231,38 @@ xnor_status xnor_conv2d_forward_kbit(const uint32_t *x_planes, int kbits, const 
                                      void *cuda_stream);
 
 /*
+ * Binary-Weight-Network convolution -- Section 3.1, Eq. 1:
+ *   I * W ~ (I (+) B) alpha,
+ * real-valued inputs, B = sign(W) and alpha from xnor_binarize_weights; (+) is a
+ * convolution that only adds and subtracts input values.  The inputs are rounded
+ * once to bfloat16 (round to nearest even) and the signed sums run on the tensor
+ * cores as bf16 x (+-1) products (exact) accumulated in fp32; then
+ *   out = sum * alpha[co] (+ residual), max(., 0) with XNOR_FLAG_RELU.
+ * Two calls, like BinActiv + BinConv:
+ *   xnor_bwn_prepare_input   x fp32 [N][C_in][H][W] (after the optional BatchNorm
+ *       affine y = fmaf(bn_scale[c], x, bn_shift[c])) -> x_stream, the bfloat16 values
+ *       in the order the convolution reads them: for each of the stride^2 phases of the
+ *       input, the pixels as one stream with zero pixels where the filter overhangs the
+ *       image, C_in padded with zeros to a multiple of 16.  xnor_bwn_input_elems(d)
+ *       gives the number of 16-bit elements of x_stream for the geometry (0: bad
+ *       descriptor); the layout is private to the two calls.
+ *   xnor_bwn_conv2d_forward  x_stream, w_packed u32 [P][C_out][2], alpha fp32 [C_out],
+ *       residual fp32 [N][C_out][H_out][W_out] or NULL (may be `out`) ->
+ *       out fp32 [N][C_out][H_out][W_out].
+ * INVALID_ARG as for the other calls.  UNSUPPORTED (nothing launched): stride > 2,
+ * more than 121 filter taps, a tile's input window of more than 256 stream positions
+ * (roughly (k_h - 1) * (W + k_w) > 120 at stride 1), or a window that does not fit
+ * shared memory beside two weight stages (C_in above ~600 at 3x3 on small images).
+ * Device-side waits are bounded as in xnor_conv2d_forward (xnor_check_device).
+ */
+size_t xnor_bwn_input_elems(const xnor_conv_desc *d);
+xnor_status xnor_bwn_prepare_input(const float *x, const float *bn_scale, const float *bn_shift,
+                                   const xnor_conv_desc *d, uint16_t *x_stream, void *cuda_stream);
+xnor_status xnor_bwn_conv2d_forward(const uint16_t *x_stream, const uint32_t *w_packed,
+                                    const float *alpha, const float *residual,
+                                    const xnor_conv_desc *d, float *out, void *cuda_stream);
+
+/*
  * Full-precision 1x1 strided convolution without bias: the projection
  * shortcut ("type B") of the ResNet-18 variant the paper binarises
  * (Section 4.2).  Its result is the `residual` of a block's second BinConv.

@@ -36,6 +36,7 @@ EXPORTS = [
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
     "xnor_maxpool2d", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
     "xnor_binactiv_kbit", "xnor_conv2d_forward_kbit",
+    "xnor_bwn_input_elems", "xnor_bwn_prepare_input", "xnor_bwn_conv2d_forward",
 ]
 
 
@@ -102,6 +103,12 @@ def load():
     lib.xnor_conv2d_forward_kbit.restype = ci
     lib.xnor_conv2d_forward_kbit.argtypes = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc),
                                              vp, vp, vp]
+    lib.xnor_bwn_input_elems.restype = ctypes.c_size_t
+    lib.xnor_bwn_input_elems.argtypes = [ctypes.POINTER(xnor_conv_desc)]
+    lib.xnor_bwn_prepare_input.restype = ci
+    lib.xnor_bwn_prepare_input.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp]
+    lib.xnor_bwn_conv2d_forward.restype = ci
+    lib.xnor_bwn_conv2d_forward.argtypes = [vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp]
     _lib = lib
     return lib
 
@@ -231,6 +238,28 @@ def xnor_conv2d_forward_kbit(x_planes, kbits, w_packed, alpha, K, residual, d, o
                                            ctypes.byref(d), _ptr(out, torch.float32),
                                            _ptr(acc_out, torch.int32), _stream(stream)),
            "xnor_conv2d_forward_kbit")
+
+
+def xnor_bwn_input_elems(d):
+    return int(load().xnor_bwn_input_elems(ctypes.byref(d)))
+
+
+def xnor_bwn_prepare_input(x, bn_scale, bn_shift, d, x_stream, stream=None):
+    _check(load().xnor_bwn_prepare_input(_ptr(x, torch.float32), _ptr(bn_scale, torch.float32),
+                                         _ptr(bn_shift, torch.float32), ctypes.byref(d),
+                                         _ptr(x_stream, torch.bfloat16), _stream(stream)),
+           "xnor_bwn_prepare_input")
+
+
+def xnor_bwn_conv2d_forward(x_stream, w_packed, alpha, residual, d, out, stream=None):
+    _check(load().xnor_bwn_conv2d_forward(_ptr(x_stream, torch.bfloat16), _ptr(w_packed, torch.int32),
+                                          _ptr(alpha, torch.float32), _ptr(residual, torch.float32),
+                                          ctypes.byref(d), _ptr(out, torch.float32), _stream(stream)),
+           "xnor_bwn_conv2d_forward")
+
+
+def alloc_bwn_input(d, device="cuda"):
+    return torch.empty((xnor_bwn_input_elems(d),), dtype=torch.bfloat16, device=device)
 
 
 BINACTIV_STATIC_MAX_PIXELS = 1 << 20

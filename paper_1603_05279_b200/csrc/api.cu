@@ -269,13 +269,43 @@ xnor_status xnor_selftest_wait_timeout(void *cuda_stream) {
 }
 
 xnor_status xnor_check_device(void *cuda_stream) {
-  int st = 0;
+  int st = 0, st2 = 0;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess ||
-      xnor::read_status_tc(&st) != cudaSuccess) {
+      xnor::read_status_tc(&st) != cudaSuccess || xnor::read_status_bwn(&st2) != cudaSuccess) {
     (void)cudaGetLastError();
     return XNOR_ERR_CUDA;
   }
-  return st == 0 ? XNOR_OK : XNOR_ERR_TIMEOUT;
+  return (st == 0 && st2 == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
+}
+
+size_t xnor_bwn_input_elems(const xnor_conv_desc *d) {
+  if (!good_desc(d)) return 0;
+  return xnor::bwn_stream_elems(xnor::make_geom(*d));
+}
+
+xnor_status xnor_bwn_prepare_input(const float *x, const float *bn_scale, const float *bn_shift,
+                                   const xnor_conv_desc *d, uint16_t *x_stream, void *cuda_stream) {
+  if (!good_desc(d)) return XNOR_ERR_INVALID_ARG;
+  if (bad_ptr(x) || bad_ptr(x_stream)) return XNOR_ERR_INVALID_ARG;
+  if ((bn_scale == nullptr) != (bn_shift == nullptr)) return XNOR_ERR_INVALID_ARG;
+  if (bn_scale && (misaligned(bn_scale) || misaligned(bn_shift))) return XNOR_ERR_INVALID_ARG;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  if (!xnor::bwn_supported(g)) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_bwn_prepare(x, bn_scale, bn_shift, g, x_stream,
+                                            (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_bwn_conv2d_forward(const uint16_t *x_stream, const uint32_t *w_packed,
+                                    const float *alpha, const float *residual,
+                                    const xnor_conv_desc *d, float *out, void *cuda_stream) {
+  if (!good_desc(d)) return XNOR_ERR_INVALID_ARG;
+  if (bad_ptr(x_stream) || bad_ptr(w_packed) || bad_ptr(alpha) || bad_ptr(out) ||
+      (residual && misaligned(residual)))
+    return XNOR_ERR_INVALID_ARG;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  if (!xnor::bwn_supported(g)) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_bwn_conv(x_stream, w_packed, alpha, residual, g, out,
+                                         (cudaStream_t)cuda_stream));
 }
 
 xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,

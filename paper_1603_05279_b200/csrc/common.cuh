@@ -113,6 +113,15 @@ cudaError_t launch_binconv_tc_fused(const uint32_t *xp, const uint32_t *wp, cons
 // A = (sum of the partial planes) / C, then K = box filter of A for geometry g.
 cudaError_t launch_binactiv_finish(const float *A_part, int parts, const ConvGeom &g, float *A,
                                    float *K, cudaStream_t st);
+// Binary-Weight-Network convolution (Eq. 1) on bf16 activations laid out as a zero-padded pixel
+// stream: elements of that stream for a geometry, its preparation from fp32 NCHW, the convolution.
+bool bwn_supported(const ConvGeom &g);
+size_t bwn_stream_elems(const ConvGeom &g);
+cudaError_t launch_bwn_prepare(const float *x, const float *scale, const float *shift,
+                               const ConvGeom &g, uint16_t *x_stream, cudaStream_t st);
+cudaError_t launch_bwn_conv(const uint16_t *x_stream, const uint32_t *wp, const float *alpha,
+                            const float *residual, const ConvGeom &g, float *out, cudaStream_t st);
+cudaError_t read_status_bwn(int *status);
 // A one-warp kernel whose bounded wait expires (nothing signals its barrier).
 cudaError_t launch_wait_timeout_selftest(cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.

@@ -55,8 +55,8 @@ def host(t):
 # A kernel that writes outside a buffer it was given usually lands in a neighbouring
 # allocation and goes unnoticed.  Outputs of the parity tests are therefore carved out of a
 # larger allocation whose head and tail hold a known pattern, checked after the calls.
-GUARD = 64                      # elements on each side (4-byte types: 256 bytes, keeps 16-byte alignment)
-_PATTERN = {torch.float32: -7.25e30, torch.int32: -0x5A5A5A5B}
+GUARD = 64                      # elements on each side (a multiple of 16 bytes for 2- and 4-byte types)
+_PATTERN = {torch.float32: -7.25e30, torch.int32: -0x5A5A5A5B, torch.bfloat16: -7.25e30}
 
 
 class Guarded:
