@@ -88,8 +88,7 @@ using namespace umma;
 constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
 constexpr int kWgtWarp0 = 5, kWgtWarps = 8;
-constexpr int kPatWarp0 = 13, kPatWarps = 3;               // warps 13-15 build patches; where a second
-constexpr int kMma2Warp = 15;                              // MMA issuer pays, warp 15 is that instead
+constexpr int kPatWarp0 = 13, kPatWarps = 3;
 constexpr int kThreads = 32 * (kPatWarp0 + kPatWarps);     // 512: 16 warps, 128 registers each
 constexpr int kTileM = 128;          // stream positions per tile = tensor-memory lanes
 constexpr int kTmemCols = 512;
@@ -132,8 +131,7 @@ struct TcParams {
   int vec_len;                 // the next layer's scale and shift; vec_len floats each
   uint32_t raw_bytes;          // size of a raw buffer: the packed input rows a patch can touch
   int nraw;                    // raw buffers per subgroup of patch warps (1 or 2)
-  int pat_base;                // dedicated patch warps: 3, or 2 when warp 15 is the second MMA issuer
-  int pat_group;               // warps that build patches: pat_base, or pat_base + 4 with four of the weight warps
+  int pat_group;               // warps that build patches: 3, or 7 with four of the weight warps
   int pat_sub;                 // subgroups they form (each builds whole patches): 3 or 1
   int wgt_warps;               // warps that expand weights: 8, or 4
   uint32_t idesc;
@@ -162,73 +160,66 @@ struct TcParams {
   int div_wq_s, div_hq_s;      // (dividends below 2^31)
 };
 
-// One MMA, issued by the elected lane while the whole warp stays converged (so that the
-// descriptor arithmetic around it can stay on the uniform datapath).  Descriptors are
-// passed as their two 32-bit halves.
-__device__ __forceinline__ void umma_mxf4_elected(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
-                                                  uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                                  uint32_t sf, uint32_t accumulate,
-                                                  uint32_t elected) {
+// One MMA.  The issuing warp elects one lane, and that lane alone runs the whole issue loop:
+// a predicate per MMA inside a converged warp costs a divergence and a reconvergence each
+// time (measured: 95 cycles per MMA against 65 for the single-thread loop, the tensor core
+// needing 64 for 128 x 128 x 64).  Descriptors are passed as their two 32-bit halves.
+__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                          uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t sf, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
       "mov.b64 da, {%1, %2};\n\t"
       "mov.b64 db, {%3, %4};\n\t"
       "setp.ne.b32 p, %6, 0;\n\t"
-      "setp.ne.b32 q, %8, 0;\n\t"
-      "@q tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %5, [%7], [%7], p;\n\t}"
+      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %5, [%7], [%7], p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
-        "r"(sf), "r"(elected)
+        "r"(sf)
       : "memory");
 }
 
-__device__ __forceinline__ void umma_commit_elected(uint32_t bar, uint32_t elected) {
-  asm volatile(
-      "{\n\t.reg .pred q;\n\t"
-      "setp.ne.b32 q, %1, 0;\n\t"
-      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-      ::"r"(bar), "r"(elected) : "memory");
+__device__ __forceinline__ void umma_commit_one(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
 }
 
 // The same for a CTA pair: one instruction drives the tensor cores of both SMs (M = 256: rows
 // 0-127 from this CTA's patch into its tensor memory, rows 128-255 the peer's; each CTA
 // supplies half of the N filter rows).  Commits signal the barrier at the same offset in both.
-__device__ __forceinline__ void umma_mxf4_pair_elected(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
-                                                       uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                                       uint32_t sf, uint32_t accumulate,
-                                                       uint32_t elected) {
+__device__ __forceinline__ void umma_mxf4_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                               uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                               uint32_t sf, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
       "mov.b64 da, {%1, %2};\n\t"
       "mov.b64 db, {%3, %4};\n\t"
       "setp.ne.b32 p, %6, 0;\n\t"
-      "setp.ne.b32 q, %8, 0;\n\t"
-      "@q tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], da, db, %5, [%7], [%7], p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], da, db, %5, [%7], [%7], p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
-        "r"(sf), "r"(elected)
+        "r"(sf)
       : "memory");
 }
 
-__device__ __forceinline__ void umma_commit_pair_elected(uint32_t bar, uint32_t elected) {
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
   asm volatile(
-      "{\n\t.reg .pred q;\n\t.reg .b16 mask;\n\t"
-      "setp.ne.b32 q, %1, 0;\n\t"
+      "{\n\t.reg .b16 mask;\n\t"
       "mov.b16 mask, 3;\n\t"
-      "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], mask;\n\t}"
-      ::"r"(bar), "r"(elected) : "memory");
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], mask;\n\t}"
+      ::"r"(bar) : "memory");
 }
 
 template <bool kPair>
 __device__ __forceinline__ void umma_issue(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
                                            uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t sf,
-                                           uint32_t accumulate, uint32_t elected) {
-  if (kPair) umma_mxf4_pair_elected(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, sf, accumulate, elected);
-  else umma_mxf4_elected(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, sf, accumulate, elected);
+                                           uint32_t accumulate) {
+  if (kPair) umma_mxf4_pair(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, sf, accumulate);
+  else umma_mxf4(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, sf, accumulate);
 }
 
 template <bool kPair>
-__device__ __forceinline__ void umma_commit_to(uint32_t bar, uint32_t elected) {
-  if (kPair) umma_commit_pair_elected(bar, elected);
-  else umma_commit_elected(bar, elected);
+__device__ __forceinline__ void umma_commit_to(uint32_t bar) {
+  if (kPair) umma_commit_pair(bar);
+  else umma_commit_one(bar);
 }
 
 __device__ __forceinline__ uint32_t elect_one() {
@@ -377,37 +368,24 @@ __device__ __forceinline__ Smem carve(uint8_t *smem, const TcParams &P) {
   return s;
 }
 
-// ------------------------------------------------------------------ MMA issuer (one warp)
-// All 32 lanes run this code converged; only the MMA and commit instructions are
-// predicated on the elected lane.  A wait's outcome is made warp-uniform with a vote.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity,
-                                               volatile int *abort_flag) {
-  return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, &g_status_tc));
-}
-
+// ------------------------------------------------------------------ MMA issuer (one thread)
 // The MMAs of one full weight stage, unrolled.
 template <int MPS, bool kPair>
 __device__ __forceinline__ void issue_stage(const TcParams &P, int j0, uint32_t d_tmem,
                                             uint32_t patch_lo, uint32_t a_hi, uint32_t b_lo,
                                             uint32_t b_hi, uint32_t b_step, uint32_t tmem_sf,
-                                            uint32_t first, uint32_t el) {
+                                            uint32_t first) {
 #pragma unroll
   for (int jj = 0; jj < MPS; ++jj)
     umma_issue<kPair>(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, a_hi, b_lo + (uint32_t)jj * b_step,
-                      b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u, el);
+                      b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u);
 }
 
-// kRes: resident schedule.  The stage barriers are then waited for only before an issuer's
-// first item (the slab stays in shared memory afterwards) and never released.
-// Resident schedule: two warps issue (`which` = 0, 1 of `nissue` = 2), taking alternate items.
-// One warp issues an MMA of 128 x 128 x 64 every ~95 cycles (measured; ~105 beside busy
-// epilogue warps) while the tensor core needs 64: two issuers keep it fed.  Each item has its own
-// patch and accumulator buffer, and a CTA stays on one slab (no stage is ever released), so the
-// two streams of MMAs depend on nothing of each other.  Streaming: one issuer (the stages of the
-// weight ring are handed from item to item in order).
+// kRes: resident schedule.  The stage barriers are then waited for only before the first item
+// (the CTA stays on one slab, which stays in shared memory) and never released.
 template <bool kRes, bool kPair>
-__device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long long i1,
-                         uint32_t tmem_base, uint32_t which, uint32_t nissue) {
+__device__ void mma_loop(const TcParams &P, const Smem &S, long long i0, long long i1,
+                         uint32_t tmem_base) {
   const uint32_t tmem_sf = tmem_base + (uint32_t)kSfCol;
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const uint32_t b_lbo = (uint32_t)P.NTh * 16u;
@@ -416,7 +394,6 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
   const uint32_t b_lo0 = ((S.ring & 0x3FFFFu) >> 4) | ((b_lbo >> 4) << 16);   // stage 0, K-step 0
   const uint32_t b_step = (2u * b_lbo) >> 4;                                   // next K-step
   const uint32_t stage_step = P.stage_bytes >> 4;
-  const uint32_t el = elect_one();
   int ws = 0, pb = 0, ab = 0;
   uint32_t wph = 0, pph = 0;
   uint32_t aph = 1u;                     // parity to wait for on the accumulator's empty barrier
@@ -427,62 +404,63 @@ __device__ void mma_role(const TcParams &P, const Smem &S, long long i0, long lo
   bool ok = true, new_tile = true;
   uint32_t patch_lo = 0;                 // patch address in descriptor units
   const uint32_t nitems = kRes ? R.total() : (uint32_t)(i1 - i0);
-  for (uint32_t it = which; it < nitems && ok; it += nissue) {
-    if (kRes) {
-      // buffers and barrier phases of the it-th item of the CTA
-      pb = (int)(it % (uint32_t)P.npb);
-      pph = (it / (uint32_t)P.npb) & 1u;
-      ab = (int)(it % (uint32_t)P.nacc);
-      aph = ((it / (uint32_t)P.nacc) & 1u) ^ 1u;
-      ws = 0;
-    }
+  for (uint32_t it = 0; it < nitems && ok; ++it) {
     if (new_tile) {
-      ok = mbar_wait_warp(S.pfull + 8u * pb, pph, S.abort_flag);
+      ok = mbar_wait(S.pfull + 8u * pb, pph, S.abort_flag, &g_status_tc);
       if (!ok) break;
       patch_lo = ((S.patch + (uint32_t)pb * P.patch_bytes) & 0x3FFFFu) >> 4;
     }
-    // resident: the slab is expanded once; an issuer waits for its stages before its first item
-    const bool wait_stages = !kRes || it == which;
-    ok = mbar_wait_warp(S.aempty + 8u * ab, aph, S.abort_flag);
+    const bool wait_stages = !kRes || it == 0;
+    ok = mbar_wait(S.aempty + 8u * ab, aph, S.abort_flag, &g_status_tc);
     if (!ok) break;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.NT);
+    if (kRes) ws = 0;
     for (int st = 0; st < nst && ok; ++st) {
       const int j0 = st * P.mps;
       const int nj = min(P.mps, P.nsteps - j0);
       const uint32_t b_lo = b_lo0 + (uint32_t)ws * stage_step;
       const uint32_t first = st == 0 ? 0u : 1u;     // the first MMA of an item overwrites
       if (wait_stages) {
-        ok = mbar_wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
+        ok = mbar_wait(S.wfull + 8u * ws, wph, S.abort_flag, &g_status_tc);
         if (!ok) break;
         tc_fence_after();
       }
-      if (nj == 4) issue_stage<4, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
-      else if (nj == 2) issue_stage<2, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
-      else if (nj == 8) issue_stage<8, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first, el);
+      if (nj == 4) issue_stage<4, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first);
+      else if (nj == 2) issue_stage<2, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first);
+      else if (nj == 8) issue_stage<8, kPair>(P, j0, d_tmem, patch_lo, desc_hi, b_lo, desc_hi, b_step, tmem_sf, first);
       else {
         for (int jj = 0; jj < nj; ++jj)
           umma_issue<kPair>(d_tmem, P.adesc_lo[j0 + jj] + patch_lo, desc_hi,
                             b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc, tmem_sf,
-                            jj == 0 ? first : 1u, el);
+                            jj == 0 ? first : 1u);
       }
-      if (!kRes) umma_commit_to<kPair>(S.wempty + 8u * ws, el);
+      if (!kRes) umma_commit_to<kPair>(S.wempty + 8u * ws);
       if (++ws == P.stages) { ws = 0; if (!kRes) wph ^= 1u; }
     }
     if (!ok) break;
     if (kRes) {
-      umma_commit_to<kPair>(S.afull + 8u * ab, el);
-      umma_commit_to<kPair>(S.pempty + 8u * pb, el);
+      // every item has its own patch
+      umma_commit_to<kPair>(S.afull + 8u * ab);
+      umma_commit_to<kPair>(S.pempty + 8u * pb);
+      if (++pb == P.npb) { pb = 0; pph ^= 1u; }
     } else {
       // next item: same tile (next slab) or the next tile
       new_tile = false;
       if (++slab == P.nslabs) { slab = 0; new_tile = true; }
-      umma_commit_to<kPair>(S.afull + 8u * ab, el);
-      if (new_tile || it + 1 == nitems) umma_commit_to<kPair>(S.pempty + 8u * pb, el);
+      umma_commit_to<kPair>(S.afull + 8u * ab);
+      if (new_tile || it + 1 == nitems) umma_commit_to<kPair>(S.pempty + 8u * pb);
       if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
-      if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
     }
+    if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
   }
+}
+
+template <bool kRes, bool kPair>
+__device__ __forceinline__ void mma_role(const TcParams &P, const Smem &S, long long i0, long long i1,
+                                         uint32_t tmem_base) {
+  if (elect_one()) mma_loop<kRes, kPair>(P, S, i0, i1, tmem_base);
+  __syncwarp();
 }
 
 // ------------------------------------------------------------------ weight producers (8 warps)
@@ -1136,12 +1114,10 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
   const ResSched R = res_sched(P.ntiles, P.nslabs, kPair);
   if (kRes ? R.total() > 0u : i0 < i1) {
     const int wt = tid - 32 * kWgtWarp0;
-    const uint32_t nissue = P.pat_base < kPatWarps ? 2u : 1u;
-    if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base, 0u, nissue); }
-    else if (warp == kMma2Warp && nissue == 2u) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base, 1u, 2u); }
+    if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base); }
     else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, warp - kPatWarp0, lane);
-    else if (kRes && P.pat_group > P.pat_base && warp >= kWgtWarp0 + 4)
-      patch_role<kRes>(P, S, i0, i1, P.pat_base + warp - (kWgtWarp0 + 4), lane);   // helpers
+    else if (kRes && P.pat_group > kPatWarps && warp >= kWgtWarp0 + 4)
+      patch_role<kRes>(P, S, i0, i1, kPatWarps + warp - (kWgtWarp0 + 4), lane);   // helpers
     else if (!kRes) {
       if (warp < kEpiWarps)
         epilogue_role<false, kFuse>(P, S, i0, 0, 0, 0, (uint32_t)(i1 - i0), 0, tmem_base, warp, 0, lane);
@@ -1253,13 +1229,12 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   if (P.off_ring + 4096 > kSmemMax) return pl;
   const size_t avail = kSmemMax - P.off_ring;
   // st weight stages, pb patch buffers, nraw raw buffers for each subgroup of patch warps
-  auto subgroups = [&](int pb) { return (P.pat_group == P.pat_base && pb >= P.pat_base) ? P.pat_base : 1; };
+  auto subgroups = [&](int pb) { return (P.pat_group == kPatWarps && pb >= kPatWarps) ? kPatWarps : 1; };
   auto fits = [&](int st, int pb, int nraw) {
     return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes +
            (size_t)(subgroups(pb) * nraw) * P.raw_bytes <= avail;
   };
   P.wgt_warps = kWgtWarps;
-  P.pat_base = kPatWarps;
   P.pat_group = kPatWarps;
   // as few slabs as fit two accumulators in the tensor-memory columns
   const int max_nt = pair ? 224 : 240;
@@ -1279,12 +1254,8 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
       // per row fits them; with many channel words per pixel (measured: from 12 on) the other
       // four then build patches instead of draining accumulators.
       const bool helpers = g.Cw >= 12 && P.NTh <= 128;
-      // Many MMAs per item on a small patch (few channel words, a large filter): one warp
-      // cannot issue the MMAs as fast as the tensor core runs them (~95 cycles against 64 for
-      // 128 x 128 x 64), and two patch warps keep up; so the third patch warp issues too.
-      P.pat_base = (!helpers && P.nsteps >= 10 * g.Cw && P.NT <= 160) ? kPatWarps - 1 : kPatWarps;
       P.wgt_warps = helpers ? kWgtWarps / 2 : kWgtWarps;
-      P.pat_group = helpers ? P.pat_base + kWgtWarps / 2 : P.pat_base;
+      P.pat_group = helpers ? kPatWarps + kWgtWarps / 2 : kPatWarps;
       plan_stage(P);
       const int nst = (P.nsteps + P.mps - 1) / P.mps;
       if (nst <= kMaxBarStages && fits(nst, 2, 1)) {
@@ -1300,7 +1271,6 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
     P.NT = slab_width(g.Co, P.nslabs, pair || fuse);
     P.NTh = pair ? P.NT / 2 : P.NT;
     P.wgt_warps = kWgtWarps;
-    P.pat_base = kPatWarps;
     P.pat_group = kPatWarps;
     plan_stage(P);
     if (!fits(2, 1, 1)) return pl;
@@ -1315,7 +1285,7 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
   // worker warps per quarter of the lanes in the resident schedule: the four epilogue warps
   // and the weight warps (all eight, or the four that are not patch helpers)
-  P.epi_split = std::min(P.pat_group > P.pat_base ? 2 : kEpiSplitMax, P.NT / (fuse ? 32 : 16));
+  P.epi_split = std::min(P.pat_group > kPatWarps ? 2 : kEpiSplitMax, P.NT / (fuse ? 32 : 16));
   if (fuse && (g.Co & 31) != 0) return pl;          // whole words of the next layer's input
   P.stages = stages; P.npb = npb;
   // small patches: every patch warp builds whole patches on its own, three at a time

@@ -85,28 +85,24 @@ __device__ __forceinline__ uint32_t elect_one() {
   return pred;
 }
 
-// One MMA of 128 x NT x 16 (bf16), issued by the elected lane of a converged warp.
-__device__ __forceinline__ void umma_bf16_elected(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
-                                                  uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                                  uint32_t accumulate, uint32_t elected) {
+// One MMA of 128 x NT x 16 (bf16).  One elected lane of the issuing warp runs the whole issue
+// loop (a predicate per MMA in a converged warp costs a divergence each time).
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                          uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
       "mov.b64 da, {%1, %2};\n\t"
       "mov.b64 db, {%3, %4};\n\t"
       "setp.ne.b32 p, %6, 0;\n\t"
-      "setp.ne.b32 q, %7, 0;\n\t"
-      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
-        "r"(elected)
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
-__device__ __forceinline__ void commit_elected(uint32_t bar, uint32_t elected) {
-  asm volatile(
-      "{\n\t.reg .pred q;\n\t"
-      "setp.ne.b32 q, %1, 0;\n\t"
-      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-      ::"r"(bar), "r"(elected) : "memory");
+__device__ __forceinline__ void commit_one(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
 }
 
 // TMA tile copy global -> shared of one operand plane of a patch: box {8, 1, ppix, 1} at
@@ -154,8 +150,8 @@ __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatil
   return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, &g_status_bwn));
 }
 
-// ------------------------------------------------------------------ MMA issuer
-__device__ void mma_role(const BwnParams &P, const Smem &S, long long i0, long long i1,
+// ------------------------------------------------------------------ MMA issuer (one thread)
+__device__ void mma_loop(const BwnParams &P, const Smem &S, long long i0, long long i1,
                          uint32_t tmem_base) {
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
@@ -165,7 +161,6 @@ __device__ void mma_role(const BwnParams &P, const Smem &S, long long i0, long l
   const uint32_t b_step = (2u * b_lbo) >> 4;
   const uint32_t a_step = (2u * P.plane_bytes) >> 4;       // next 16 channels of the same tap
   const uint32_t stage_step = P.stage_bytes >> 4;
-  const uint32_t el = elect_one();
   int ws = 0, pb = 0, ab = 0;
   uint32_t wph = 0, pph = 0, aph = 1u;
   int slab = (int)(i0 % P.nslabs);
@@ -174,11 +169,11 @@ __device__ void mma_role(const BwnParams &P, const Smem &S, long long i0, long l
   const uint32_t nitems = (uint32_t)(i1 - i0);
   for (uint32_t it = 0; it < nitems && ok; ++it) {
     if (new_tile) {
-      ok = wait_warp(S.pfull + 8u * pb, pph, S.abort_flag);
+      ok = mbar_wait(S.pfull + 8u * pb, pph, S.abort_flag, &g_status_bwn);
       if (!ok) break;
       patch_lo = ((S.patch + (uint32_t)pb * P.patch_bytes) & 0x3FFFFu) >> 4;
     }
-    ok = wait_warp(S.aempty + 8u * ab, aph, S.abort_flag);
+    ok = mbar_wait(S.aempty + 8u * ab, aph, S.abort_flag, &g_status_bwn);
     if (!ok) break;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.NT);
@@ -186,27 +181,33 @@ __device__ void mma_role(const BwnParams &P, const Smem &S, long long i0, long l
     for (int st = 0; st < nst && ok; ++st) {
       const int j0 = st * P.mps;
       const int nj = min(P.mps, P.nsteps - j0);
-      ok = wait_warp(S.wfull + 8u * ws, wph, S.abort_flag);
+      ok = mbar_wait(S.wfull + 8u * ws, wph, S.abort_flag, &g_status_bwn);
       if (!ok) break;
       tc_fence_after();
       const uint32_t b_lo = b_lo0 + (uint32_t)ws * stage_step;
       for (int jj = 0; jj < nj; ++jj) {
         const uint32_t a_lo = ((patch_lo + P.tap_lo[tap] + (uint32_t)c16 * a_step) & 0x3FFFu) | a_lbo_hi;
-        umma_bf16_elected(d_tmem, a_lo, desc_hi, b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc,
-                          (j0 + jj) == 0 ? 0u : 1u, el);
+        umma_bf16(d_tmem, a_lo, desc_hi, b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc,
+                  (j0 + jj) == 0 ? 0u : 1u);
         if (++c16 == P.cpt) { c16 = 0; ++tap; }
       }
-      commit_elected(S.wempty + 8u * ws, el);
+      commit_one(S.wempty + 8u * ws);
       if (++ws == P.stages) { ws = 0; wph ^= 1u; }
     }
     if (!ok) break;
     new_tile = false;
     if (++slab == P.nslabs) { slab = 0; new_tile = true; }
-    commit_elected(S.afull + 8u * ab, el);
-    if (new_tile || it + 1 == nitems) commit_elected(S.pempty + 8u * pb, el);
+    commit_one(S.afull + 8u * ab);
+    if (new_tile || it + 1 == nitems) commit_one(S.pempty + 8u * pb);
     if (new_tile) { if (++pb == P.npb) { pb = 0; pph ^= 1u; } }
     if (++ab == P.nacc) { ab = 0; aph ^= 1u; }
   }
+}
+
+__device__ __forceinline__ void mma_role(const BwnParams &P, const Smem &S, long long i0, long long i1,
+                                         uint32_t tmem_base) {
+  if (elect_one()) mma_loop(P, S, i0, i1, tmem_base);
+  __syncwarp();
 }
 
 // ------------------------------------------------------------------ TMA producer (one warp)
