@@ -38,9 +38,9 @@ BF16_FALLBACK_TFLOPS = 1590.0
 # guide, arithmetic-instruction throughput table, compute capability 10.0); one result
 # covers 32 one-bit MACs.
 POPC_PER_CLK_PER_SM = 16
-# DRAM traffic of the dominant kernel from one ncu capture (profiles/step_kernels_alexnet.md):
-# dram__bytes_read.sum + dram__bytes_write.sum summed over the four BinConv launches of one
-# step of the default workload.  Valid only for the kernel source it was taken from.
+# DRAM traffic of the dominant kernel from one ncu capture: dram__bytes_read.sum +
+# dram__bytes_write.sum summed over the four BinConv launches of one step of the default
+# workload.  Valid only for the kernel source it was taken from (hash below); null otherwise.
 NCU_TRAFFIC = {"kernel_sha1": "2c5af8e4edf24572ab0755be0093681529d9235e", "bytes_per_step": 160.8e6}
 
 
@@ -242,13 +242,13 @@ class ClockSampler:
 class LayersJob:
     """Independent layers: per layer binarize_weights -> binactiv -> conv."""
 
-    def __init__(self, name, layer_ids, batch, rank):
+    def __init__(self, name, layer_ids, batch, rank, variant="xnor", kbits=2):
         import torch
         from paper_1603_05279_b200.runner import LAUNCHES_PER_LAYER, LayerBuffers
         self.torch = torch
         shapes = [wl.scaled(wl.CONFIGS[name][i], batch) for i in layer_ids]
         self.shapes = shapes
-        self.layers = [LayerBuffers(s) for s in shapes]
+        self.layers = [LayerBuffers(s, variant=variant, kbits=kbits) for s in shapes]
         self.host_x, self.host_w, self.host_out = [], [], []
         for li, L in zip(layer_ids, self.layers):
             seed = du.rank_seed(wl.layer_seed(name, li), rank)
@@ -257,7 +257,10 @@ class LayersJob:
             self.host_out.append(torch.empty(L.out.shape, dtype=torch.float32).pin_memory())
             L.x.copy_(self.host_x[-1])
             L.w.copy_(self.host_w[-1])
-        self.launches = LAUNCHES_PER_LAYER * len(self.layers)
+        # kernels per layer: binarize 1, BinActiv 2 (pack, box filter), BinConv 1 (k-bit: one per
+        # plane; Binary-Weight: prepare 1, convolution 1)
+        per_layer = {"xnor": LAUNCHES_PER_LAYER, "bwn": 3, "kbit": 3 + kbits}[variant]
+        self.launches = per_layer * len(self.layers)
         self.macs = sum(wl.macs(s) for s in shapes)
         self.conv_macs = [wl.macs(s) for s in shapes]
         self.images = batch
@@ -466,8 +469,11 @@ def run_ours(args):
     if args.workload == "chain":
         job = ChainJob(args.batch, rank, fused=args.fused)
     else:
-        job = LayersJob(args.workload, args.layer_ids, args.batch, rank)
+        job = LayersJob(args.workload, args.layer_ids, args.batch, rank, variant=args.variant,
+                        kbits=args.kbits)
     torch.cuda.synchronize()
+    # the per-clock rates of the two pipes, measured now on this GPU (untimed prologue)
+    mma_rate, popc_rate = X.xnor_measure_peaks(stream)
 
     props = torch.cuda.get_device_properties(local)
     gpu_id = getattr(props, "uuid", None)
@@ -551,37 +557,63 @@ def run_ours(args):
     value = du.job_throughput(job.macs, args.steps, world, elapsed_ms) / 1e12
     e2e_value = du.job_throughput(job.macs, args.steps, world, e2e_ms) / 1e12
 
-    full = args.batch == default_batch(args.workload) and \
+    all_layers = args.batch == default_batch(args.workload) and \
         (args.workload == "chain" or args.layer_ids == list(range(len(wl.CONFIGS[args.workload]))))
+    full = all_layers and args.variant == "xnor"
     peaks = measured_peaks()
     clocks = sampler.summary(t_load0, t_load1)
     conv_ms = sum(per["conv"].values())
     conv_macs = sum(job.conv_macs)
     engine = args.engine
     n_conv = len(job.conv_macs)
-    if engine != "popc":
-        # tensor-core peak for the operand type in use = measured bf16 peak x the nominal
-        # ratio of that type to bf16 (e2m1: 9 / 2.25 = 4, int8: 2); the sustained figure,
-        # because the kernel is timed inside a long step.  2 flops per 1-bit MAC.
-        ratio, kind = 4, "e2m1 (fp4)"
-        roofline = {"kernel": "BinConv tensor-core kernel (one launch per layer, %d per step)"
-                              % n_conv, "bound": "tensor",
+    sms = props.multi_processor_count
+    clk_mhz = clocks["sm_mhz"] or 1965.0
+    if args.variant == "bwn":
+        # bf16 x (+-1 as bf16) on kind::f16: the measured bf16 GEMM peak; the burst figure when the
+        # sampled clock is the maximum one, else the sustained figure
+        burst = clocks["sm_max_mhz"] is not None and clk_mhz >= 0.97 * (clocks["sm_max_mhz"] or clk_mhz)
+        peak = peaks["bf16"] if burst else peaks["bf16_sustained"]
+        roofline = {"kernel": "bwn_conv_kernel (%d launches per step)" % n_conv, "bound": "tensor",
+                    "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                    "peak_source": "%s bf16 GEMM TFLOP/s, %s figure (SM clock %.0f MHz during the run)"
+                                   % (peaks["source"], "burst" if burst else "sustained", clk_mhz),
+                    "traffic": None}
+    elif engine != "popc":
+        # Tensor-core peak of the operand type in use, measured on this GPU before the timed
+        # region: 1-bit MACs per clock per SM of tcgen05.mma kind::mxf4 on operands in shared
+        # memory, times the SMs, times the median SM clock sampled during the timed steps (so
+        # the peak is the one that holds at the clock the kernels really ran at).  2 flops per MAC.
+        peak = 2 * mma_rate * sms * clk_mhz * 1e6 / 1e12
+        roofline = {"kernel": "BinConv tensor-core kernel (%d launches per step)" % n_conv,
+                    "bound": "tensor",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12,
-                    "peak": ratio * peaks["bf16_sustained"], "unit": "TFLOP/s",
-                    "peak_source": "%d x %s sustained bf16 TFLOP/s (nominal %s : bf16 ratio)"
-                                   % (ratio, peaks["source"], kind), "traffic": None}
+                    "peak": peak, "unit": "TFLOP/s",
+                    "peak_source": "measured in this run: tcgen05.mma kind::mxf4 (e2m1) 128x256x64 from "
+                                   "shared memory = %.0f MAC/clk/SM x %d SMs x %.0f MHz (median SM clock "
+                                   "sampled during the timed steps; reasons: %s)"
+                                   % (mma_rate, sms, clk_mhz, ",".join(clocks["reasons"]) or "none"),
+                    "peak_nominal": {"4 x bf16 burst": 4 * peaks["bf16"],
+                                     "4 x bf16 sustained": 4 * peaks["bf16_sustained"],
+                                     "note": "%s bf16 GEMM TFLOP/s x the nominal e2m1 : bf16 ratio"
+                                             % peaks["source"]},
+                    "mac_per_clk_per_sm": {
+                        "peak_measured": round(mma_rate, 1),
+                        "achieved": round(conv_macs / (conv_ms / 1e3) / (clk_mhz * 1e6) / sms, 1),
+                        "per_layer": [round(job.conv_macs[i] / (per["conv"][k] / 1e3) / (clk_mhz * 1e6) / sms, 1)
+                                      for i, k in enumerate(sorted(per["conv"]))]},
+                    "traffic": None}
     else:
-        clk = (clocks["sm_mhz"] or 1965.0) * 1e6
-        peak = POPC_PER_CLK_PER_SM * 32 * props.multi_processor_count * clk * 2 / 1e12
+        peak = popc_rate * 32 * sms * clk_mhz * 1e6 * 2 / 1e12
         roofline = {"kernel": "binconv_popc_kernel (%d launches per step)" % n_conv,
                     "bound": "alu",
                     "achieved": 2 * conv_macs / (conv_ms / 1e3) / 1e12, "peak": peak,
                     "unit": "TFLOP/s",
-                    "peak_source": "derived: 16 popc/clk/SM x 32 bits x %d SMs x median SM clock "
-                                   "during the run" % props.multi_processor_count,
+                    "peak_source": "measured in this run: %.1f popc/clk/SM (XOR + popc + add chains) x 32 "
+                                   "bits x %d SMs x %.0f MHz (median SM clock during the run)"
+                                   % (popc_rate, sms, clk_mhz),
                     "traffic": None}
     roofline["frac"] = roofline["achieved"] / roofline["peak"]
-    if engine != "popc" and full and args.workload == "alexnet" and \
+    if engine != "popc" and args.variant == "xnor" and full and args.workload == "alexnet" and \
             NCU_TRAFFIC["kernel_sha1"] == kernel_sha1():
         roofline["traffic"] = NCU_TRAFFIC["bytes_per_step"]
         roofline["traffic_note"] = ("bytes per step over the 4 launches; below the algorithmic "
@@ -602,7 +634,14 @@ def run_ours(args):
         ho, wo = wl.out_hw(sh)
         return 4 * (sh.N * sh.H * sh.W * cw + sh.C_out * sh.k * sh.k * cw + sh.N * ho * wo * (1 + sh.C_out)
                     + sh.C_out)
-    hbm_floor = [conv_bytes(sh) / (peaks["hbm_gbs"] * 1e9) * 1e6 for sh in job.shapes]
+    # layers of the chain that add a shortcut read it too
+    def residual_bytes(i, sh):
+        if args.workload != "chain" or i % 2 == 0:
+            return 0
+        ho, wo = wl.out_hw(sh)
+        return 4 * sh.N * sh.C_out * ho * wo
+    hbm_floor = [(conv_bytes(sh) + residual_bytes(i, sh)) / (peaks["hbm_gbs"] * 1e9) * 1e6
+                 for i, sh in enumerate(job.shapes)]
     pipe_floor = [2 * m / (roofline["peak"] * 1e12) * 1e6 for m in job.conv_macs]
     breakdown = {
         "conv_floor_us": {"hbm": [round(v, 1) for v in hbm_floor],
@@ -622,13 +661,17 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
-        "dtype": ("u32 bit words (XOR+popcount), int32 sums, fp32 scaling" if engine == "popc"
+        "dtype": ("bf16 activations x 1-bit weights (as +-1 bf16), fp32 accumulation" if args.variant == "bwn"
+                  else "u32 bit words (XOR+popcount), int32 sums, fp32 scaling" if engine == "popc"
                   else "e2m1 (fp4) tensor-core operands from 1-bit words, exact integer sums in "
                        "fp32, fp32 scaling"),
         "data": "synthetic",
-        "config": {"workload": name if full else "subset of " + name,
+        "config": {"workload": name if full else
+                   (name + " (" + args.variant + " variant)") if all_layers and args.variant != "xnor"
+                   else "subset of " + name,
                    "layers": [s.name for s in job.shapes],
                    "batch_per_gpu": job.images, "engine": engine,
+                   "variant": args.variant + ("%d" % args.kbits if args.variant == "kbit" else ""),
                    "fused_binactiv": bool(getattr(job, "fused", False)),
                    "l2": "step working set %d MB of inputs+outputs (L2 is 126 MB); no flush"
                          % ((job.h2d + job.d2h + (job.act_bytes if args.workload == "chain" else 0))
@@ -669,6 +712,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true",
                     help="time call-by-call launches instead of a CUDA graph of the step")
     ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_stream"])
+    ap.add_argument("--variant", default="xnor", choices=["xnor", "bwn", "kbit"],
+                    help="layer workloads only: the XNOR block (default, the bench line), the "
+                         "Binary-Weight-Network convolution on real inputs, or k-bit activations")
+    ap.add_argument("--kbits", type=int, default=2, help="bits of the k-bit variant")
     ap.add_argument("--workload", default="alexnet", choices=sorted(WORKLOAD_NAMES),
                     help="shape set (the bench line proper is the default, alexnet)")
     ap.add_argument("--layers", default="",

@@ -360,6 +360,24 @@ xnor_status xnor_set_engine(xnor_engine e);
 xnor_engine xnor_get_engine(void);
 
 /*
+ * Measures, on the current device, the per-clock rates of the two pipes a binary
+ * convolution can run on (Section 4.1 reasons in binary operations per clock):
+ *   mma_mac_per_clk_per_sm   1-bit multiply-accumulates per SM clock of the tensor
+ *                            cores on the instruction the BinConv kernel issues
+ *                            (tcgen05.mma kind::mxf4 on operands in shared memory,
+ *                            128 x 256 x 64 per instruction);
+ *   popc_per_clk_per_sm      32-bit population counts (with their XOR and add) per
+ *                            SM clock on the CUDA cores (one covers 32 1-bit MACs).
+ * Both are HOST pointers.  Multiply by the number of SMs and the SM clock observed
+ * while the kernels of interest run to get a peak in operations per second.  The
+ * call launches two short kernels (about a millisecond each, twice) on `cuda_stream`
+ * and SYNCHRONISES that stream; it allocates nothing.  For benchmarks, not for the
+ * data path.  XNOR_ERR_CUDA when a launch fails or a bounded wait inside gives up.
+ */
+xnor_status xnor_measure_peaks(double *mma_mac_per_clk_per_sm, double *popc_per_clk_per_sm,
+                               void *cuda_stream);
+
+/*
  * The one call that synchronises: waits for `cuda_stream`, then reads the
  * device-side status word.  Every wait inside the tensor-core kernel (on a
  * shared-memory barrier) is bounded; a wait that expires records

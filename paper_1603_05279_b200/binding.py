@@ -36,7 +36,7 @@ EXPORTS = [
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
     "xnor_maxpool2d", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
     "xnor_binactiv_kbit", "xnor_conv2d_forward_kbit",
-    "xnor_bwn_input_elems", "xnor_bwn_prepare_input", "xnor_bwn_conv2d_forward",
+    "xnor_bwn_input_elems", "xnor_bwn_prepare_input", "xnor_bwn_conv2d_forward", "xnor_measure_peaks",
 ]
 
 
@@ -109,6 +109,8 @@ def load():
     lib.xnor_bwn_prepare_input.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp]
     lib.xnor_bwn_conv2d_forward.restype = ci
     lib.xnor_bwn_conv2d_forward.argtypes = [vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp]
+    lib.xnor_measure_peaks.restype = ci
+    lib.xnor_measure_peaks.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
     _lib = lib
     return lib
 
@@ -238,6 +240,13 @@ def xnor_conv2d_forward_kbit(x_planes, kbits, w_packed, alpha, K, residual, d, o
                                            ctypes.byref(d), _ptr(out, torch.float32),
                                            _ptr(acc_out, torch.int32), _stream(stream)),
            "xnor_conv2d_forward_kbit")
+
+
+def xnor_measure_peaks(stream=None):
+    """(1-bit MACs per clock per SM on the tensor pipe, popc per clock per SM), measured now."""
+    a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(load().xnor_measure_peaks(ctypes.byref(a), ctypes.byref(b), _stream(stream)), "xnor_measure_peaks")
+    return a.value, b.value
 
 
 def xnor_bwn_input_elems(d):

@@ -278,6 +278,15 @@ xnor_status xnor_check_device(void *cuda_stream) {
   return (st == 0 && st2 == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
 }
 
+xnor_status xnor_measure_peaks(double *mma_mac_per_clk_per_sm, double *popc_per_clk_per_sm,
+                               void *cuda_stream) {
+  if (mma_mac_per_clk_per_sm == nullptr || popc_per_clk_per_sm == nullptr) return XNOR_ERR_INVALID_ARG;
+  const cudaError_t e = xnor::measure_pipe_peaks(mma_mac_per_clk_per_sm, popc_per_clk_per_sm,
+                                                 (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) (void)cudaGetLastError();
+  return from_cuda(e);
+}
+
 size_t xnor_bwn_input_elems(const xnor_conv_desc *d) {
   if (!good_desc(d)) return 0;
   return xnor::bwn_stream_elems(xnor::make_geom(*d));

@@ -378,19 +378,29 @@ binactiv_pack_kbit_kernel(const float *__restrict__ x, const float *__restrict__
       uint32_t words[7] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
       float p0 = 0.0f, p1 = 0.0f;
       const int c0 = cw * 32, nc = min(32, C - c0);
-      for (int j = 0; j < nc; ++j) {
-        float y = __ldg(src + (size_t)(c0 + j) * HW);
-        if (scale != nullptr) y = __fmaf_rn(__ldg(scale + c0 + j), y, __ldg(shift + c0 + j));
-        if (j & 1) p1 += fabsf(y); else p0 += fabsf(y);
-        // largest index whose decision point is <= y, by bisection over the sorted tau
-        int idx = 0;
-        for (int b = kbits - 1; b >= 0; --b) {
-          const int cand = idx + (1 << b);
-          if (y >= tau[cand]) idx = cand;
-        }
+      for (int j0 = 0; j0 < nc; j0 += 8) {
+        float yv[8];                       // eight loads in flight before any is used
 #pragma unroll
-        for (int b = 0; b < 7; ++b)
-          if (b < kbits) words[b] |= (uint32_t)((idx >> b) & 1) << j;
+        for (int q = 0; q < 8; ++q)
+          yv[q] = j0 + q < nc ? __ldg(src + (size_t)(c0 + j0 + q) * HW) : 0.0f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int j = j0 + q;
+          if (j < nc) {
+            float y = yv[q];
+            if (scale != nullptr) y = __fmaf_rn(__ldg(scale + c0 + j), y, __ldg(shift + c0 + j));
+            if (q & 1) p1 += fabsf(y); else p0 += fabsf(y);
+            // largest index whose decision point is <= y, by bisection over the sorted tau
+            int idx = 0;
+            for (int b = kbits - 1; b >= 0; --b) {
+              const int cand = idx + (1 << b);
+              if (y >= tau[cand]) idx = cand;
+            }
+#pragma unroll
+            for (int b = 0; b < 7; ++b)
+              if (b < kbits) words[b] |= (uint32_t)((idx >> b) & 1) << j;
+          }
+        }
       }
       asum += p0 + p1;
 #pragma unroll

@@ -108,8 +108,7 @@ binconv_popc_kernel(const uint32_t *__restrict__ xp, const uint32_t *__restrict_
     if (co >= P.Co) break;
     const int acc = nvalid * P.C - 2 * pops[f];
     const size_t o = ((size_t)n * P.Co + co) * HoWo + op;
-    float v = __fmul_rn(__fmul_rn((float)acc, kv), __ldg(alpha + co));
-    if (epi.out_scale != 1.0f) v = __fmul_rn(v, epi.out_scale);
+    float v = __fmul_rn(__fmul_rn((float)acc, kv), __fmul_rn(__ldg(alpha + co), epi.out_scale));
     if (residual) v += residual[o];
     if (epi.relu) v = fmaxf(v, 0.0f);
     out[o] = v;

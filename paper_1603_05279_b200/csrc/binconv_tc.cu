@@ -110,7 +110,7 @@ struct TcParams {
   float *out;
   int32_t *acc_out;
   int relu;                    // max(v, 0) on every stored value
-  float out_scale;             // extra factor of D K alpha (1 unless several calls build one output)
+  float out_scale;             // extra factor of D K alpha (1 unless several calls build one output), folded into the staged alpha
   int acc_shift, acc_accum;    // acc_out receives D << acc_shift, stored or added to its content
   int N, C, H, W, Co, kh, kw, stride, pad, Ho, Wo, Cw;
   int Hq, Wq, leadY, leadX;    // stream geometry of every phase plane
@@ -823,7 +823,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t howo = (uint32_t)HoWo;
   // the fast store paths: offsets of 16 consecutive filters fit 32 bits, no integer output
-  const bool small = HoWo < ((size_t)1 << 27) && P.acc_out == nullptr && P.out_scale == 1.0f;
+  const bool small = HoWo < ((size_t)1 << 27) && P.acc_out == nullptr;
   const bool relu = P.relu != 0;
   const bool plain = small && P.residual == nullptr, with_res = small && P.residual != nullptr;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -937,7 +937,6 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
           if (co + j < P.Co) {
             const float d = __int_as_float(r[j]);
             float v = __fmul_rn(__fmul_rn(d, kv), lds_f(S.alpha + (uint32_t)((co + j) * 4)));
-            if (P.out_scale != 1.0f) v = __fmul_rn(v, P.out_scale);
             if (P.residual) v += res[j];
             if (relu) v = fmaxf(v, 0.0f);
             P.out[o0 + (size_t)j * HoWo] = v;
@@ -1065,9 +1064,10 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // per-filter vectors of the epilogue, zero beyond C_out (one global round trip per CTA
-  // instead of one per 16 columns drained)
+  // instead of one per 16 columns drained); alpha carries the call's extra output factor
+  // (1 except in the passes of a k-bit convolution; a product with 1 is exact)
   for (int i = tid; i < P.vec_len; i += kThreads) {
-    reinterpret_cast<float *>(smem + P.off_vec)[i] = i < P.Co ? __ldg(P.alpha + i) : 0.0f;
+    reinterpret_cast<float *>(smem + P.off_vec)[i] = i < P.Co ? __fmul_rn(__ldg(P.alpha + i), P.out_scale) : 0.0f;
     if (kFuse && P.nscale != nullptr) {
       reinterpret_cast<float *>(smem + P.off_vec)[P.vec_len + i] = i < P.Co ? __ldg(P.nscale + i) : 0.0f;
       reinterpret_cast<float *>(smem + P.off_vec)[2 * P.vec_len + i] = i < P.Co ? __ldg(P.nshift + i) : 0.0f;

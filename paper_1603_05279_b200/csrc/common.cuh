@@ -15,7 +15,7 @@ struct ConvGeom {
 // What the BinConv epilogues do beyond Eq. 11's D K alpha (+ residual).
 struct EpiOpts {
   int relu;          // max(v, 0) on the stored value
-  float out_scale;   // v = D K alpha out_scale (1: as Eq. 11; other values take the general path)
+  float out_scale;   // v = D K (alpha out_scale); 1: as Eq. 11
   int acc_shift;     // acc_out receives D << acc_shift ...
   int acc_accum;     // ... added to what acc_out holds (1) or stored (0)
 };
@@ -122,6 +122,10 @@ cudaError_t launch_bwn_prepare(const float *x, const float *scale, const float *
 cudaError_t launch_bwn_conv(const uint16_t *x_stream, const uint32_t *wp, const float *alpha,
                             const float *residual, const ConvGeom &g, float *out, cudaStream_t st);
 cudaError_t read_status_bwn(int *status);
+// Measured rates of the tensor pipe (1-bit MACs of the mxf4 MMA per clock per SM) and of the
+// CUDA-core population count (popc per clock per SM) on the current device.  Synchronises.
+cudaError_t measure_pipe_peaks(double *mma_mac_per_clk_per_sm, double *popc_per_clk_per_sm,
+                               cudaStream_t st);
 // A one-warp kernel whose bounded wait expires (nothing signals its barrier).
 cudaError_t launch_wait_timeout_selftest(cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.

@@ -12,8 +12,11 @@ from . import workloads as wl
 class LayerBuffers:
     """All device tensors of one layer; inputs are filled by the caller."""
 
-    def __init__(self, shape, device="cuda", with_acc=False, with_bn=True):
+    def __init__(self, shape, device="cuda", with_acc=False, with_bn=True, variant="xnor", kbits=2):
+        """variant: "xnor" (the block of Eq. 11), "bwn" (real inputs, binary weights, Eq. 1) or
+        "kbit" (q_k activations with `kbits` bits in place of sign)."""
         s = shape
+        self.variant, self.kbits = variant, kbits
         self.shape = s
         self.desc = B.desc_of(s)
         self.x = torch.empty((s.N, s.C_in, s.H, s.W), dtype=torch.float32, device=device)
@@ -25,17 +28,35 @@ class LayerBuffers:
         self.out = B.alloc_out(self.desc, device=device)
         self.acc = B.alloc_out(self.desc, torch.int32, device) if with_acc else None
         self.residual = None
+        if variant == "bwn":
+            self.x_stream = B.alloc_bwn_input(self.desc, device)
+        elif variant == "kbit":
+            self.x_planes = torch.empty((kbits,) + tuple(self.x_packed.shape), dtype=torch.int32,
+                                        device=device)
 
     def binarize_weights(self, stream=None):
         B.xnor_binarize_weights(self.w, self.w_packed, self.alpha, stream)
 
     def binactiv(self, stream=None):
-        B.xnor_binactiv(self.x, self.bn_scale, self.bn_shift, self.desc, self.x_packed, self.A,
-                        self.K, stream)
+        if self.variant == "bwn":
+            B.xnor_bwn_prepare_input(self.x, self.bn_scale, self.bn_shift, self.desc, self.x_stream, stream)
+        elif self.variant == "kbit":
+            B.xnor_binactiv_kbit(self.x, self.bn_scale, self.bn_shift, self.desc, self.kbits,
+                                 self.x_planes, self.A, self.K, stream)
+        else:
+            B.xnor_binactiv(self.x, self.bn_scale, self.bn_shift, self.desc, self.x_packed, self.A,
+                            self.K, stream)
 
     def conv(self, stream=None):
-        B.xnor_conv2d_forward(self.x_packed, self.w_packed, self.alpha, self.K, self.residual,
-                              self.desc, self.out, self.acc, stream)
+        if self.variant == "bwn":
+            B.xnor_bwn_conv2d_forward(self.x_stream, self.w_packed, self.alpha, self.residual,
+                                      self.desc, self.out, stream)
+        elif self.variant == "kbit":
+            B.xnor_conv2d_forward_kbit(self.x_planes, self.kbits, self.w_packed, self.alpha, self.K,
+                                       self.residual, self.desc, self.out, self.acc, stream)
+        else:
+            B.xnor_conv2d_forward(self.x_packed, self.w_packed, self.alpha, self.K, self.residual,
+                                  self.desc, self.out, self.acc, stream)
 
     def forward(self, stream=None, with_weights=True):
         if with_weights:
