@@ -47,7 +47,9 @@ typedef enum {
   XNOR_ERR_INVALID_ARG = 1, /* null/misaligned pointer, non-positive size, k > H + 2 pad ... */
   XNOR_ERR_UNSUPPORTED = 2, /* a shape the kernels were not built for (see each call)       */
   XNOR_ERR_CUDA = 3,        /* the launch failed; the CUDA error was read and cleared        */
-  XNOR_ERR_TIMEOUT = 4      /* a bounded device-side wait gave up (see xnor_check_device)    */
+  XNOR_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up (see xnor_check_device)    */
+  XNOR_ERR_BOUNDS = 5       /* checking build only: a kernel computed an address outside its
+                               buffer; the access was skipped (see xnor_built_with_bounds_check) */
 } xnor_status;
 
 /* Geometry of one convolution layer.  Square or rectangular filters, one
@@ -76,6 +78,13 @@ typedef struct {
 
 /* Library version: major*10000 + minor*100 + patch. */
 int xnor_version(void);
+
+/* 1 when the library was compiled with -DXNOR_BOUNDS_CHECK, else 0.  In that build the
+ * tensor-core BinConv kernel compares every shared-memory address its producers compute and
+ * every global index its epilogue stores to with the extent of the buffer, skips an access that
+ * fails and records it; xnor_check_device then returns XNOR_ERR_BOUNDS (once).  The ordinary
+ * build carries none of these checks.  Meant for running the parity suite once over a change. */
+int xnor_built_with_bounds_check(void);
 
 /* Static, human-readable name of a status code. */
 const char *xnor_status_string(xnor_status s);
@@ -383,7 +392,8 @@ xnor_status xnor_measure_peaks(double *mma_mac_per_clk_per_sm, double *popc_per_
  * shared-memory barrier) is bounded; a wait that expires records
  * XNOR_ERR_TIMEOUT there, the kernel stops issuing work, releases its tensor
  * memory and returns, and the outputs of that launch are undefined.  Returns
- * XNOR_OK, XNOR_ERR_TIMEOUT (the word is then cleared) or XNOR_ERR_CUDA.
+ * XNOR_OK, XNOR_ERR_TIMEOUT (the word is then cleared), XNOR_ERR_CUDA or, from a
+ * checking build, XNOR_ERR_BOUNDS.
  */
 xnor_status xnor_check_device(void *cuda_stream);
 

@@ -11,13 +11,16 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libxnor.so")
+# XNOR_LIB selects another build of the same library in this directory (the checking build,
+# libxnor_check.so); nothing else is ever loaded.
+LIB_PATH = os.path.join(_HERE, os.path.basename(os.environ.get("XNOR_LIB", "libxnor.so")))
 
 XNOR_OK = 0
 XNOR_ERR_INVALID_ARG = 1
 XNOR_ERR_UNSUPPORTED = 2
 XNOR_ERR_CUDA = 3
 XNOR_ERR_TIMEOUT = 4
+XNOR_ERR_BOUNDS = 5
 
 XNOR_FLAG_RELU = 1
 XNOR_FLAG_K_VALID_TAPS = 2
@@ -31,7 +34,7 @@ XNOR_ENGINE_UMMA_PAIR = 5
 XNOR_ENGINE_UMMA_PAIR_STREAM = 6
 
 EXPORTS = [
-    "xnor_version", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
+    "xnor_version", "xnor_built_with_bounds_check", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
     "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
     "xnor_maxpool2d", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
@@ -65,6 +68,7 @@ def load():
     lib = ctypes.CDLL(LIB_PATH)
     vp, ci = ctypes.c_void_p, ctypes.c_int
     lib.xnor_version.restype = ci
+    lib.xnor_built_with_bounds_check.restype = ci
     lib.xnor_status_string.restype = ctypes.c_char_p
     lib.xnor_status_string.argtypes = [ci]
     lib.xnor_words_per_pixel.restype = ctypes.c_size_t
@@ -149,6 +153,10 @@ def desc_of(s):
 
 def xnor_version():
     return int(load().xnor_version())
+
+
+def xnor_built_with_bounds_check():
+    return int(load().xnor_built_with_bounds_check())
 
 
 def status_string(status):

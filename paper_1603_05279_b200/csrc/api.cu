@@ -32,7 +32,15 @@ xnor_status from_cuda(cudaError_t e) { return e == cudaSuccess ? XNOR_OK : XNOR_
 
 extern "C" {
 
-int xnor_version(void) { return 100; }
+int xnor_version(void) { return 200; }
+
+int xnor_built_with_bounds_check(void) {
+#ifdef XNOR_BOUNDS_CHECK
+  return 1;
+#else
+  return 0;
+#endif
+}
 
 const char *xnor_status_string(xnor_status s) {
   switch (s) {
@@ -41,6 +49,7 @@ const char *xnor_status_string(xnor_status s) {
     case XNOR_ERR_UNSUPPORTED: return "XNOR_ERR_UNSUPPORTED";
     case XNOR_ERR_CUDA: return "XNOR_ERR_CUDA";
     case XNOR_ERR_TIMEOUT: return "XNOR_ERR_TIMEOUT";
+    case XNOR_ERR_BOUNDS: return "XNOR_ERR_BOUNDS";
   }
   return "XNOR_ERR_UNKNOWN";
 }
@@ -275,6 +284,7 @@ xnor_status xnor_check_device(void *cuda_stream) {
     (void)cudaGetLastError();
     return XNOR_ERR_CUDA;
   }
+  if (st >= 1000) return XNOR_ERR_BOUNDS;
   return (st == 0 && st2 == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
 }
 

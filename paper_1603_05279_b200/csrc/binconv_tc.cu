@@ -70,6 +70,17 @@ namespace xnor {
 
 __device__ int g_status_tc = 0;
 
+// Checking build (-DXNOR_BOUNDS_CHECK): every shared-memory address a producer computes and
+// every global index the epilogue stores to is compared with the extent of its buffer; the
+// first violation is recorded (its site number) and the access is skipped, so nothing traps.
+// In the ordinary build in_bounds() is the constant true and its argument is never evaluated.
+#ifdef XNOR_BOUNDS_CHECK
+__device__ int g_bounds_tc = 0;
+#define in_bounds(cond, site) ((cond) ? true : (atomicCAS(&xnor::g_bounds_tc, 0, (site)), false))
+#else
+#define in_bounds(cond, site) true
+#endif
+
 namespace {
 
 using namespace umma;
@@ -524,6 +535,8 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
   uint32_t wph = wph0;        // parity to wait for on the empty barriers
   bool ok = true;
   const uint32_t row_off = (uint32_t)row * 16u + (uint32_t)(2 * jj0) * b_lbo;
+  const uint32_t ring_end = S.ring + (uint32_t)P.stages * P.stage_bytes;
+  (void)ring_end;
 #pragma unroll 1
   while (cc.item < i1 && ok) {
     ok = mbar_wait_relaxed(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_tc, XNOR_SLEEP_WGT);
@@ -546,8 +559,10 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
         expand_signs<false>(pf[0][u].y, v1);
         const uint32_t a = stage + (uint32_t)(2 * u) * b_lbo;
         const uint32_t sw = (kSwap && ((sbits >> u) & 1u)) ? b_lbo : 0u;
-        sts128(a + sw, v0[0], v0[1], v0[2], v0[3]);
-        sts128(a + b_lbo - sw, v1[0], v1[1], v1[2], v1[3]);
+        if (in_bounds(a >= S.ring && a + b_lbo + 16u <= ring_end, 1)) {
+          sts128(a + sw, v0[0], v0[1], v0[2], v0[3]);
+          sts128(a + b_lbo - sw, v1[0], v1[1], v1[2], v1[3]);
+        }
       }
     } else if (on) {
 #pragma unroll
@@ -561,8 +576,10 @@ __device__ bool weight_role(const TcParams &P, const Smem &S, long long nitems, 
           expand_signs<false>(pf[0][u].y, v1);
           v1[0] &= keep; v1[1] &= keep; v1[2] &= keep; v1[3] &= keep;
           const uint32_t a = stage + (uint32_t)(2 * u) * b_lbo;
-          sts128(swap ? a + b_lbo : a, v0[0], v0[1], v0[2], v0[3]);
-          sts128(swap ? a : a + b_lbo, v1[0], v1[1], v1[2], v1[3]);
+          if (in_bounds(a >= S.ring && a + b_lbo + 16u <= ring_end, 2)) {
+            sts128(swap ? a + b_lbo : a, v0[0], v0[1], v0[2], v0[3]);
+            sts128(swap ? a : a + b_lbo, v1[0], v1[1], v1[2], v1[3]);
+          }
         }
       }
     }
@@ -665,8 +682,9 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     const size_t a1 = min((b1 + 15) & ~(size_t)15, tensor_bytes & ~(size_t)15);
     const uint32_t bulk = a1 > a0 ? (uint32_t)(a1 - a0) : 0u;
     for (size_t b = a0 + bulk; b < b1; b += 4)           // at most 3 words, at the tensor's end
-      sts32(dst + (uint32_t)(b - a0), __ldg(P.xp + (b >> 2)));
-    if (bulk) {
+      if (in_bounds((uint32_t)(b - a0) + 4u <= P.raw_bytes, 3))
+        sts32(dst + (uint32_t)(b - a0), __ldg(P.xp + (b >> 2)));
+    if (bulk && in_bounds(bulk <= P.raw_bytes && a0 + bulk <= tensor_bytes, 4)) {
       mbar_arrive_expect_tx(bar, bulk);
       bulk_copy_g2s(dst, reinterpret_cast<const uint8_t *>(P.xp) + a0, bulk, bar);
     } else {
@@ -750,7 +768,8 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
 #pragma unroll
       for (int b = 0; b < 2; ++b) {
         wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
-        if (real[b]) {
+        if (real[b] && in_bounds(src[b] >= S.raw + rb * P.raw_bytes &&
+                                 src[b] + 4u * (uint32_t)min(4, P.Cw - w0[b]) <= S.raw + (rb + 1u) * P.raw_bytes, 6)) {
           if (vec) {
             lds128(src[b], wv[b]);
           } else {
@@ -774,7 +793,9 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
               if (tail && w0[b] + i == P.Cw - 1) {       // channels beyond C_in are 0
                 v0 &= tm[0]; v1 &= tm[1]; v2 &= tm[2]; v3 &= tm[3];
               }
-              sts128(dst[b] + (uint32_t)i * plane_bytes, v0, v1, v2, v3);
+              if (in_bounds(dst[b] + (uint32_t)i * plane_bytes >= patch &&
+                            dst[b] + (uint32_t)i * plane_bytes + 16u <= patch + P.patch_bytes, 5))
+                sts128(dst[b] + (uint32_t)i * plane_bytes, v0, v1, v2, v3);
             }
           }
         }
@@ -822,6 +843,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
   };
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t howo = (uint32_t)HoWo;
+  const size_t out_elems = (size_t)P.N * P.Co * HoWo;
+  (void)out_elems;
   // the fast store paths: offsets of 16 consecutive filters fit 32 bits, no integer output
   const bool small = HoWo < ((size_t)1 << 27) && P.acc_out == nullptr;
   const bool relu = P.relu != 0;
@@ -905,7 +928,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
           for (int jj = 0; jj < 4; ++jj)
           {
             const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
-            op[(uint32_t)(j4 * 4 + jj) * howo] = relu ? fmaxf(v, 0.0f) : v;
+            if (in_bounds(obase + (size_t)(co + j4 * 4 + jj) * HoWo < out_elems, 7))
+              op[(uint32_t)(j4 * 4 + jj) * howo] = relu ? fmaxf(v, 0.0f) : v;
           }
         }
       } else if (co + 16 <= P.Co && with_res) {
@@ -920,7 +944,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
             const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]) + res[j4 * 4 + jj];
-            *op = relu ? fmaxf(v, 0.0f) : v;
+            if (in_bounds((size_t)(op - P.out) < out_elems, 8)) *op = relu ? fmaxf(v, 0.0f) : v;
             op += HoWo;
           }
         }
@@ -939,7 +963,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
             float v = __fmul_rn(__fmul_rn(d, kv), lds_f(S.alpha + (uint32_t)((co + j) * 4)));
             if (P.residual) v += res[j];
             if (relu) v = fmaxf(v, 0.0f);
-            P.out[o0 + (size_t)j * HoWo] = v;
+            if (in_bounds(o0 + (size_t)j * HoWo < out_elems, 9)) P.out[o0 + (size_t)j * HoWo] = v;
             if (P.acc_out) {
               int32_t *ap = P.acc_out + o0 + (size_t)j * HoWo;
               *ap = (P.acc_accum ? *ap : 0) + (__float2int_rn(d) << P.acc_shift);
@@ -981,7 +1005,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
           float v = __fmul_rn(__fmul_rn(__int_as_float(r[j]), kv), a4[jj]);
           if (P.residual != nullptr) v += res[j];
           if (relu) v = fmaxf(v, 0.0f);
-          if (P.out != nullptr) op[(uint32_t)j * howo] = v;
+          if (P.out != nullptr && in_bounds(obase + (size_t)(co + j) * HoWo < out_elems, 10))
+            op[(uint32_t)j * howo] = v;
           const float y = P.nscale != nullptr ? __fmaf_rn(s4[jj], v, h4[jj]) : v;
           half |= (y >= 0.0f ? 1u : 0u) << j;
           if (jj == 0) as0 += fabsf(y);
@@ -1016,14 +1041,15 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
         if (co0 + b * 16 >= P.Co) continue;
         emit_fused(b, cur);
         if ((k & 1) && valid) {                  // the pair is complete: its word of the next input
-          P.xp_next[(obase_pix) * (size_t)P.Cw_next + (size_t)((co0 + b * 16) >> 5)] = word;
+          if (in_bounds(obase_pix < (size_t)P.N * HoWo && ((co0 + b * 16) >> 5) < P.Cw_next, 11))
+            P.xp_next[(obase_pix) * (size_t)P.Cw_next + (size_t)((co0 + b * 16) >> 5)] = word;
           word = 0u;
         }
       } else {
         emit(b, cur);
       }
     }
-    if (kFuse && valid)
+    if (kFuse && valid && in_bounds(obase_pix < (size_t)P.N * HoWo, 12))
       P.A_part[(size_t)(slab * esplit + e) * ((size_t)P.N * HoWo) + obase_pix] = (as0 + as1) + (as2 + as3);
     px = npx;
     tile = ntile;
@@ -1469,6 +1495,16 @@ cudaError_t read_status_tc(int *status) {
     const int zero = 0;
     e = cudaMemcpyToSymbol(g_status_tc, &zero, sizeof(int));
   }
+#ifdef XNOR_BOUNDS_CHECK
+  // checking build: a recorded violation wins over everything else (1000 + its site number)
+  int site = 0;
+  if (e == cudaSuccess) e = cudaMemcpyFromSymbol(&site, g_bounds_tc, sizeof(int));
+  if (e == cudaSuccess && site != 0) {
+    const int zero = 0;
+    e = cudaMemcpyToSymbol(g_bounds_tc, &zero, sizeof(int));
+    *status = 1000 + site;
+  }
+#endif
   return e;
 }
 
