@@ -290,8 +290,22 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   }
   const int sms = sm_count_of_current_device();
   const long long nbatches = ((total_pix + kPix - 1) / kPix + PG - 1) / PG;
-  const unsigned grid = (unsigned)(nbatches < 3ll * sms ? nbatches : 3ll * sms);   // 3 blocks fit an SM
   const bool v16 = ((g.H * g.W) & 3) == 0;
+  // persistent grid: as many blocks as are resident at once (the shared-memory split the driver
+  // picks for this kernel decides whether two or three fit an SM), so that no block waits for
+  // a second wave
+  const void *kern = scale ? (v16 ? (const void *)binactiv_pack_kernel<true, true>
+                                  : (const void *)binactiv_pack_kernel<true, false>)
+                           : (v16 ? (const void *)binactiv_pack_kernel<false, true>
+                                  : (const void *)binactiv_pack_kernel<false, false>);
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * kWarps, smem) != cudaSuccess ||
+      per_sm < 1) {
+    (void)cudaGetLastError();
+    per_sm = 2;
+  }
+  const long long resident = (long long)per_sm * sms;
+  const unsigned grid = (unsigned)(nbatches < resident ? nbatches : resident);
 #define XNOR_PACK(BN, V16) binactiv_pack_kernel<BN, V16><<<grid, 32 * kWarps, smem, st>>>( \
       x, scale, shift, total_pix, g.C, g.H * g.W, g.Cw, G, PG, x_packed, A)
   if (scale) { if (v16) XNOR_PACK(true, true); else XNOR_PACK(true, false); }
