@@ -41,7 +41,7 @@ POPC_PER_CLK_PER_SM = 16
 # DRAM traffic of the dominant kernel from one ncu capture: dram__bytes_read.sum +
 # dram__bytes_write.sum summed over the four BinConv launches of one step of the default
 # workload.  Valid only for the kernel source it was taken from (hash below); null otherwise.
-NCU_TRAFFIC = {"kernel_sha1": "2c5af8e4edf24572ab0755be0093681529d9235e", "bytes_per_step": 160.8e6}
+NCU_TRAFFIC = {"kernel_sha1": "1760ee56f190583d7bae6905d1a02dd9680c4dd9", "bytes_per_step": 147.9e6}
 
 
 def kernel_sha1():

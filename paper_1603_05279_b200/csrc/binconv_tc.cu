@@ -62,6 +62,7 @@
 //  otherwise the weights of every item pass through a ring of stages (items in
 //  tile-major order, so that a patch serves all slabs of its tile).
 #include <algorithm>
+#include <mutex>
 
 #include "common.cuh"
 #include "umma_common.cuh"
@@ -1350,7 +1351,7 @@ namespace {
 
 // The plan of a variant.  kTcAuto (measured on the AlexNet and ResNet-18 shapes): one CTA per
 // SM unless only a pair, each CTA holding half of a slab, can keep the filters resident.
-Plan plan_variant(const ConvGeom &g, TcVariant v, bool fuse = false) {
+Plan plan_variant_uncached(const ConvGeom &g, TcVariant v, bool fuse) {
   switch (v) {
     case kTcSingle: return make_plan(g, 0, false, fuse);
     case kTcSingleStream: return make_plan(g, 1, false, fuse);
@@ -1381,6 +1382,40 @@ cudaError_t launch_variant(const Plan &pl, unsigned units, cudaStream_t st) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, binconv_tc_kernel<kRes, kPair, kFuse>, pl.P);
+}
+
+}  // namespace
+
+// The last plans made, by (geometry, variant, fused): one call of the library plans its shape
+// two or three times (support check, then launch), and a network repeats a few shapes; planning
+// evaluates up to 800 descriptor words.  Plans hold no pointers until a launcher fills them in.
+namespace {
+
+struct PlanKey {
+  int N, C, H, W, Co, kh, kw, stride, pad, variant, fuse;
+  bool operator==(const PlanKey &o) const {
+    return N == o.N && C == o.C && H == o.H && W == o.W && Co == o.Co && kh == o.kh && kw == o.kw &&
+           stride == o.stride && pad == o.pad && variant == o.variant && fuse == o.fuse;
+  }
+};
+
+Plan plan_variant(const ConvGeom &g, TcVariant v, bool fuse = false) {
+  constexpr int kSlots = 16;
+  static std::mutex mu;
+  static PlanKey keys[kSlots];
+  static Plan plans[kSlots];
+  static bool used[kSlots] = {};
+  static int next = 0;
+  const PlanKey key{g.N, g.C, g.H, g.W, g.Co, g.kh, g.kw, g.stride, g.pad, (int)v, fuse ? 1 : 0};
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < kSlots; ++i)
+    if (used[i] && keys[i] == key) return plans[i];
+  const int slot = next;
+  next = (next + 1) % kSlots;
+  plans[slot] = plan_variant_uncached(g, v, fuse);
+  keys[slot] = key;
+  used[slot] = true;
+  return plans[slot];
 }
 
 }  // namespace
