@@ -4,7 +4,7 @@
 // The inputs are rounded once to bfloat16 and laid out as the "pixel stream" the XNOR kernel
 // uses (every input row preceded by lead zero pixels, every image by lead zero rows, one
 // stream per stride phase), but materialised in memory with the padding written as zeros:
-//   x_stream  bf16 [phases][L][Cp],  L = N*Hq*Wq stream positions, Cp = C rounded up to 16.
+//   x_stream  bf16 [phases][L][Cp],  L = N*Hq*Wq stream positions, Cp = C rounded up to 32.
 // With GEMM row m = stream position of an output pixel, tap (ky,kx) reads position
 // m + shift(ky,kx) of one phase: a CTA fetches the ppix = 128 + halo positions a tile touches
 // ONCE, with one TMA tile copy per phase and group of 8 channels (box = 8 channels x ppix
@@ -17,9 +17,10 @@
 // filter row).  tcgen05.mma kind::f16 (bf16 x bf16, fp32 accumulation in tensor memory): every
 // product is +-x exactly; only the fp32 accumulation rounds.
 //
-// Roles (448 threads, persistent, one CTA per SM, items = (pixel tile, filter slab) in tile-major
-// order, a contiguous range per CTA): warps 0-3 epilogue (D * alpha (+ residual) -> NCHW), warp 4
-// issues the MMAs, warp 5 issues the TMA copies, warps 6-13 expand weights.  Every wait is
+// Roles (576 threads, persistent, one CTA per SM, items = (pixel tile, filter slab) in tile-major
+// order, a contiguous range per CTA): warps 0-7 epilogue (D * alpha (+ residual) -> NCHW; two
+// warps per quarter of the lanes, taking alternate groups of 16 columns), warp 8 issues the MMAs,
+// warp 9 issues the TMA copies, warps 10-17 expand weights.  Every wait is
 // bounded; on expiry the CTA records XNOR_ERR_TIMEOUT, stops, and frees its tensor memory.
 #include <cuda.h>
 
@@ -36,11 +37,11 @@ namespace {
 
 using namespace umma;
 
-constexpr int kEpiWarps = 4;
-constexpr int kMmaWarp = 4;
-constexpr int kTmaWarp = 5;
-constexpr int kWgtWarp0 = 6, kWgtWarps = 8;
-constexpr int kThreads = 32 * (kWgtWarp0 + kWgtWarps);   // 448
+constexpr int kEpiWarps = 8;          // two per quarter of the tensor-memory lanes
+constexpr int kMmaWarp = 8;
+constexpr int kTmaWarp = 9;
+constexpr int kWgtWarp0 = 10, kWgtWarps = 8;
+constexpr int kThreads = 32 * (kWgtWarp0 + kWgtWarps);   // 576: 18 warps, 112 registers each
 constexpr int kTileM = 128;
 constexpr int kTmemCols = 512;
 constexpr int kMaxAcc = 4;
@@ -56,7 +57,7 @@ struct alignas(64) BwnParams {
   const float *alpha, *residual;
   float *out;
   int N, C, H, W, Co, kh, kw, stride, pad, Ho, Wo, Cw;
-  int Cp, cpt;                 // channels padded to 16; K-steps per tap = Cp / 16
+  int Cp, cpt;                 // channels padded to 32; K-steps per tap = Cp / 16 (even)
   int Hq, Wq, leadY, leadX;
   long long L;
   int ntiles, nslabs, NT, nacc, ppix, npb, stages, mps, nsteps, ntaps, phases;
@@ -116,6 +117,12 @@ __device__ __forceinline__ void tma_load_plane(uint32_t dst, const CUtensorMap *
       ::"r"(dst), "l"(tmap), "r"(0), "r"(group), "r"(pos), "r"(phase), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ float lds_f(uint32_t addr) {
   float v;
   asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
@@ -244,50 +251,75 @@ __device__ void tma_role(const BwnParams &P, const Smem &S, long long i0, long l
 }
 
 // ------------------------------------------------------------------ weight producers (8 warps)
-// Eight sign bits -> eight bfloat16 values +-1 (0x3F80 / 0xBF80), channel 2i in the low half
-// of register i.  A set bit is +1.
-__device__ __forceinline__ void expand_byte(uint32_t bits, uint32_t v[4]) {
-  const uint32_t inv = ~bits;
+// Byte kByte of a packed word (eight sign bits, a set bit is +1) -> eight bfloat16 values +-1
+// (0x3F80 / 0xBF80), channel 2i in the low half of register i.  `inv` is the complemented word:
+// its bit is the sign bit of the value.  Four operations per register, all shifts constant.
+template <int kByte>
+__device__ __forceinline__ void expand_byte(uint32_t inv, uint32_t v[4]) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
-    v[i] = 0x3F803F80u | (((inv >> (2 * i)) & 1u) << 15) | (((inv >> (2 * i + 1)) & 1u) << 31);
+  for (int i = 0; i < 4; ++i) {
+    constexpr int base = 8 * kByte;
+    const int p = base + 2 * i;                         // bit of the low value; p + 1 of the high one
+    const uint32_t lo = p <= 15 ? (inv << (15 - p)) : (inv >> (p - 15));
+    const uint32_t hi = inv << (30 - p);
+    v[i] = 0x3F803F80u | (lo & 0x8000u) | (hi & 0x80000000u);
+  }
 }
 
-// A stage holds mps K-steps of NT filter rows: piece (2 jj + half) of NT x 16 bytes.  K-step
-// j = tap * cpt + c16 takes bits 16 (c16 & 1) .. + 15 of packed word tap * Cw + c16 / 2 of the
-// filter.  Thread mapping: row = wt % rows_mod, the 256 / rows_mod groups split the K-steps.
+// A stage holds mps K-steps (mps / 2 packed words) of NT filter rows: piece (2 jj + half) of
+// NT x 16 bytes.  K-step j is bits 16 (j & 1) .. + 15 of packed word j >> 1 of the filter (the
+// channels are padded to whole words), so a word expands to four consecutive pieces.  Thread
+// mapping: row = wt % rows_mod, the 256 / rows_mod groups split the words of a stage (at most
+// two words per thread and stage).  The words of the NEXT stage are fetched before the current
+// one is expanded: the filters are re-read (from L2) for every work item.
 __device__ void weight_role(const BwnParams &P, const Smem &S, long long i0, long long i1, int wt,
                             int lane) {
+  constexpr int kMaxWords = 2;
   const int nst = (P.nsteps + P.mps - 1) / P.mps;
+  const int wps = P.mps >> 1, nwords = P.nsteps >> 1;   // words per stage, per filter row
   const int row = wt % P.rows_mod, grp = wt / P.rows_mod;
-  const int gs = P.grp_steps;
-  const bool grp_on = grp * gs < P.mps && row < P.NT;
+  const int wpt = P.grp_steps;                          // words per thread and stage (1 or 2)
+  const bool grp_on = grp * wpt < wps && row < P.NT;
   const uint32_t b_lbo = (uint32_t)P.NT * 16u;
+  auto fetch = [&](int st, int co, uint32_t w[kMaxWords]) {
+#pragma unroll
+    for (int u = 0; u < kMaxWords; ++u) {
+      const int wl = grp * wpt + u, f = st * wps + wl;
+      w[u] = 0u;
+      if (grp_on && u < wpt && wl < wps && f < nwords && co < P.Co)
+        w[u] = __ldg(P.wp + packed_weight_index(P.Co, co, f));
+    }
+  };
   int ws = 0;
   uint32_t wph = 1u;
   bool ok = true;
   int slab = (int)(i0 % P.nslabs);
+  uint32_t cur[kMaxWords], nxt[kMaxWords];
+  fetch(0, slab * P.NT + row, cur);
   for (long long it = i0; it < i1 && ok; ++it) {
-    const int co = slab * P.NT + row;
+    int nslab = slab + 1;
+    if (nslab == P.nslabs) nslab = 0;
     for (int st = 0; st < nst && ok; ++st) {
+      // the stage after this one: the next of this item, or the first of the next item
+#pragma unroll
+      for (int u = 0; u < kMaxWords; ++u) nxt[u] = 0u;
+      if (st + 1 < nst) fetch(st + 1, slab * P.NT + row, nxt);
+      else if (it + 1 < i1) fetch(0, nslab * P.NT + row, nxt);
       ok = mbar_wait_relaxed(S.wempty + 8u * ws, wph, S.abort_flag, &g_status_bwn, 50);
       if (!ok) break;
       if (grp_on) {
         const uint32_t stage = S.ring + (uint32_t)ws * P.stage_bytes + (uint32_t)row * 16u;
-        for (int u = 0; u < gs; ++u) {
-          const int jj = grp * gs + u, j = st * P.mps + jj;
-          if (jj < P.mps && j < P.nsteps) {
-            const int tap = j / P.cpt, c16 = j - tap * P.cpt;
-            const int f = tap * P.Cw + (c16 >> 1);
-            uint32_t w = 0u;
-            if (co < P.Co) w = __ldg(P.wp + packed_weight_index(P.Co, co, f));
-            const uint32_t half = (w >> (16 * (c16 & 1))) & 0xFFFFu;
-            uint32_t v0[4], v1[4];
-            expand_byte(half & 0xFFu, v0);
-            expand_byte(half >> 8, v1);
-            const uint32_t a = stage + (uint32_t)(2 * jj) * b_lbo;
-            sts128(a, v0[0], v0[1], v0[2], v0[3]);
-            sts128(a + b_lbo, v1[0], v1[1], v1[2], v1[3]);
+#pragma unroll
+        for (int u = 0; u < kMaxWords; ++u) {
+          const int wl = grp * wpt + u;
+          if (u < wpt && wl < wps && st * wps + wl < nwords) {
+            const uint32_t inv = ~cur[u];
+            const uint32_t a = stage + (uint32_t)(4 * wl) * b_lbo;       // pieces 4 wl .. 4 wl + 3
+            uint32_t v[4];
+            expand_byte<0>(inv, v); sts128(a, v[0], v[1], v[2], v[3]);
+            expand_byte<1>(inv, v); sts128(a + b_lbo, v[0], v[1], v[2], v[3]);
+            expand_byte<2>(inv, v); sts128(a + 2u * b_lbo, v[0], v[1], v[2], v[3]);
+            expand_byte<3>(inv, v); sts128(a + 3u * b_lbo, v[0], v[1], v[2], v[3]);
           }
         }
       }
@@ -295,17 +327,21 @@ __device__ void weight_role(const BwnParams &P, const Smem &S, long long i0, lon
       __syncwarp();
       if (lane == 0) mbar_arrive(S.wfull + 8u * ws);
       if (++ws == P.stages) { ws = 0; wph ^= 1u; }
+#pragma unroll
+      for (int u = 0; u < kMaxWords; ++u) cur[u] = nxt[u];
     }
-    if (++slab == P.nslabs) slab = 0;
+    slab = nslab;
   }
 }
 
-// ------------------------------------------------------------------ epilogue (4 warps)
-// Warp w reads tensor-memory lanes 32 w .. + 31 (stream positions) and all the slab's columns
-// (filters); for one filter a warp stores 32 consecutive pixels of the NCHW output.
+// ------------------------------------------------------------------ epilogue (8 warps)
+// A warp reads tensor-memory lanes 32 q .. + 31 (stream positions) of its quarter q and the
+// groups of 16 columns (filters) e, e + 2, ...; for one filter a warp stores 32 consecutive
+// pixels of the NCHW output.
 __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, long long i1,
-                              uint32_t tmem_base, int quarter, int lane) {
+                              uint32_t tmem_base, int quarter, int e, int lane) {
   const int b_end = P.NT / 16;
+  const int nk = (b_end - e + 1) / 2;                 // groups of this warp per item
   const size_t HoWo = (size_t)P.Ho * P.Wo;
   const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
   const bool relu = P.relu != 0;
@@ -338,14 +374,20 @@ __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, l
     const uint32_t t_acc = t_lane + (uint32_t)(ab * P.NT);
     const int co0 = slab * P.NT;
     int32_t nx[16], cur[16];
-    tmem_ld16(t_acc, nx);
+    if (nk > 0) tmem_ld16(t_acc + (uint32_t)(e * 16), nx);
+    else {                                       // a slab of 16 filters: nothing for the second warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
+    }
 #pragma unroll 1
-    for (int b = 0; b < b_end; ++b) {
+    for (int k = 0; k < nk; ++k) {
+      const int b = e + 2 * k;
       tmem_wait16(nx);
 #pragma unroll
       for (int j = 0; j < 16; ++j) cur[j] = nx[j];
-      if (b + 1 < b_end) {
-        tmem_ld16(t_acc + (uint32_t)((b + 1) * 16), nx);
+      if (k + 1 < nk) {
+        tmem_ld16(t_acc + (uint32_t)((b + 2) * 16), nx);
       } else {                                   // last load done: release the accumulator
         tc_fence_before();
         __syncwarp();
@@ -354,6 +396,22 @@ __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, l
       if (!px.valid) continue;
       const int co = co0 + b * 16;
       const size_t o0 = px.obase + (size_t)co * HoWo;
+      if (co + 16 <= P.Co && P.residual == nullptr && HoWo < ((size_t)1 << 27)) {
+        // whole group, no residual: 32-bit offsets from one pointer
+        float *op = P.out + o0;
+        const uint32_t howo = (uint32_t)HoWo;
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4) {
+          const float4 al = lds_f4(S.alpha + (uint32_t)(co * 4 + j4 * 16));
+          const float a4[4] = {al.x, al.y, al.z, al.w};
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const float v = __fmul_rn(__int_as_float(cur[j4 * 4 + jj]), a4[jj]);
+            op[(uint32_t)(j4 * 4 + jj) * howo] = relu ? fmaxf(v, 0.0f) : v;
+          }
+        }
+        continue;
+      }
       float res[16];
       if (P.residual != nullptr) {
 #pragma unroll
@@ -412,7 +470,7 @@ bwn_conv_kernel(const __grid_constant__ BwnParams P) {
   const long long i0 = total * blockIdx.x / gridDim.x;
   const long long i1 = total * (blockIdx.x + 1) / gridDim.x;
   if (i0 < i1) {
-    if (warp < kEpiWarps) epilogue_role(P, S, i0, i1, tmem_base, warp, lane);
+    if (warp < kEpiWarps) epilogue_role(P, S, i0, i1, tmem_base, warp & 3, warp >> 2, lane);
     else if (warp == kMmaWarp) mma_role(P, S, i0, i1, tmem_base);
     else if (warp == kTmaWarp) tma_role(P, S, i0, i1, lane);
     else weight_role(P, S, i0, i1, tid - 32 * kWgtWarp0, lane);
@@ -508,7 +566,7 @@ StreamGeom stream_geom(const ConvGeom &g) {
   const int Wd = std::max(std::max(Wc, g.Wo + q.dxmax - q.leadX), g.Wo);
   q.Hq = q.leadY + Hd; q.Wq = q.leadX + Wd;
   q.L = (long long)g.N * q.Hq * q.Wq;
-  q.Cp = (g.C + 15) / 16 * 16;
+  q.Cp = (g.C + 31) / 32 * 32;      // whole packed words: K-step j is half j & 1 of word j >> 1
   return q;
 }
 
@@ -564,9 +622,9 @@ BwnPlan make_plan(const ConvGeom &g) {
   int ntp = 16;
   while (ntp < P.NT) ntp *= 2;
   P.rows_mod = ntp;
-  const int groups = std::max(1, 32 * kWgtWarps / ntp);
-  P.mps = std::min(8, std::max(2, 4 * groups));
-  P.grp_steps = (P.mps + groups - 1) / groups;
+  const int groups = std::max(1, 32 * kWgtWarps / ntp);    // >= 2: slabs hold at most 128 filters
+  P.mps = 8;                                               // K-steps per stage = 4 packed words per row
+  P.grp_steps = std::max(1, (P.mps / 2) / groups);         // words per thread and stage: 2 or 1
   P.stage_bytes = (uint32_t)P.mps * (uint32_t)P.NT * 32u;
   P.off_vec = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
   P.vec_len = (g.Co + 15) / 16 * 16 + 256;
