@@ -61,6 +61,10 @@ struct alignas(64) BwnParams {
   int Hq, Wq, leadY, leadX;
   long long L;
   int ntiles, nslabs, NT, nacc, ppix, npb, stages, mps, nsteps, ntaps, phases;
+  int tpi;                     // pixel tiles per work item (1 or 2): every weight stage then serves
+                               // tpi MMAs, so the filter rows are expanded once per tpi * 128 pixels;
+                               // ntiles counts items' worth of tiles (groups of tpi stream tiles)
+  int nload, box_pos;          // TMA copies per operand plane of a patch and their extent in positions
   int rows_mod, grp_steps;
   uint32_t plane_bytes, phase_bytes, patch_bytes, stage_bytes;
   uint32_t off_vec, off_ring, off_patch;
@@ -183,7 +187,7 @@ __device__ void mma_loop(const BwnParams &P, const Smem &S, long long i0, long l
     ok = mbar_wait(S.aempty + 8u * ab, aph, S.abort_flag, &g_status_bwn);
     if (!ok) break;
     tc_fence_after();
-    const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.NT);
+    const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.tpi * P.NT);
     int tap = 0, c16 = 0;                    // K-step j = tap * cpt + c16
     for (int st = 0; st < nst && ok; ++st) {
       const int j0 = st * P.mps;
@@ -196,6 +200,11 @@ __device__ void mma_loop(const BwnParams &P, const Smem &S, long long i0, long l
         const uint32_t a_lo = ((patch_lo + P.tap_lo[tap] + (uint32_t)c16 * a_step) & 0x3FFFu) | a_lbo_hi;
         umma_bf16(d_tmem, a_lo, desc_hi, b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc,
                   (j0 + jj) == 0 ? 0u : 1u);
+        // the item's second pixel tile: the same patch 128 positions (128 x 16 bytes) further,
+        // the same filter rows, the next accumulator
+        if (P.tpi == 2)
+          umma_bf16(d_tmem + (uint32_t)P.NT, a_lo + (uint32_t)kTileM, desc_hi,
+                    b_lo + (uint32_t)jj * b_step, desc_hi, P.idesc, (j0 + jj) == 0 ? 0u : 1u);
         if (++c16 == P.cpt) { c16 = 0; ++tap; }
       }
       commit_one(S.wempty + 8u * ws);
@@ -231,12 +240,14 @@ __device__ void tma_role(const BwnParams &P, const Smem &S, long long i0, long l
       const uint32_t bar = S.pfull + 8u * pb;
       const uint32_t dst = S.patch + pb * P.patch_bytes;
       mbar_arrive_expect_tx(bar, P.patch_bytes);
-      const int pos = (tile0 + (int)seq) * kTileM;
+      const int pos = (tile0 + (int)seq) * P.tpi * kTileM;
       const int ngroups = P.Cp / 8;
       for (int ph = 0; ph < P.phases; ++ph)
         for (int g8 = 0; g8 < ngroups; ++g8)
-          tma_load_plane(dst + (uint32_t)ph * P.phase_bytes + (uint32_t)g8 * P.plane_bytes, &P.tmap, g8,
-                         pos, ph, bar);
+          for (int ld = 0; ld < P.nload; ++ld)
+            tma_load_plane(dst + (uint32_t)ph * P.phase_bytes + (uint32_t)g8 * P.plane_bytes +
+                               (uint32_t)(ld * P.box_pos) * 16u,
+                           &P.tmap, g8, pos + ld * P.box_pos, ph, bar);
     }
     started = seq + 1u;
   }
@@ -362,7 +373,6 @@ __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, l
     }
     return px;
   };
-  Pix px = decode(tile);
   int ab = 0;
   uint32_t fph = 0;
   bool ok = true;
@@ -371,15 +381,18 @@ __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, l
     ok = mbar_wait_relaxed(S.afull + 8u * ab, fph, S.abort_flag, &g_status_bwn, 200);
     if (!ok) break;
     tc_fence_after();
-    const uint32_t t_acc = t_lane + (uint32_t)(ab * P.NT);
     const int co0 = slab * P.NT;
-    int32_t nx[16], cur[16];
-    if (nk > 0) tmem_ld16(t_acc + (uint32_t)(e * 16), nx);
-    else {                                       // a slab of 16 filters: nothing for the second warp
+    if (nk == 0) {                               // a slab of 16 filters: nothing for the second warp
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
     }
+   for (int tt = 0; tt < P.tpi && nk > 0; ++tt) {   // the item's pixel tiles, one accumulator each
+    const Pix px = decode(tile * P.tpi + tt);
+    const bool last_tile = tt + 1 == P.tpi;
+    const uint32_t t_acc = t_lane + (uint32_t)((ab * P.tpi + tt) * P.NT);
+    int32_t nx[16], cur[16];
+    tmem_ld16(t_acc + (uint32_t)(e * 16), nx);
 #pragma unroll 1
     for (int k = 0; k < nk; ++k) {
       const int b = e + 2 * k;
@@ -388,7 +401,7 @@ __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, l
       for (int j = 0; j < 16; ++j) cur[j] = nx[j];
       if (k + 1 < nk) {
         tmem_ld16(t_acc + (uint32_t)((b + 2) * 16), nx);
-      } else {                                   // last load done: release the accumulator
+      } else if (last_tile) {                    // last load of the item done: release its accumulators
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(S.aempty + 8u * ab);
@@ -427,7 +440,8 @@ __device__ void epilogue_role(const BwnParams &P, const Smem &S, long long i0, l
         }
       }
     }
-    if (++slab == P.nslabs) { slab = 0; ++tile; if (it + 1 < nitems) px = decode(tile); }
+   }
+    if (++slab == P.nslabs) { slab = 0; ++tile; }
     if (++ab == P.nacc) { ab = 0; fph ^= 1u; }
   }
 }
@@ -605,19 +619,13 @@ BwnPlan make_plan(const ConvGeom &g) {
   P.phases = q.phases;
   P.ntaps = g.kh * g.kw;
   P.nsteps = P.ntaps * P.cpt;
-  P.ntiles = (int)((q.L + kTileM - 1) / kTileM);
   const int halo = (q.dymax - q.dymin) * q.Wq + (q.dxmax - q.dxmin);
-  P.ppix = (kTileM + halo + 7) / 8 * 8;
-  if (P.ppix > 256) return pl;                            // TMA box extent
-  if (q.L + P.ppix + 2 * kTileM >= (1ll << 31)) return pl;
-  P.plane_bytes = (uint32_t)P.ppix * 16u;
-  P.phase_bytes = P.plane_bytes * (uint32_t)(P.Cp / 8);
-  P.patch_bytes = P.phase_bytes * (uint32_t)P.phases;
+  if ((kTileM + halo + 7) / 8 * 8 > 256) return pl;        // a tile's window: at most one TMA box
+  if (q.L + 4 * kTileM + 256 >= (1ll << 31)) return pl;
   // filter slabs: as few as fit two accumulators into the tensor-memory columns
   const int max_nt = 128;
   P.nslabs = (g.Co + max_nt - 1) / max_nt;
   P.NT = ((g.Co + P.nslabs - 1) / P.nslabs + 15) / 16 * 16;
-  P.nacc = std::max(1, std::min(kMaxAcc, kTmemCols / P.NT));
   // weight stages: rows_mod threads cover the rows, the other groups split a stage's K-steps
   int ntp = 16;
   while (ntp < P.NT) ntp *= 2;
@@ -629,7 +637,23 @@ BwnPlan make_plan(const ConvGeom &g) {
   P.off_vec = (uint32_t)((kCtrlBytes + 127) / 128 * 128);
   P.vec_len = (g.Co + 15) / 16 * 16 + 256;
   P.off_ring = (uint32_t)((P.off_vec + (size_t)P.vec_len * 4 + 127) / 128 * 128);
-  if (P.off_ring + 2 * (size_t)P.stage_bytes + P.patch_bytes > kSmemMax) return pl;
+  // Two pixel tiles per work item when their common window (256 + halo positions) fits beside two
+  // weight stages: the expansion of the filter rows, which bounds the kernel, is then shared by
+  // two MMAs.  The window is fetched with one or two TMA copies per operand plane (box <= 256).
+  const int stream_tiles = (int)((q.L + kTileM - 1) / kTileM);
+  for (P.tpi = (kTmemCols / P.NT >= 2 && stream_tiles >= 2) ? 2 : 1; P.tpi >= 1; --P.tpi) {
+    P.ppix = (P.tpi * kTileM + halo + 7) / 8 * 8;
+    P.nload = P.ppix > 256 ? 2 : 1;
+    if (P.nload == 2) P.ppix = (P.ppix + 15) / 16 * 16;   // two boxes of a multiple of 8 positions
+    P.box_pos = P.ppix / P.nload;
+    P.plane_bytes = (uint32_t)P.ppix * 16u;
+    P.phase_bytes = P.plane_bytes * (uint32_t)(P.Cp / 8);
+    P.patch_bytes = P.phase_bytes * (uint32_t)P.phases;
+    if (P.off_ring + 2 * (size_t)P.stage_bytes + P.patch_bytes <= kSmemMax) break;
+  }
+  if (P.tpi < 1) return pl;
+  P.ntiles = (stream_tiles + P.tpi - 1) / P.tpi;
+  P.nacc = std::max(1, std::min(kMaxAcc, kTmemCols / (P.NT * P.tpi)));
   const size_t avail = kSmemMax - P.off_ring;
   int stages = 2, npb = 1;
   auto fits = [&](int st, int pb) { return (size_t)st * P.stage_bytes + (size_t)pb * P.patch_bytes <= avail; };
@@ -694,7 +718,7 @@ cudaError_t launch_bwn_conv(const uint16_t *x_stream, const uint32_t *wp, const 
   if (encode == nullptr) return cudaErrorNotSupported;
   const cuuint64_t dims[4] = {8, (cuuint64_t)(P.Cp / 8), (cuuint64_t)P.L, (cuuint64_t)P.phases};
   const cuuint64_t strides[3] = {16, (cuuint64_t)P.Cp * 2, (cuuint64_t)P.L * P.Cp * 2};
-  const cuuint32_t box[4] = {8, 1, (cuuint32_t)P.ppix, 1};
+  const cuuint32_t box[4] = {8, 1, (cuuint32_t)P.box_pos, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   if (encode(&P.tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t *>(x_stream), dims,
              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
