@@ -499,13 +499,22 @@ bwn_conv_kernel(const __grid_constant__ BwnParams P) {
 // ------------------------------------------------------------------ input preparation
 // fp32 NCHW (after the optional BatchNorm affine) -> bf16 stream [phase][position][Cp], zeros at
 // padding positions and in channels C .. Cp - 1.  A block handles 32 consecutive stream
-// positions of one phase for all channels: reads run along the positions (consecutive input
-// pixels), writes along the channels; the 32 x 32 transposition goes through shared memory.
+// positions of one phase, 64 channels at a time: reads run along the positions (consecutive
+// input pixels, eight loads per thread in flight), writes along the channels (a lane packs two
+// channels, a warp writes the 128 bytes of a position); the transposition goes through shared
+// memory.
+__device__ __forceinline__ uint32_t bf16_rne(float v) {
+  // round to nearest even on the bit pattern (NaN and infinity pass through truncated)
+  uint32_t u = __float_as_uint(v);
+  if ((u & 0x7F800000u) != 0x7F800000u) u += 0x7FFFu + ((u >> 16) & 1u);
+  return u >> 16;
+}
+
 __global__ void __launch_bounds__(256)
 bwn_prepare_kernel(const float *__restrict__ x, const float *__restrict__ scale,
                    const float *__restrict__ shift, int N, int C, int H, int W, int s, int Hq, int Wq,
                    int leadY, int leadX, long long L, int Cp, uint16_t *__restrict__ xs) {
-  __shared__ float tile[32][33];
+  __shared__ float tile[64][33];
   const int lane = threadIdx.x & 31, wy = threadIdx.x >> 5;      // 8 warps
   const long long nblk = (L + 31) / 32;
   const int phase = (int)(blockIdx.x / nblk);
@@ -525,29 +534,30 @@ bwn_prepare_kernel(const float *__restrict__ x, const float *__restrict__ scale,
     src = ((size_t)n * C * H + iy) * W + ix;
   }
   const size_t plane = (size_t)H * W;
-  uint16_t *dst = xs + ((size_t)phase * L + m0) * Cp;
-  for (int c0 = 0; c0 < Cp; c0 += 32) {
-    // warp wy reads channels c0 + wy, + 8, ... of the 32 positions
+  uint32_t *dst = reinterpret_cast<uint32_t *>(xs + ((size_t)phase * L + m0) * Cp);   // Cp is even
+  for (int c0 = 0; c0 < Cp; c0 += 64) {
+    // warp wy reads channels c0 + wy, + 8, ..., + 56 of the 32 positions
+    float v[8];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < 8; ++q) {
       const int ch = c0 + wy + 8 * q;
-      float v = 0.0f;
-      if (real && ch < C) {
-        v = __ldg(x + src + (size_t)ch * plane);
-        if (scale != nullptr) v = __fmaf_rn(__ldg(scale + ch), v, __ldg(shift + ch));
-      }
-      tile[wy + 8 * q][lane] = v;
+      v[q] = (real && ch < C) ? __ldg(x + src + (size_t)ch * plane) : 0.0f;
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int ch = c0 + wy + 8 * q;
+      if (scale != nullptr && real && ch < C) v[q] = __fmaf_rn(__ldg(scale + ch), v[q], __ldg(shift + ch));
+      tile[wy + 8 * q][lane] = v[q];
     }
     __syncthreads();
-    // warp wy writes positions wy, wy + 8, ...: lane = channel
+    // warp wy writes positions wy, wy + 8, ...: lane = channels c0 + 2 lane, + 1
+    if (c0 + 2 * lane < Cp) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int pos = wy + 8 * q;
-      if (m0 + pos < L && c0 + lane < Cp) {
-        // round to nearest even bfloat16 on the bit pattern (finite inputs; NaN/inf pass through)
-        uint32_t u = __float_as_uint(tile[lane][pos]);
-        if ((u & 0x7F800000u) != 0x7F800000u) u += 0x7FFFu + ((u >> 16) & 1u);
-        dst[(size_t)pos * Cp + c0 + lane] = (uint16_t)(u >> 16);
+      for (int q = 0; q < 4; ++q) {
+        const int pos = wy + 8 * q;
+        if (m0 + pos < L)
+          dst[((size_t)pos * Cp + c0) / 2 + lane] =
+              bf16_rne(tile[2 * lane][pos]) | (bf16_rne(tile[2 * lane + 1][pos]) << 16);
       }
     }
     __syncthreads();
