@@ -278,14 +278,15 @@ xnor_status xnor_selftest_wait_timeout(void *cuda_stream) {
 }
 
 xnor_status xnor_check_device(void *cuda_stream) {
-  int st = 0, st2 = 0;
+  int st = 0, st2 = 0, st3 = 0;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess ||
-      xnor::read_status_tc(&st) != cudaSuccess || xnor::read_status_bwn(&st2) != cudaSuccess) {
+      xnor::read_status_tc(&st) != cudaSuccess || xnor::read_status_bwn(&st2) != cudaSuccess ||
+      xnor::read_status_act(&st3) != cudaSuccess) {
     (void)cudaGetLastError();
     return XNOR_ERR_CUDA;
   }
   if (st >= 1000) return XNOR_ERR_BOUNDS;
-  return (st == 0 && st2 == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
+  return (st == 0 && st2 == 0 && st3 == 0) ? XNOR_OK : XNOR_ERR_TIMEOUT;
 }
 
 xnor_status xnor_measure_peaks(double *mma_mac_per_clk_per_sm, double *popc_per_clk_per_sm,

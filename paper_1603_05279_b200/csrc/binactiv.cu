@@ -4,6 +4,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "umma_common.cuh"
 
 namespace xnor {
 
@@ -184,6 +185,244 @@ binactiv_pack_kernel(const float *__restrict__ x, const float *__restrict__ scal
   asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
+// ---------------------------------------------------------------------------
+// Whole-image variant for planes whose size is not a multiple of four pixels.  There a
+// channel's 128-byte run of 32 pixels starts on a 4-byte boundary only, and fetching the
+// runs one by one is bounded by the number of memory instructions, not by HBM.  An image
+// (C x H x W floats) is contiguous and, with C % 4 == 0, starts on a 16-byte boundary: a block
+// streams it as chunks of `cc` whole channel planes with one bulk copy each (a dedicated warp
+// issues them, `nbuf` chunks deep, also across images), and the eight consumer warps pack out
+// of shared memory: unit = (group of 32 pixels, 8 channels), lane = pixel, so the eight
+// values of a lane are `H W` words apart (no bank conflicts).  A unit yields one byte of the
+// packed words and a partial sum of |y|.  The pixel groups (and, on small planes, the channel
+// blocks) of a warp are the same for every chunk, so a lane keeps the |y| sums of its pixels in
+// registers through the whole image: no atomics, a fixed order.  At the end of an image the
+// block has A of the whole image in shared memory, so K (the box filter of A) is computed
+// here too, and the packed words leave as one contiguous run.
+constexpr int kImgWarps = 16;
+constexpr int kImgThreads = 32 * (kImgWarps + 1);
+constexpr int kImgMaxBufs = 4;
+constexpr int kImgRounds = 4;                    // pixel groups per warp: planes of up to 1024 pixels
+
+__device__ int g_status_act = 0;
+
+struct ImgParams {
+  const float *x, *scale, *shift;
+  uint32_t *x_packed;
+  float *A, *K;
+  int N, C, H, W, Cw;
+  int cc, nbuf;                    // channels per chunk (multiple of 8, divides C), chunks in flight
+  uint32_t chunk_bytes;            // cc * H * W * 4, a multiple of 16
+  uint32_t off_buf, off_words, off_apart, off_aimg, off_bn;   // byte offsets in shared memory
+  int kh, kw, stride, pad, Ho, Wo, valid_taps;
+};
+
+__device__ __forceinline__ float lds_f(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+
+// Barrier over the consumer warps with a bounded wait (a plain bar.sync would wait for ever
+// for a warp that gave up).
+__device__ __forceinline__ bool img_sync(uint32_t bar, uint32_t &phase, int lane, volatile int *abort_flag) {
+  __syncwarp();
+  if (lane == 0) umma::mbar_arrive(bar);
+  const bool ok = umma::mbar_wait(bar, phase, abort_flag, &g_status_act);
+  phase ^= 1u;
+  return __all_sync(0xFFFFFFFFu, ok);
+}
+
+template <bool kHasBN, int KS>
+__global__ void __launch_bounds__(kImgThreads, 2)
+binactiv_image_kernel(const __grid_constant__ ImgParams P) {
+  using namespace umma;
+  extern __shared__ __align__(128) uint8_t smem_img[];
+  // [0, 64): full barriers, [64, 128): empty barriers, 128: consumer barrier, 136: abort flag
+  const uint32_t base = smem_u32(smem_img);
+  const uint32_t full = base, empty = base + 8u * kImgMaxBufs, cbar = base + 16u * kImgMaxBufs;
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_img + 16 * kImgMaxBufs + 8);
+  uint8_t *wbytes = smem_img + P.off_words;                               // [HW][Cw * 4]
+  float *apart = reinterpret_cast<float *>(smem_img + P.off_apart);       // [warps per pixel group][HW]
+  float *aimg = reinterpret_cast<float *>(smem_img + P.off_aimg);         // [HW]
+  float2 *bn = reinterpret_cast<float2 *>(smem_img + P.off_bn);           // [C]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int HW = P.H * P.W, nsub = P.cc >> 3, nchunks = P.C / P.cc;
+  const int npg = (HW + 31) >> 5;
+
+  const int my_images = ((int)blockIdx.x < P.N) ? (P.N - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  const long long total = (long long)my_images * nchunks;
+  // producer state: next chunk to issue (image pn, chunk pch of it) into buffer pb
+  long long q = 0;
+  int pn = blockIdx.x, pch = 0, pb = 0;
+  uint32_t eph = 1u;                   // parity of an empty barrier's phase before its first completion
+  auto issue_chunk = [&]() {
+    const float *src = P.x + ((size_t)pn * P.C + (size_t)pch * P.cc) * HW;
+    mbar_arrive_expect_tx(full + 8u * pb, P.chunk_bytes);
+    bulk_copy_g2s(base + P.off_buf + (uint32_t)pb * P.chunk_bytes, src, P.chunk_bytes, full + 8u * pb);
+    if (++pch == nchunks) { pch = 0; pn += gridDim.x; }
+    if (++pb == P.nbuf) { pb = 0; eph ^= 1u; }
+  };
+  const bool producer = warp == kImgWarps && lane == 0;
+  if (producer) {
+    for (int i = 0; i < kImgMaxBufs; ++i) {
+      mbar_init(full + 8u * i, 1);
+      mbar_init(empty + 8u * i, kImgWarps);
+    }
+    mbar_init(cbar, kImgWarps);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // the first copies start before the rest of the block has set up: every buffer is free
+    for (; q < total && q < P.nbuf; ++q) issue_chunk();
+  }
+  // bytes of channels beyond C (C % 32 != 0) are never written by a unit: they stay zero
+  for (int i = tid; i < HW * P.Cw; i += kImgThreads) reinterpret_cast<uint32_t *>(wbytes)[i] = 0u;
+  if (kHasBN)
+    for (int c = tid; c < P.C; c += kImgThreads) bn[c] = make_float2(__ldg(P.scale + c), __ldg(P.shift + c));
+  __syncthreads();
+
+  if (warp == kImgWarps) {
+    // ---- producer: one thread issues every copy of this block
+    if (lane == 0) {
+      bool ok = true;
+      for (; q < total; ++q) {
+        ok = mbar_wait(empty + 8u * pb, eph, abort_flag, &g_status_act);
+        if (!ok) break;
+        issue_chunk();
+      }
+      if (!ok) {
+        // gave up: the copies already issued (at most one per buffer) must land before the
+        // block's shared memory is released
+        for (long long back = 1; back <= P.nbuf && back <= q; ++back) {
+          const long long c = q - back;
+          const uint32_t bar = full + 8u * (uint32_t)(c % P.nbuf), par = (uint32_t)(c / P.nbuf) & 1u;
+          for (int i = 0; i < (1 << 20) && !mbar_try(bar, par); ++i) {}
+        }
+      }
+    }
+    return;
+  }
+
+  // ---- consumers
+  // Warp -> (pixel groups, 8-channel blocks): with at least eight pixel groups a warp takes the
+  // groups warp, warp + 8, ... (at most kImgRounds) and every channel block; with fewer, the
+  // warps of a pixel group share the channel blocks (slot, slot + slots, ...).
+  const int slots = npg >= kImgWarps ? 1 : kImgWarps / npg;
+  const int pg0 = npg >= kImgWarps ? warp : warp % npg;
+  const int slot = npg >= kImgWarps ? 0 : warp / npg;
+  const bool has_work = slot < slots;
+  const int pstep = 32 * kImgWarps;
+  const uint32_t plane4 = (uint32_t)HW * 4u;
+  const uint32_t bn_addr = base + P.off_bn;
+  int b = 0;
+  uint32_t fph = 0u, cph = 0u;
+  for (int n = blockIdx.x; n < P.N; n += gridDim.x) {
+    float asum[kImgRounds];
+#pragma unroll
+    for (int r = 0; r < kImgRounds; ++r) asum[r] = 0.0f;
+    for (int ch = 0; ch < nchunks; ++ch) {
+      if (!mbar_wait(full + 8u * b, fph, abort_flag, &g_status_act)) return;
+      if (has_work) {
+        // 32-bit shared addresses: one add per load (the stride between channels is H W words)
+        const uint32_t buf = base + P.off_buf + (uint32_t)b * P.chunk_bytes + (uint32_t)(pg0 * 32 + lane) * 4u;
+        for (int sb = slot; sb < nsub; sb += slots) {
+          const int c0 = ch * P.cc + sb * 8;
+          float4 ss[4];                       // (scale, shift) of two channels per load
+          if (kHasBN) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ss[j] = lds_f4(bn_addr + (uint32_t)(c0 + 2 * j) * 8u);
+          }
+          uint32_t ta[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) ta[j] = buf + (uint32_t)(sb * 8 + j) * plane4;
+          uint8_t *wb = wbytes + (size_t)(pg0 * 32 + lane) * (P.Cw * 4) + (c0 >> 3);
+#pragma unroll
+          for (int r = 0; r < kImgRounds; ++r) {
+            if (pg0 * 32 + lane + r * pstep < HW) {
+              float y[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) y[j] = lds_f(ta[j] + (uint32_t)(r * pstep * 4));
+              uint32_t bits = 0u;
+              float p0 = 0.0f, p1 = 0.0f;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                float v = y[j];
+                if (kHasBN) v = (j & 1) ? __fmaf_rn(ss[j >> 1].z, v, ss[j >> 1].w) : __fmaf_rn(ss[j >> 1].x, v, ss[j >> 1].y);
+                if (v >= 0.0f) bits |= 1u << j;
+                if (j & 1) p1 += fabsf(v); else p0 += fabsf(v);
+              }
+              wb[(size_t)(r * pstep) * (P.Cw * 4)] = (uint8_t)bits;
+              asum[r] += p0 + p1;
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty + 8u * b);
+      if (++b == P.nbuf) { b = 0; fph ^= 1u; }
+    }
+    if (has_work) {
+#pragma unroll
+      for (int r = 0; r < kImgRounds; ++r)
+        if (pg0 * 32 + lane + r * pstep < HW) apart[slot * HW + pg0 * 32 + lane + r * pstep] = asum[r];
+    }
+    // the image is packed: A, the packed words, then K from the A just formed
+    if (!img_sync(cbar, cph, lane, abort_flag)) return;
+    for (int p = tid; p < HW; p += 32 * kImgWarps) {
+      float sum = 0.0f;
+      for (int s = 0; s < slots; ++s) sum += apart[s * HW + p];
+      const float a = sum / (float)P.C;
+      P.A[(size_t)n * HW + p] = a;
+      aimg[p] = a;
+    }
+    {
+      uint32_t *dst = P.x_packed + (size_t)n * HW * P.Cw;
+      const uint32_t *srcw = reinterpret_cast<const uint32_t *>(wbytes);
+      for (int i = tid; i < HW * P.Cw; i += 32 * kImgWarps) dst[i] = srcw[i];
+    }
+    if (!img_sync(cbar, cph, lane, abort_flag)) return;
+    const int HoWo = P.Ho * P.Wo;
+    for (int i = tid; i < HoWo; i += 32 * kImgWarps) {
+      const int oy = i / P.Wo, ox = i - oy * P.Wo;
+      const int y0 = oy * P.stride - P.pad, x0 = ox * P.stride - P.pad;
+      float s = 0.0f;
+      if (KS > 0) {
+        // square KS x KS filter: every tap a predicated load in straight-line code, summed in
+        // tap order (taps outside the image add zero)
+        float v[KS > 0 ? KS * KS : 1];
+#pragma unroll
+        for (int ky = 0; ky < KS; ++ky)
+#pragma unroll
+          for (int kx = 0; kx < KS; ++kx) {
+            const int iy = y0 + ky, ix = x0 + kx;
+            const bool in = iy >= 0 && iy < P.H && ix >= 0 && ix < P.W;
+            v[ky * KS + kx] = in ? aimg[iy * P.W + ix] : 0.0f;
+          }
+#pragma unroll
+        for (int t = 0; t < KS * KS; ++t) s += v[t];
+      } else {
+        const int ky0 = y0 < 0 ? -y0 : 0, ky1 = min(P.kh, P.H - y0);
+        const int kx0 = x0 < 0 ? -x0 : 0, kx1 = min(P.kw, P.W - x0);
+        for (int ky = ky0; ky < ky1; ++ky) {
+          const float *row = aimg + (y0 + ky) * P.W + x0;
+          for (int kx = kx0; kx < kx1; ++kx) s += row[kx];
+        }
+      }
+      int div = P.kh * P.kw;
+      if (P.valid_taps) {
+        const int ny = min(P.kh, P.H - y0) - max(0, -y0), nx = min(P.kw, P.W - x0) - max(0, -x0);
+        div = (ny > 0 && nx > 0) ? ny * nx : 0;
+      }
+      P.K[(size_t)n * HoWo + i] = div > 0 ? s / (float)div : 0.0f;
+    }
+  }
+}
+
 // K = box filter of zero-padded A.  One thread per output; blockIdx.y = image, so the index
 // arithmetic is 32-bit and cheap.  KS > 0: square KS x KS filter, every tap a predicated load
 // in straight-line code, so all of a thread's loads are in flight together (a loop with
@@ -258,7 +497,86 @@ bool pack_plan(const ConvGeom &g, bool bn, PackPlan *pl) {
   return pl->smem <= kPackSmemMax;
 }
 
+constexpr size_t kImgSmemMax = 112 * 1024;       // two blocks per SM
+constexpr uint32_t kImgHeader = 256;             // barriers and the abort flag
+
+// Whether the whole-image kernel serves this call, and with which chunking: planes that are
+// not a multiple of four pixels, whole bytes of packed channels, an image start on a 16-byte
+// boundary, enough images to occupy the SMs, and a chunk of at least eight channel planes
+// small enough that two (better four) of them fit beside the staged outputs of an image.
+bool image_plan(const ConvGeom &g, const float *x, bool bn, int sms, ImgParams *ip) {
+  const long long HW = (long long)g.H * g.W;
+  if ((HW & 3) == 0 || (g.C & 7) != 0 || (reinterpret_cast<uintptr_t>(x) & 15) != 0) return false;
+  if (g.N < sms / 2 || HW > 32 * kImgWarps * kImgRounds) return false;
+  const int npg = (int)((HW + 31) / 32);
+  const int slots = npg >= kImgWarps ? 1 : kImgWarps / npg;
+  for (int pass = 0; pass < 3; ++pass) {
+    const int nbuf = pass == 0 ? 4 : pass == 1 ? 3 : 2;
+    const long long chunk_max = pass == 0 ? 24 * 1024 : pass == 1 ? 32 * 1024 : 48 * 1024;
+    int cc = 0;
+    for (int c = 8; c <= g.C; c += 8)
+      if (g.C % c == 0 && (long long)c * HW * 4 <= chunk_max) cc = c;
+    if (cc == 0) continue;
+    const uint32_t chunk = (uint32_t)(cc * HW * 4);
+    uint32_t off = kImgHeader;
+    ip->off_buf = off; off += (uint32_t)nbuf * chunk;
+    ip->off_words = off; off += (uint32_t)(HW * g.Cw * 4);
+    ip->off_apart = off; off += (uint32_t)(slots * HW * 4);
+    ip->off_aimg = off; off += (uint32_t)(HW * 4);
+    off = (off + 15u) & ~15u;
+    ip->off_bn = off; off += bn ? (uint32_t)g.C * 8u : 0u;
+    if (off > kImgSmemMax) continue;
+    ip->cc = cc; ip->nbuf = nbuf; ip->chunk_bytes = chunk;
+    return true;
+  }
+  return false;
+}
+
+template <bool kHasBN, int KS>
+cudaError_t launch_image_variant(const ImgParams &ip, int sms, size_t smem, cudaStream_t st) {
+  static bool attr_flags[64] = {};
+  bool &attr_set = attr_done_for_current_device(attr_flags);
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(binactiv_image_kernel<kHasBN, KS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kImgSmemMax);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
+    attr_set = true;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, binactiv_image_kernel<kHasBN, KS>, kImgThreads,
+                                                    smem) != cudaSuccess || per_sm < 1) {
+    (void)cudaGetLastError();
+    per_sm = 1;
+  }
+  const long long resident = (long long)per_sm * sms;
+  const unsigned grid = (unsigned)(ip.N < resident ? ip.N : resident);
+  binactiv_image_kernel<kHasBN, KS><<<grid, kImgThreads, smem, st>>>(ip);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_binactiv_image(const ImgParams &ip, bool bn, int sms, cudaStream_t st) {
+  const size_t smem = (size_t)ip.off_bn + (bn ? (size_t)ip.C * 8 : 0);
+  const int ks = ip.kh == ip.kw ? ip.kh : 0;
+#define XNOR_IMG(KS) (bn ? launch_image_variant<true, KS>(ip, sms, smem, st) \
+                         : launch_image_variant<false, KS>(ip, sms, smem, st))
+  if (ks == 1) return XNOR_IMG(1);
+  if (ks == 3) return XNOR_IMG(3);
+  if (ks == 5) return XNOR_IMG(5);
+  if (ks == 7) return XNOR_IMG(7);
+  return XNOR_IMG(0);
+#undef XNOR_IMG
+}
+
 }  // namespace
+
+cudaError_t read_status_act(int *status) {
+  cudaError_t e = cudaMemcpyFromSymbol(status, g_status_act, sizeof(int));
+  if (e == cudaSuccess && *status != 0) {
+    const int zero = 0;
+    e = cudaMemcpyToSymbol(g_status_act, &zero, sizeof(int));
+  }
+  return e;
+}
 
 // Shapes the BinActiv kernels cover: the staged words fit shared memory (C_in <= 2976 with a
 // BatchNorm affine, more without) and one grid row per image.
@@ -273,6 +591,17 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   const long long total_pix = (long long)g.N * g.H * g.W;
   PackPlan pl;
   if (g.N > 65535 || !pack_plan(g, scale != nullptr, &pl)) return cudaErrorInvalidValue;
+  const int sms = sm_count_of_current_device();
+  {
+    ImgParams ip;
+    if (image_plan(g, x, scale != nullptr, sms, &ip)) {
+      ip.x = x; ip.scale = scale; ip.shift = shift; ip.x_packed = x_packed; ip.A = A; ip.K = K;
+      ip.N = g.N; ip.C = g.C; ip.H = g.H; ip.W = g.W; ip.Cw = g.Cw;
+      ip.kh = g.kh; ip.kw = g.kw; ip.stride = g.stride; ip.pad = g.pad; ip.Ho = g.Ho; ip.Wo = g.Wo;
+      ip.valid_taps = (g.flags & XNOR_FLAG_K_VALID_TAPS) ? 1 : 0;
+      return launch_binactiv_image(ip, scale != nullptr, sms, st);
+    }
+  }
   const int G = pl.G, PG = pl.PG;
   const size_t smem = pl.smem;
   static bool attr_flags[64] = {};
@@ -288,7 +617,6 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
     attr_set = true;
   }
-  const int sms = sm_count_of_current_device();
   const long long nbatches = ((total_pix + kPix - 1) / kPix + PG - 1) / PG;
   const bool v16 = ((g.H * g.W) & 3) == 0;
   // persistent grid: as many blocks as are resident at once (the shared-memory split the driver

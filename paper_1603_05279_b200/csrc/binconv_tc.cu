@@ -922,17 +922,23 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4)
           al[j4] = lds_f4(S.alpha + (uint32_t)(co * 4 + j4 * 16));
+        // the 16 products first, then the 16 stores (and the ReLU test once per group, not per
+        // value): two multiplies, an address and a store per output
+        float v[16];
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
-          const float a4[4] = {al[j4].x, al[j4].y, al[j4].z, al[j4].w};
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj)
-          {
-            const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]);
-            if (in_bounds(obase + (size_t)(co + j4 * 4 + jj) * HoWo < out_elems, 7))
-              op[(uint32_t)(j4 * 4 + jj) * howo] = relu ? fmaxf(v, 0.0f) : v;
-          }
+          v[j4 * 4 + 0] = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + 0]), kv), al[j4].x);
+          v[j4 * 4 + 1] = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + 1]), kv), al[j4].y);
+          v[j4 * 4 + 2] = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + 2]), kv), al[j4].z);
+          v[j4 * 4 + 3] = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + 3]), kv), al[j4].w);
         }
+        if (relu) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = fmaxf(v[j], 0.0f);
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (in_bounds(obase + (size_t)(co + j) * HoWo < out_elems, 7)) op[(uint32_t)j * howo] = v[j];
       } else if (co + 16 <= P.Co && with_res) {
         const float *rp = P.residual + obase + (size_t)co * HoWo;
         float res[16];

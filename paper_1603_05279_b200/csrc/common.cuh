@@ -130,6 +130,8 @@ cudaError_t measure_pipe_peaks(double *mma_mac_per_clk_per_sm, double *popc_per_
 cudaError_t launch_wait_timeout_selftest(cudaStream_t st);
 // Reads (and clears if set) the device status word of the tensor-core kernel.
 cudaError_t read_status_tc(int *status);
+// Same for the BinActiv kernel that waits on bulk copies.
+cudaError_t read_status_act(int *status);
 cudaError_t launch_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride, int pad,
                              bool relu, float *out, cudaStream_t st);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,

@@ -197,3 +197,47 @@ def test_binactiv_with_many_channels_and_pixels(oracle):
         X.xnor_binactiv(torch.empty((2, 4000, 8, 8), device="cuda"), torch.ones(4000, device="cuda"),
                         torch.zeros(4000, device="cuda"), big, *X.alloc_binactiv(big))
     assert e.value.status == B.XNOR_ERR_UNSUPPORTED
+
+
+# N, C, H, W, k, stride, pad, BatchNorm affine, flags
+IMAGE_PATH_SHAPES = [
+    (256, 96, 27, 27, 5, 1, 2, True, 0),            # AlexNet conv2's input: 8-channel chunks
+    (200, 384, 13, 13, 3, 1, 1, False, 0),          # conv4 / conv5: 32-channel chunks
+    (150, 40, 13, 13, 3, 2, 1, True, B.XNOR_FLAG_K_VALID_TAPS),   # a word with 8 channels only
+    (96, 512, 7, 7, 3, 1, 1, True, 0),              # ResNet's last stage
+    (80, 8, 31, 33, 7, 2, 3, True, 0),              # 1023 pixels: one chunk per image
+    (300, 24, 5, 9, 1, 1, 0, False, 0),             # more images than resident blocks
+]
+
+
+@pytest.mark.parametrize("shape", IMAGE_PATH_SHAPES)
+def test_binactiv_on_planes_of_odd_size_with_many_images(oracle, shape):
+    """Inputs whose planes are not a multiple of four pixels, with enough images to occupy the
+    GPU, go through the kernel that streams whole images with bulk copies and forms K in the same
+    launch: bits identical, A and K within tolerance, on the first, middle and last images and
+    on the one after the first round of blocks; nothing written outside the outputs."""
+    N, C, H, W, k, stride, pad, bn, flags = shape
+    g = np.random.Generator(np.random.Philox(sum(shape[:7])))
+    x = g.standard_normal((N, C, H, W), dtype=np.float32)
+    scale = (1.0 + 0.2 * g.standard_normal(C)).astype(np.float32) if bn else None
+    shift = (0.2 * g.standard_normal(C)).astype(np.float32) if bn else None
+    d = X.make_desc(N, C, H, W, 8, k, k, stride, pad, flags)
+    gs = GuardSet()
+    xp, A, K = (gs.like(n, t) for n, t in zip(("x_packed", "A", "K"), X.alloc_binactiv(d)))
+    xp.fill_(-1); A.fill_(float("nan")); K.fill_(float("nan"))
+    X.xnor_binactiv(dev(x), None if scale is None else dev(scale), None if shift is None else dev(shift),
+                    d, xp, A, K)
+    X.xnor_check_device()
+    gs.check()
+    assert bool(torch.isfinite(A).all()) and bool(torch.isfinite(K).all())
+    for n in sorted({0, 1, N // 2, min(N - 1, 296), N - 1}):
+        y = x[n:n + 1] if scale is None else oracle.bn_affine(x[n:n + 1], scale, shift)
+        assert np.array_equal(unpack_activations(host(xp[n:n + 1]), C), oracle.sign(y).reshape(y.shape)), n
+        A_or = oracle.channel_abs_mean(y)
+        assert_close(host(A[n:n + 1]), A_or, "A of image %d" % n)
+        K_or = (oracle.box_filter_valid_taps if flags & B.XNOR_FLAG_K_VALID_TAPS else oracle.box_filter)(
+            A_or, k, k, stride, pad)
+        assert_close(host(K[n:n + 1]), K_or, "K of image %d" % n)
+    # bits of channels beyond C_in in the last word are zero, as from the other BinActiv kernel
+    if C % 32:
+        assert int((xp[..., -1].to(torch.int64) & 0xFFFFFFFF).max()) < (1 << (C % 32))
