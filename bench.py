@@ -244,7 +244,7 @@ class LayersJob:
 
     def __init__(self, name, layer_ids, batch, rank, variant="xnor", kbits=2):
         import torch
-        from paper_1603_05279_b200.runner import LAUNCHES_PER_LAYER, LayerBuffers
+        from paper_1603_05279_b200.runner import LayerBuffers
         self.torch = torch
         shapes = [wl.scaled(wl.CONFIGS[name][i], batch) for i in layer_ids]
         self.shapes = shapes
@@ -257,10 +257,7 @@ class LayersJob:
             self.host_out.append(torch.empty(L.out.shape, dtype=torch.float32).pin_memory())
             L.x.copy_(self.host_x[-1])
             L.w.copy_(self.host_w[-1])
-        # kernels per layer: binarize 1, BinActiv 2 (pack, box filter), BinConv 1 (k-bit: one per
-        # plane; Binary-Weight: prepare 1, convolution 1)
-        per_layer = {"xnor": LAUNCHES_PER_LAYER, "bwn": 3, "kbit": 3 + kbits}[variant]
-        self.launches = per_layer * len(self.layers)
+        self.launches = sum(L.launches() for L in self.layers)
         self.macs = sum(wl.macs(s) for s in shapes)
         self.conv_macs = [wl.macs(s) for s in shapes]
         self.images = batch

@@ -147,6 +147,17 @@ xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn
                           void *cuda_stream);
 
 /*
+ * How many kernels xnor_binactiv launches for this call: 2 (pack + A, then the box
+ * filter for K) or 1.  One kernel serves inputs whose planes are not a multiple of
+ * four pixels (H*W % 4 != 0, at most 2048 pixels) when C_in % 8 == 0 and N is at least
+ * half the SM count: a block then streams whole images and forms K from the A it
+ * holds.  Both paths give the same bits; A (and K) may differ in the last place, the
+ * channel sums being taken in another order.  0 for a bad descriptor or a shape
+ * xnor_binactiv refuses.  has_bn != 0 = with bn_scale / bn_shift.
+ */
+int xnor_binactiv_launches(const xnor_conv_desc *d, int has_bn);
+
+/*
  * xnor_binactiv without a caller-supplied A buffer.  (The paper has no
  * counterpart; this exists for callers that cannot allocate.)
  *

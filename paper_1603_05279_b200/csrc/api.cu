@@ -224,6 +224,13 @@ bool good_desc(const xnor_conv_desc *d) {
 
 }  // namespace
 
+int xnor_binactiv_launches(const xnor_conv_desc *d, int has_bn) {
+  if (!good_desc(d)) return 0;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  if (!xnor::binactiv_supported(g, has_bn != 0)) return 0;
+  return xnor::binactiv_launch_count(g, has_bn != 0);
+}
+
 int xnor_conv2d_binactiv_parts(const xnor_conv_desc *d) {
   if (!good_desc(d) || current_engine() == XNOR_ENGINE_POPC || d->k_h > 11 || d->k_w > 11 ||
       (long long)d->C_in * d->k_h * d->k_w >= (1LL << 24))

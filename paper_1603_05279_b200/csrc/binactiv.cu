@@ -501,12 +501,12 @@ constexpr size_t kImgSmemMax = 112 * 1024;       // two blocks per SM
 constexpr uint32_t kImgHeader = 256;             // barriers and the abort flag
 
 // Whether the whole-image kernel serves this call, and with which chunking: planes that are
-// not a multiple of four pixels, whole bytes of packed channels, an image start on a 16-byte
-// boundary, enough images to occupy the SMs, and a chunk of at least eight channel planes
+// not a multiple of four pixels, whole bytes of packed channels (with the 16-byte alignment of
+// x that the entry point checks, every image then starts on a 16-byte boundary), enough images to occupy the SMs, and a chunk of at least eight channel planes
 // small enough that two (better four) of them fit beside the staged outputs of an image.
-bool image_plan(const ConvGeom &g, const float *x, bool bn, int sms, ImgParams *ip) {
+bool image_plan(const ConvGeom &g, bool bn, int sms, ImgParams *ip) {
   const long long HW = (long long)g.H * g.W;
-  if ((HW & 3) == 0 || (g.C & 7) != 0 || (reinterpret_cast<uintptr_t>(x) & 15) != 0) return false;
+  if ((HW & 3) == 0 || (g.C & 7) != 0) return false;
   if (g.N < sms / 2 || HW > 32 * kImgWarps * kImgRounds) return false;
   const int npg = (int)((HW + 31) / 32);
   const int slots = npg >= kImgWarps ? 1 : kImgWarps / npg;
@@ -569,6 +569,11 @@ cudaError_t launch_binactiv_image(const ImgParams &ip, bool bn, int sms, cudaStr
 
 }  // namespace
 
+int binactiv_launch_count(const ConvGeom &g, bool has_bn) {
+  ImgParams ip;
+  return image_plan(g, has_bn, sm_count_of_current_device(), &ip) ? 1 : 2;
+}
+
 cudaError_t read_status_act(int *status) {
   cudaError_t e = cudaMemcpyFromSymbol(status, g_status_act, sizeof(int));
   if (e == cudaSuccess && *status != 0) {
@@ -594,7 +599,7 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   const int sms = sm_count_of_current_device();
   {
     ImgParams ip;
-    if (image_plan(g, x, scale != nullptr, sms, &ip)) {
+    if (image_plan(g, scale != nullptr, sms, &ip)) {
       ip.x = x; ip.scale = scale; ip.shift = shift; ip.x_packed = x_packed; ip.A = A; ip.K = K;
       ip.N = g.N; ip.C = g.C; ip.H = g.H; ip.W = g.W; ip.Cw = g.Cw;
       ip.kh = g.kh; ip.kw = g.kw; ip.stride = g.stride; ip.pad = g.pad; ip.Ho = g.Ho; ip.Wo = g.Wo;

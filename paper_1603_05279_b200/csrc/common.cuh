@@ -132,6 +132,8 @@ cudaError_t launch_wait_timeout_selftest(cudaStream_t st);
 cudaError_t read_status_tc(int *status);
 // Same for the BinActiv kernel that waits on bulk copies.
 cudaError_t read_status_act(int *status);
+// Kernels launch_binactiv launches for this shape (1 or 2).
+int binactiv_launch_count(const ConvGeom &g, bool has_bn);
 cudaError_t launch_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride, int pad,
                              bool relu, float *out, cudaStream_t st);
 cudaError_t launch_shortcut_conv1x1(const float *x, const float *w, int N, int C, int H, int W,

@@ -65,12 +65,27 @@ class LayerBuffers:
         self.conv(stream)
 
     # algorithmic bytes, as the roofline of each kernel counts them
+    def binactiv_launches(self):
+        if self.variant == "bwn":
+            return 1
+        if self.variant == "kbit":
+            return 2
+        return B.xnor_binactiv_launches(self.desc, self.bn_scale is not None)
+
+    def launches(self):
+        """Kernels one forward() launches: binarize 1, BinActiv 1 or 2 (pack + A, box filter; one
+        kernel where a block streams whole images), BinConv 1 (k-bit: one per plane)."""
+        conv = self.kbits if self.variant == "kbit" else 1
+        return 1 + self.binactiv_launches() + conv
+
     def binactiv_bytes(self):
         s = self.shape
         ho, wo = wl.out_hw(s)
         cw = (s.C_in + 31) // 32
         px = s.N * s.H * s.W
-        return 4 * (px * s.C_in + px * cw + 2 * px + s.N * ho * wo)
+        # A is written once and, where K comes from a second kernel, read once
+        a_passes = 2 if self.binactiv_launches() == 2 else 1
+        return 4 * (px * s.C_in + px * cw + a_passes * px + s.N * ho * wo)
 
     def conv_bytes(self):
         s = self.shape
@@ -84,8 +99,6 @@ class LayerBuffers:
         return 4 * s.C_out * s.C_in * s.k * s.k
 
 
-# kernels launched by one forward(): binarize 1, binactiv 2 (pack, box filter), conv 1
-LAUNCHES_PER_LAYER = 4
 
 
 class ChainRunner:
@@ -223,8 +236,9 @@ class ChainRunner:
             self.run_layer(i, stream)
 
     def launches_per_forward(self):
-        # per layer: pack, box filter, conv; plus one kernel per projection shortcut
-        return 3 * len(self.layers) + len(self.proj)
+        # per layer: BinActiv (one or two kernels), conv; plus one kernel per projection shortcut
+        act = sum(B.xnor_binactiv_launches(L["desc"], True) for L in self.layers)
+        return act + len(self.layers) + len(self.proj)
 
     def macs(self):
         return sum(wl.macs(s) for s in self.shapes)

@@ -183,6 +183,7 @@ def test_binactiv_with_many_channels_and_pixels(oracle):
     d = X.make_desc(N, C, H, W, 8, 3, 3, 1, 1)
     gs = GuardSet()
     xp, A, K = (gs.like(n, t) for n, t in zip(("x_packed", "A", "K"), X.alloc_binactiv(d)))
+    assert X.xnor_binactiv_launches(d, True) == 2
     X.xnor_binactiv(dev(x), dev(scale), dev(shift), d, xp, A, K)
     gs.check()
     for n in (0, 100, 255):
@@ -225,11 +226,21 @@ def test_binactiv_on_planes_of_odd_size_with_many_images(oracle, shape):
     gs = GuardSet()
     xp, A, K = (gs.like(n, t) for n, t in zip(("x_packed", "A", "K"), X.alloc_binactiv(d)))
     xp.fill_(-1); A.fill_(float("nan")); K.fill_(float("nan"))
-    X.xnor_binactiv(dev(x), None if scale is None else dev(scale), None if shift is None else dev(shift),
-                    d, xp, A, K)
+    xd = dev(x)
+    sc, sh = (None, None) if scale is None else (dev(scale), dev(shift))
+    assert X.xnor_binactiv_launches(d, bn) == 1
+    X.xnor_binactiv(xd, sc, sh, d, xp, A, K)
     X.xnor_check_device()
     gs.check()
     assert bool(torch.isfinite(A).all()) and bool(torch.isfinite(K).all())
+    # a few images alone take the two-kernel path: same bits
+    d8 = X.make_desc(8, C, H, W, 8, k, k, stride, pad, flags)
+    assert X.xnor_binactiv_launches(d8, bn) == 2
+    xp2, A2, K2 = X.alloc_binactiv(d8)
+    X.xnor_binactiv(xd[N - 8:].contiguous(), sc, sh, d8, xp2, A2, K2)
+    assert torch.equal(xp2, xp[N - 8:])
+    assert_close(host(A2), host(A[N - 8:]), "A of the two paths")
+    assert_close(host(K2), host(K[N - 8:]), "K of the two paths")
     for n in sorted({0, 1, N // 2, min(N - 1, 296), N - 1}):
         y = x[n:n + 1] if scale is None else oracle.bn_affine(x[n:n + 1], scale, shift)
         assert np.array_equal(unpack_activations(host(xp[n:n + 1]), C), oracle.sign(y).reshape(y.shape)), n
