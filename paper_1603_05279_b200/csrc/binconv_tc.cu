@@ -393,6 +393,32 @@ __device__ __forceinline__ void issue_stage(const TcParams &P, int j0, uint32_t 
                       b_hi, P.idesc, tmem_sf, jj == 0 ? first : 1u);
 }
 
+// All MMAs of an item whose filter rows are already in shared memory (resident schedule, every
+// item but the first).  The stages of the ring are contiguous, so K-step j reads its filter
+// rows at b_lo0 + j b_step.  The patch descriptors of a batch of K-steps are fetched together
+// and the batch is issued in straight-line code: per MMA two additions and the instruction,
+// no load on its path (the stage-by-stage loop below needs ~100 cycles per MMA next to the
+// other roles, the tensor core 64).
+template <bool kPair>
+__device__ __forceinline__ void issue_item_flat(const TcParams &P, uint32_t d_tmem, uint32_t patch_lo,
+                                                uint32_t desc_hi, uint32_t b_lo0, uint32_t b_step,
+                                                uint32_t tmem_sf) {
+  constexpr int kBatch = 16;
+  uint32_t b = b_lo0;
+  for (int j0 = 0; j0 < P.nsteps; j0 += kBatch) {
+    uint32_t a[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) a[i] = j0 + i < P.nsteps ? P.adesc_lo[j0 + i] + patch_lo : 0u;
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      if (j0 + i < P.nsteps) {
+        umma_issue<kPair>(d_tmem, a[i], desc_hi, b, desc_hi, P.idesc, tmem_sf, (j0 + i) > 0 ? 1u : 0u);
+        b += b_step;
+      }
+    }
+  }
+}
+
 // kRes: resident schedule.  The stage barriers are then waited for only before the first item
 // (the CTA stays on one slab, which stays in shared memory) and never released.
 template <bool kRes, bool kPair>
@@ -428,6 +454,8 @@ __device__ void mma_loop(const TcParams &P, const Smem &S, long long i0, long lo
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + (uint32_t)(ab * P.NT);
     if (kRes) ws = 0;
+    if (kRes && !wait_stages) issue_item_flat<kPair>(P, d_tmem, patch_lo, desc_hi, b_lo0, b_step, tmem_sf);
+    else
     for (int st = 0; st < nst && ok; ++st) {
       const int j0 = st * P.mps;
       const int nj = min(P.mps, P.nsteps - j0);
@@ -911,8 +939,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
     Pix npx = px;
     if (next_new && it + 1 < nitems) npx = decode(ntile);
 
-    // Every store address is formed on its own from the group's base (no chain of pointer
-    // increments).
+    // Store addresses step from filter to filter by one multiply-add each (forming every
+    // address from the group's base takes two instructions per store and measured slower).
     auto emit = [&](int b, const int32_t r[16]) {
       if (!valid) return;
       const int co = co0 + b * 16;
@@ -936,14 +964,17 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] = fmaxf(v[j], 0.0f);
         }
+        // one address per store, each one multiply-add from the one before
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (in_bounds(obase + (size_t)(co + j) * HoWo < out_elems, 7)) op[(uint32_t)j * howo] = v[j];
+        for (int j = 0; j < 16; ++j) {
+          if (in_bounds(obase + (size_t)(co + j) * HoWo < out_elems, 7)) *op = v[j];
+          op += howo;
+        }
       } else if (co + 16 <= P.Co && with_res) {
         const float *rp = P.residual + obase + (size_t)co * HoWo;
         float res[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) res[j] = rp[(size_t)j * HoWo];
+        for (int j = 0; j < 16; ++j) { res[j] = *rp; rp += howo; }
 #pragma unroll
         for (int j4 = 0; j4 < 4; ++j4) {
           const float4 al = lds_f4(S.alpha + (uint32_t)(co * 4 + j4 * 16));
@@ -952,7 +983,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
           for (int jj = 0; jj < 4; ++jj) {
             const float v = __fmul_rn(__fmul_rn(__int_as_float(r[j4 * 4 + jj]), kv), a4[jj]) + res[j4 * 4 + jj];
             if (in_bounds((size_t)(op - P.out) < out_elems, 8)) *op = relu ? fmaxf(v, 0.0f) : v;
-            op += HoWo;
+            op += howo;
           }
         }
       } else {
@@ -994,7 +1025,7 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
       if (P.residual != nullptr) {
         const float *rp = P.residual + obase + (size_t)co * HoWo;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) res[j] = rp[(uint32_t)j * howo];
+        for (int j = 0; j < 16; ++j) { res[j] = *rp; rp += howo; }
       }
 #pragma unroll
       for (int j4 = 0; j4 < 4; ++j4) {
@@ -1012,8 +1043,8 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
           float v = __fmul_rn(__fmul_rn(__int_as_float(r[j]), kv), a4[jj]);
           if (P.residual != nullptr) v += res[j];
           if (relu) v = fmaxf(v, 0.0f);
-          if (P.out != nullptr && in_bounds(obase + (size_t)(co + j) * HoWo < out_elems, 10))
-            op[(uint32_t)j * howo] = v;
+          if (P.out != nullptr && in_bounds(obase + (size_t)(co + j) * HoWo < out_elems, 10)) *op = v;
+          op += howo;
           const float y = P.nscale != nullptr ? __fmaf_rn(s4[jj], v, h4[jj]) : v;
           half |= (y >= 0.0f ? 1u : 0u) << j;
           if (jj == 0) as0 += fabsf(y);
@@ -1025,19 +1056,16 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
       word |= half << (co & 16);              // C_out % 32 == 0: a group is the low or the high half
     };
 
-    // One copy of the code: the next 16 columns are being loaded into `nx` while the
-    // current 16 (copied out to `cur`) are scaled and stored.
-    int32_t nx[16], cur[16];
-    tmem_ld16(t_acc + (uint32_t)(group_of(0) * 16), nx);
+    // 16 columns at a time: load, wait, scale and store.  (Loading the next 16 during the
+    // stores of the current ones saves the ~50 cycles of a tensor-memory load per group but
+    // costs 16 register copies, which take longer here.)
+    int32_t cur[16];
 #pragma unroll 1
     for (int k = 0; k < nk; ++k) {
       const int b = group_of(k);
-      tmem_wait16(nx);
-#pragma unroll
-      for (int j = 0; j < 16; ++j) cur[j] = nx[j];
-      if (k + 1 < nk) {
-        tmem_ld16(t_acc + (uint32_t)(group_of(k + 1) * 16), nx);
-      } else {                                   // that was the last load: release the buffer
+      tmem_ld16(t_acc + (uint32_t)(b * 16), cur);
+      tmem_wait16(cur);
+      if (k + 1 == nk) {                         // that was the last load: release the buffer
         tc_fence_before();
         __syncwarp();
         if (lane == 0) { if (P.pair) mbar_arrive_cluster(S.aempty + 8u * ab, 0u); else mbar_arrive(S.aempty + 8u * ab); }
