@@ -112,6 +112,7 @@ constexpr int kMaxBarStages = 32;    // stage barriers (the resident schedule ha
 constexpr int kEpiSplitMax = 3;      // warps per lane quarter in the resident epilogue
 constexpr int kMaxPatchBufs = 4;
 constexpr int kMaxRaw = 6;            // raw buffers: up to 2 for each of up to 3 subgroups of patch warps
+constexpr int kPatUnits = 2;         // patch units a warp works on together
 constexpr int kMaxSteps = 800;       // K-steps (MMAs) per work item (< 1024: swap_mask)
 constexpr size_t kCtrlBytes = 1024;
 constexpr size_t kSmemMax = 232448 - 1024;
@@ -170,6 +171,8 @@ struct TcParams {
   int any_swap;                // some bit of swap_mask is set
   uint32_t div_wq_m, div_hq_m; // multipliers and shifts of the exact divisions by Wq and Hq
   int div_wq_s, div_hq_s;      // (dividends below 2^31)
+  uint32_t div_pg_m, div_g_m;  // the same for the patch units: by phases * ngrp and by ngrp
+  int div_pg_s, div_g_s;       // (ngrp = groups of four channel words)
 };
 
 // One MMA.  The issuing warp elects one lane, and that lane alone runs the whole issue loop:
@@ -764,18 +767,19 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
     const uint32_t m0 = ((uint32_t)tile * tmul + S.rank) * kTileM;
     const uint32_t raw = S.raw + rb * P.raw_bytes +
                          (uint32_t)(((size_t)g0 * row_bytes) & 15u);   // where row g0 starts
-    // two units per pass: their loads are issued together, then both are expanded
+    // kPatUnits units at a time: their index arithmetic and loads are independent chains the
+    // warp can overlap, then all are expanded
 #pragma unroll 1
-    for (int u0 = (int)mi; u0 < nunits; u0 += 2 * (int)gsize) {
-      uint32_t src[2], dst[2], sm[2], mc[2][3], wv[2][4];
-      int w0[2];
-      bool on[2], real[2];
+    for (int u0 = (int)mi; u0 < nunits; u0 += kPatUnits * (int)gsize) {
+      uint32_t src[kPatUnits], dst[kPatUnits], sm[kPatUnits], mc[kPatUnits][3], wv[kPatUnits][4];
+      int w0[kPatUnits];
+      bool on[kPatUnits], real[kPatUnits];
 #pragma unroll
-      for (int b = 0; b < 2; ++b) {
+      for (int b = 0; b < kPatUnits; ++b) {
         const int u = u0 + b * (int)gsize;
-        const int pass = u / (phases * ngrp);
+        const int pass = (int)fast_div((uint32_t)u, P.div_pg_m, P.div_pg_s);
         const int rem = u - pass * (phases * ngrp);
-        const int phase = rem / ngrp;
+        const int phase = (int)fast_div((uint32_t)rem, P.div_g_m, P.div_g_s);
         w0[b] = (rem - phase * ngrp) * 4;
         const int q = pass * 32 + lane;
         on[b] = u < nunits && q < P.ppix;
@@ -784,7 +788,7 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
         const int c = (int)(sq - r * (uint32_t)P.Wq);
         const uint32_t n = fast_div(r, P.div_hq_m, P.div_hq_s);
         const int ry = (int)(r - n * (uint32_t)P.Hq);
-        const int py = phase / s, px = phase - py * s;
+        const int py = phase >> (s - 1), px = phase & (s - 1);     // stride 1 or 2
         const int rrow = (ry - P.leadY) * s + py, rcol = (c - P.leadX) * s + px;
         real[b] = on[b] && sq < (uint32_t)P.L && ry >= P.leadY && c >= P.leadX && rrow < P.H &&
                   rcol < P.W;
@@ -795,7 +799,7 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
         dst[b] = patch + (uint32_t)(phase * P.Cw + w0[b]) * plane_bytes + (uint32_t)q * 16u;
       }
 #pragma unroll
-      for (int b = 0; b < 2; ++b) {
+      for (int b = 0; b < kPatUnits; ++b) {
         wv[b][0] = wv[b][1] = wv[b][2] = wv[b][3] = 0u;
         if (real[b] && in_bounds(src[b] >= S.raw + rb * P.raw_bytes &&
                                  src[b] + 4u * (uint32_t)min(4, P.Cw - w0[b]) <= S.raw + (rb + 1u) * P.raw_bytes, 6)) {
@@ -809,7 +813,7 @@ __device__ void patch_role(const TcParams &P, const Smem &S, long long i0, long 
         }
       }
 #pragma unroll
-      for (int b = 0; b < 2; ++b) {
+      for (int b = 0; b < kPatUnits; ++b) {
         if (on[b]) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -1375,6 +1379,9 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   };
   magic((uint32_t)P.Wq, &P.div_wq_m, &P.div_wq_s);
   magic((uint32_t)P.Hq, &P.div_hq_m, &P.div_hq_s);
+  const uint32_t ngrp = (uint32_t)(P.Cw + 3) / 4u;
+  magic((uint32_t)(s * s) * ngrp, &P.div_pg_m, &P.div_pg_s);
+  magic(ngrp, &P.div_g_m, &P.div_g_s);
   pl.ok = true;
   return pl;
 }
