@@ -24,6 +24,7 @@ from .binding import (  # noqa: F401
     scale_output_k,
     round_bf16,
     bwn_conv,
+    binary_gradient_backward,
     shortcut_conv1x1,
     maxpool2d,
     speedup_model,

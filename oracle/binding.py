@@ -224,6 +224,23 @@ def bwn_conv(x, B, alpha, stride, pad, residual=None):
     return out
 
 
+def binary_gradient_backward(g, B, alpha, pad, in_hw, round_products=False):
+    """Backward convolution with the gradient binarised to gmax * sign(g) and the filters
+    alpha * B (Section 3.2, "Binary Gradient"), stride 1.  g [N][Co][Ho][Wo], B [Co][C][kh][kw];
+    returns (gmax [N], gin [N][C][H][W])."""
+    g, alpha = _f32(g), _f32(alpha)
+    B = np.ascontiguousarray(B, dtype=np.int8)
+    N, Co, Ho, Wo = g.shape
+    Co2, C, kh, kw = B.shape
+    H, W = in_hw
+    assert Co == Co2 and Ho == out_extent(H, kh, 1, pad) and Wo == out_extent(W, kw, 1, pad)
+    gmax = np.empty((N,), np.float32)
+    gin = np.empty((N, C, H, W), np.float32)
+    _load().oracle_binary_gradient_backward(_p(g), _p(B), _p(alpha), *_i(N, C, H, W, Co, kh, kw, pad),
+                                            ctypes.c_int(1 if round_products else 0), _p(gmax), _p(gin))
+    return gmax, gin
+
+
 def shortcut_conv1x1(x, w, stride):
     x, w = _f32(x), _f32(w)
     N, C, H, W = x.shape

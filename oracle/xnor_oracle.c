@@ -23,7 +23,8 @@
  * Options beyond the main path (each a function of its own further down, all
  * pinned by the CPU tests): the border variant of K that divides by the taps
  * inside the image, ReLU on the block's output, k-bit activations q_k in place
- * of sign(), and the Binary-Weight-Network convolution of Eq. 1 on real inputs.
+ * of sign(), the Binary-Weight-Network convolution of Eq. 1 on real inputs, and
+ * the backward convolution with a binarised gradient.
  *
  * The only parallelism is an OpenMP "parallel for" over independent outer
  * indices (images, filters); loop bodies are unchanged by it.
@@ -403,6 +404,58 @@ void oracle_bwn_conv(const float *x, const int8_t *B, const float *alpha,
           double v = s * (double)alpha[co];
           if (residual) v += (double)residual[o];
           out[o] = (float)v;
+        }
+}
+
+/* Binary-gradient backward convolution, Section 3.2, "Binary Gradient".
+ * The backward pass of a layer convolves the gradient g that arrives at the
+ * convolution's output with the weight filters; as in Algorithm 1 the filters
+ * are the binarised ones, alpha * sign(W).  The gradient is binarised the way
+ * the forward operands are, sign(g), but scaled by max_i |g_i| instead of the
+ * mean of Eq. 6.  Readings where the paragraph is silent: the maximum is taken
+ * over one image's gradient tensor [Co][Ho][Wo] (images stay independent);
+ * sign(0) = +1 as everywhere; stride 1, zero padding.  Result: the gradient with
+ * respect to the convolution's input,
+ *   gin[n][c][y][x] = sum_{co,ky,kx} alpha[co] B[co][c][ky][kx] gmax[n]
+ *                                    sign(g[n][co][y + pad - ky][x + pad - kx]),
+ * taps outside the gradient's extent contributing 0.
+ * round_products != 0: every product gmax[n] * alpha[co] is formed in fp32 and
+ * rounded to bfloat16 before it enters the sum (the operand format of the
+ * tensor-core convolution that the library runs this on). */
+void oracle_binary_gradient_backward(const float *g, const int8_t *B, const float *alpha, int N,
+                                     int C, int H, int W, int Co, int kh, int kw, int pad,
+                                     int round_products, float *gmax, float *gin) {
+  const int Ho = out_extent(H, kh, 1, pad), Wo = out_extent(W, kw, 1, pad);
+  const size_t per_image = (size_t)Co * Ho * Wo;
+  for (int n = 0; n < N; ++n) {
+    float m = 0.0f;
+    for (size_t i = 0; i < per_image; ++i) {
+      const float a = fabsf(g[(size_t)n * per_image + i]);
+      if (a > m) m = a;
+    }
+    gmax[n] = m;
+  }
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int c = 0; c < C; ++c)
+      for (int y = 0; y < H; ++y)
+        for (int x = 0; x < W; ++x) {
+          double s = 0.0;
+          for (int co = 0; co < Co; ++co) {
+            float t = gmax[n] * alpha[co];
+            if (round_products) oracle_round_bf16(&t, 1, &t);
+            for (int ky = 0; ky < kh; ++ky)
+              for (int kx = 0; kx < kw; ++kx) {
+                const int oy = y + pad - ky, ox = x + pad - kx;
+                if (oy < 0 || oy >= Ho || ox < 0 || ox >= Wo) continue;
+                const float gv = g[(((size_t)n * Co + co) * Ho + oy) * Wo + ox];
+                const int sg = gv >= 0.0f ? 1 : -1;
+                const int b = B[(((size_t)co * C + c) * kh + ky) * kw + kx] > 0 ? 1 : -1;
+                if (sg * b > 0) s += (double)t;
+                else s -= (double)t;
+              }
+          }
+          gin[(((size_t)n * C + c) * H + y) * W + x] = (float)s;
         }
 }
 

@@ -242,3 +242,90 @@ def test_bwn_conv_special_cases(oracle):
     wc = np.where(g.random((2, 4, 3, 3)) < 0.5, -0.125, 0.125).astype(np.float32)
     Bc, ac = oracle.binarize_weights(wc)
     assert np.array_equal(oracle.bwn_conv(xc, Bc, ac, 1, 0), oracle.xnor_block(xc, wc, 1, 0).out)
+
+
+# --------------------------------------------------------------------------- binary gradient
+# N, C, H, W, Co, kh, kw, pad
+BGRAD_CASES = [(2, 5, 6, 7, 3, 3, 3, 1), (1, 33, 5, 4, 2, 3, 2, 1), (2, 4, 9, 8, 3, 5, 5, 2),
+               (2, 8, 5, 6, 3, 1, 1, 0), (3, 6, 7, 7, 4, 3, 3, 0), (1, 3, 6, 5, 2, 3, 3, 2)]
+
+
+@pytest.mark.parametrize("case", BGRAD_CASES)
+def test_binary_gradient_backward_is_the_library_gradient_of_the_binarised_convolution(oracle, case):
+    """With the gradient replaced by gmax * sign(g), the result is what automatic differentiation
+    gives for conv2d(x, alpha * B) with that upstream gradient (Section 3.2, "Binary Gradient";
+    Algorithm 1: the backward pass uses the binarised filters)."""
+    N, C, H, W, Co, kh, kw, p = case
+    g = rng(300 + sum(case))
+    w = g.standard_normal((Co, C, kh, kw)).astype(np.float32)
+    B, alpha = oracle.binarize_weights(w)
+    Ho, Wo = H + 2 * p - kh + 1, W + 2 * p - kw + 1
+    grad = g.standard_normal((N, Co, Ho, Wo)).astype(np.float32)
+    grad[0, 0, 0, 0] = 0.0                                            # sign(0) = +1
+    gmax, gin = oracle.binary_gradient_backward(grad, B, alpha, p, (H, W))
+    assert np.array_equal(gmax, np.abs(grad).reshape(N, -1).max(axis=1))
+    x = torch.zeros((N, C, H, W), dtype=torch.float64, requires_grad=True)
+    wt = torch.from_numpy(B).double() * torch.from_numpy(alpha).double()[:, None, None, None]
+    ghat = torch.from_numpy(np.where(grad >= 0, 1.0, -1.0)) * torch.from_numpy(gmax).double()[:, None, None, None]
+    ref, = torch.autograd.grad(F.conv2d(x, wt, padding=p), x, grad_outputs=ghat)
+    assert np.allclose(gin, ref.numpy(), rtol=1e-6, atol=1e-6 * float(np.abs(ref.numpy()).max()))
+
+
+def test_binary_gradient_backward_special_cases(oracle):
+    g = rng(310)
+    N, C, H, W, Co, k, p = 2, 4, 5, 6, 3, 3, 1
+    B = np.where(g.random((Co, C, k, k)) < 0.5, -1, 1).astype(np.int8)
+    alpha = np.array([0.5, 2.0, 0.25], np.float32)
+    grad = g.standard_normal((N, Co, H, W)).astype(np.float32)
+    gmax, gin = oracle.binary_gradient_backward(grad, B, alpha, p, (H, W))
+    # the scale is the largest magnitude, not the mean: one large entry sets it alone
+    big = grad.copy(); big[1, 2, 3, 3] = -50.0
+    gmax_b, gin_b = oracle.binary_gradient_backward(big, B, alpha, p, (H, W))
+    assert gmax_b[1] == 50.0 and gmax_b[0] == gmax[0] and np.array_equal(gin_b[0], gin[0])
+    # only the signs and the maximum of g matter: same signs, same maximum -> same result
+    other = np.sign(grad) * g.random(grad.shape).astype(np.float32) * gmax[:, None, None, None]
+    other = np.where(np.abs(grad) == gmax[:, None, None, None], grad, other).astype(np.float32)
+    assert np.array_equal(oracle.binary_gradient_backward(other, B, alpha, p, (H, W))[1], gin)
+    # scaling g by a power of two scales the result; negating g (no zeros in it) negates it
+    assert np.array_equal(oracle.binary_gradient_backward(4 * grad, B, alpha, p, (H, W))[1], 4 * gin)
+    assert np.array_equal(oracle.binary_gradient_backward(-grad, B, alpha, p, (H, W))[1], -gin)
+    # 1x1 filters, one output channel: gin = gmax alpha B[0][c] sign(g)
+    B1 = np.array([1, -1, 1], np.int8).reshape(1, 3, 1, 1)
+    g1 = g.standard_normal((1, 1, 4, 4)).astype(np.float32)
+    m1, gin1 = oracle.binary_gradient_backward(g1, B1, np.array([0.75], np.float32), 0, (4, 4))
+    want = (m1[0] * 0.75) * np.where(g1 >= 0, 1.0, -1.0)[:, 0][:, None] * B1.reshape(1, 3, 1, 1)
+    assert np.allclose(gin1, want, rtol=1e-6)
+    # brute force on a tiny case, taps that leave the gradient's extent contribute nothing
+    Bs = np.where(g.random((2, 1, 2, 2)) < 0.5, -1, 1).astype(np.int8)
+    gs = g.standard_normal((1, 2, 3, 3)).astype(np.float32)                 # H = W = 4, k = 2, pad 0
+    a2 = np.array([1.0, 3.0], np.float32)
+    ms, gins = oracle.binary_gradient_backward(gs, Bs, a2, 0, (4, 4))
+    for y, x in itertools.product(range(4), range(4)):
+        tot = 0.0
+        for co, ky, kx in itertools.product(range(2), range(2), range(2)):
+            oy, ox = y - ky, x - kx
+            if 0 <= oy < 3 and 0 <= ox < 3:
+                tot += float(a2[co]) * int(Bs[co, 0, ky, kx]) * (1.0 if gs[0, co, oy, ox] >= 0 else -1.0)
+        assert np.isclose(gins[0, 0, y, x], float(ms[0]) * tot, rtol=1e-6, atol=1e-6)
+
+
+def test_binary_gradient_backward_product_rounding(oracle):
+    """round_products rounds gmax * alpha to bfloat16: no effect when the products are
+    representable, otherwise the result is that of the rounded products."""
+    g = rng(320)
+    B = np.where(g.random((3, 4, 3, 3)) < 0.5, -1, 1).astype(np.int8)
+    grad = g.standard_normal((2, 3, 5, 5)).astype(np.float32)
+    grad[:, 0, 0, 0] = [4.0, -8.0]                                           # gmax = 4, 8
+    exact_alpha = np.array([0.5, 1.25, 3.0], np.float32)
+    a = oracle.binary_gradient_backward(grad, B, exact_alpha, 1, (5, 5), round_products=False)[1]
+    b = oracle.binary_gradient_backward(grad, B, exact_alpha, 1, (5, 5), round_products=True)[1]
+    assert np.array_equal(a, b)
+    alpha = np.array([0.3337, 1.2345, 0.071], np.float32)
+    r = oracle.binary_gradient_backward(grad, B, alpha, 1, (5, 5), round_products=True)[1]
+    for n, m in enumerate((4.0, 8.0)):
+        t = oracle.round_bf16((np.float32(m) * alpha).astype(np.float32))
+        # the rounded products as the filter scales of an unrounded run with gmax = 1
+        unit = np.where(grad[n:n + 1] >= 0, 1.0, -1.0).astype(np.float32)
+        want = oracle.binary_gradient_backward(unit, B, t, 1, (5, 5), round_products=False)[1]
+        assert np.allclose(r[n:n + 1], want, rtol=1e-6, atol=1e-6)
+    assert not np.array_equal(r, oracle.binary_gradient_backward(grad, B, alpha, 1, (5, 5))[1])
