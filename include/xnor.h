@@ -283,6 +283,40 @@ xnor_status xnor_bwn_conv2d_forward(const uint16_t *x_stream, const uint32_t *w_
                                     const xnor_conv_desc *d, float *out, void *cuda_stream);
 
 /*
+ * Backward convolution with a binarised gradient -- Section 3.2, "Binary Gradient":
+ * the convolution between the weight filters and the gradient that bounds the
+ * backward pass of a layer, with the gradient binarised like the forward operands
+ * but scaled by max_i |g_i| (not by the mean of Eq. 6), and, as in Algorithm 1,
+ * the binarised filters alpha * sign(W).  For the forward layer described by d
+ * (stride 1, k_h = k_w), with g the gradient at the convolution's output,
+ *   gmax[n]            = max over image n of |g|
+ *   grad_in[n][c][y][x] = sum_{co,ky,kx} alpha[co] sign(W[co][c][ky][kx]) gmax[n]
+ *                                        sign(g[n][co][y + pad - ky][x + pad - kx])
+ * (taps outside g contribute 0; sign(0) = +1): the gradient with respect to the
+ * convolution's input.  alpha sits inside the sum over the filters, so this is a
+ * convolution of the real tensor gmax alpha[co] sign(g) with +-1 filters: it runs
+ * on the Binary-Weight kernel (above), each product gmax[n] * alpha[co] formed in
+ * fp32 and rounded once to bfloat16, sums in fp32.
+ *   xnor_binarize_weights_transposed   w fp32 [C_out][C_in][k_h][k_w] ->
+ *       wT_packed u32 [P'][C_in][2], P' = ceil(k_h*k_w*ceil(C_out/32) / 2): the sign
+ *       bits as the backward convolution contracts them (channels = the filters co,
+ *       taps turned by 180 degrees), word-pair-major like w_packed.  Once per layer.
+ *   xnor_binary_gradient_backward   g fp32 [N][C_out][H_out][W_out], wT_packed,
+ *       alpha fp32 [C_out] (from xnor_binarize_weights) -> gmax fp32 [N],
+ *       grad_in fp32 [N][C_in][H][W]; g_stream is scratch of
+ *       xnor_bgrad_stream_elems(d) 16-bit elements (0: bad descriptor or unsupported).
+ * INVALID_ARG as for the other calls.  UNSUPPORTED (nothing launched): stride != 1,
+ * k_h != k_w, N > 65535, or a geometry the Binary-Weight kernel refuses (its limits
+ * apply to the convolution of [C_out][H_out][W_out] with pad k - 1 - pad).
+ */
+size_t xnor_bgrad_stream_elems(const xnor_conv_desc *d);
+xnor_status xnor_binarize_weights_transposed(const float *w, int C_out, int C_in, int k_h, int k_w,
+                                             uint32_t *wT_packed, void *cuda_stream);
+xnor_status xnor_binary_gradient_backward(const float *g, const uint32_t *wT_packed,
+                                          const float *alpha, const xnor_conv_desc *d, float *gmax,
+                                          uint16_t *g_stream, float *grad_in, void *cuda_stream);
+
+/*
  * Full-precision 1x1 strided convolution without bias: the projection
  * shortcut ("type B") of the ResNet-18 variant the paper binarises
  * (Section 4.2).  Its result is the `residual` of a block's second BinConv.

@@ -39,7 +39,8 @@ EXPORTS = [
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
     "xnor_maxpool2d", "xnor_binactiv_launches", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
     "xnor_binactiv_kbit", "xnor_conv2d_forward_kbit",
-    "xnor_bwn_input_elems", "xnor_bwn_prepare_input", "xnor_bwn_conv2d_forward", "xnor_measure_peaks",
+    "xnor_bwn_input_elems", "xnor_bwn_prepare_input", "xnor_bwn_conv2d_forward",
+    "xnor_bgrad_stream_elems", "xnor_binarize_weights_transposed", "xnor_binary_gradient_backward", "xnor_measure_peaks",
 ]
 
 
@@ -115,6 +116,12 @@ def load():
     lib.xnor_bwn_prepare_input.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp]
     lib.xnor_bwn_conv2d_forward.restype = ci
     lib.xnor_bwn_conv2d_forward.argtypes = [vp, vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp]
+    lib.xnor_bgrad_stream_elems.restype = ctypes.c_size_t
+    lib.xnor_bgrad_stream_elems.argtypes = [ctypes.POINTER(xnor_conv_desc)]
+    lib.xnor_binarize_weights_transposed.restype = ci
+    lib.xnor_binarize_weights_transposed.argtypes = [vp, ci, ci, ci, ci, vp, vp]
+    lib.xnor_binary_gradient_backward.restype = ci
+    lib.xnor_binary_gradient_backward.argtypes = [vp, vp, vp, ctypes.POINTER(xnor_conv_desc), vp, vp, vp, vp]
     lib.xnor_measure_peaks.restype = ci
     lib.xnor_measure_peaks.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
     _lib = lib
@@ -280,6 +287,39 @@ def xnor_bwn_conv2d_forward(x_stream, w_packed, alpha, residual, d, out, stream=
                                           _ptr(alpha, torch.float32), _ptr(residual, torch.float32),
                                           ctypes.byref(d), _ptr(out, torch.float32), _stream(stream)),
            "xnor_bwn_conv2d_forward")
+
+
+def xnor_bgrad_stream_elems(d):
+    return int(load().xnor_bgrad_stream_elems(ctypes.byref(d)))
+
+
+def xnor_binarize_weights_transposed(w, wT_packed, stream=None):
+    """w fp32 [C_out][C_in][k_h][k_w] -> sign bits for the backward convolution (alloc_weights_transposed)."""
+    Co, C, kh, kw = w.shape
+    _check(load().xnor_binarize_weights_transposed(_ptr(w, torch.float32), Co, C, kh, kw,
+                                                   _ptr(wT_packed, torch.int32), _stream(stream)),
+           "xnor_binarize_weights_transposed")
+
+
+def xnor_binary_gradient_backward(g, wT_packed, alpha, d, gmax, g_stream, grad_in, stream=None):
+    _check(load().xnor_binary_gradient_backward(_ptr(g, torch.float32), _ptr(wT_packed, torch.int32),
+                                                _ptr(alpha, torch.float32), ctypes.byref(d),
+                                                _ptr(gmax, torch.float32), _ptr(g_stream, torch.bfloat16),
+                                                _ptr(grad_in, torch.float32), _stream(stream)),
+           "xnor_binary_gradient_backward")
+
+
+def alloc_weights_transposed(C_out, C_in, k_h, k_w, device="cuda"):
+    """Packed sign words [P'][C_in][2] of the backward convolution."""
+    pairs = (k_h * k_w * ((C_out + 31) // 32) + 1) // 2
+    return torch.empty((pairs, C_in, 2), dtype=torch.int32, device=device)
+
+
+def alloc_bgrad(d, device="cuda"):
+    """(gmax [N], g_stream scratch, grad_in [N][C_in][H][W]) for xnor_binary_gradient_backward."""
+    return (torch.empty((d.N,), dtype=torch.float32, device=device),
+            torch.empty((xnor_bgrad_stream_elems(d),), dtype=torch.bfloat16, device=device),
+            torch.empty((d.N, d.C_in, d.H, d.W), dtype=torch.float32, device=device))
 
 
 def alloc_bwn_input(d, device="cuda"):

@@ -1,7 +1,7 @@
 // C-ABI entry points of libxnor: argument checks and dispatch.  No kernel code.
 #include <atomic>
 
-#include "common.cuh"
+#include "bgrad.cuh"
 
 namespace {
 
@@ -333,6 +333,53 @@ xnor_status xnor_bwn_conv2d_forward(const uint16_t *x_stream, const uint32_t *w_
   if (!xnor::bwn_supported(g)) return XNOR_ERR_UNSUPPORTED;
   return from_cuda(xnor::launch_bwn_conv(x_stream, w_packed, alpha, residual, g, out,
                                          (cudaStream_t)cuda_stream));
+}
+
+namespace {
+
+// Geometry of the backward convolution of the forward layer d: the gradient
+// [C_out][H_out][W_out] convolved at stride 1 with pad k - 1 - pad gives [C_in][H][W].
+bool backward_geom(const xnor_conv_desc *d, xnor::ConvGeom *gb) {
+  if (!good_desc(d) || d->stride != 1 || d->k_h != d->k_w || d->N > 65535) return false;
+  const xnor::ConvGeom g = xnor::make_geom(*d);
+  xnor_conv_desc b = *d;
+  b.C_in = d->C_out; b.C_out = d->C_in; b.H = g.Ho; b.W = g.Wo;
+  b.pad = d->k_h - 1 - d->pad; b.flags = 0;
+  *gb = xnor::make_geom(b);
+  return gb->Ho == d->H && gb->Wo == d->W && xnor::bwn_supported(*gb);
+}
+
+}  // namespace
+
+size_t xnor_bgrad_stream_elems(const xnor_conv_desc *d) {
+  xnor::ConvGeom gb;
+  return backward_geom(d, &gb) ? xnor::bwn_stream_elems(gb) : 0;
+}
+
+xnor_status xnor_binarize_weights_transposed(const float *w, int C_out, int C_in, int k_h, int k_w,
+                                             uint32_t *wT_packed, void *cuda_stream) {
+  if (bad_ptr(w) || bad_ptr(wT_packed)) return XNOR_ERR_INVALID_ARG;
+  if (C_out <= 0 || C_in <= 0 || k_h <= 0 || k_w <= 0) return XNOR_ERR_INVALID_ARG;
+  if ((long long)k_h * k_w * ((C_out + 31) / 32) > 12288) return XNOR_ERR_UNSUPPORTED;
+  return from_cuda(xnor::launch_binarize_weights_transposed(w, C_out, C_in, k_h, k_w, wT_packed,
+                                                            (cudaStream_t)cuda_stream));
+}
+
+xnor_status xnor_binary_gradient_backward(const float *g, const uint32_t *wT_packed,
+                                          const float *alpha, const xnor_conv_desc *d, float *gmax,
+                                          uint16_t *g_stream, float *grad_in, void *cuda_stream) {
+  if (!good_desc(d)) return XNOR_ERR_INVALID_ARG;
+  if (bad_ptr(g) || bad_ptr(wT_packed) || bad_ptr(alpha) || bad_ptr(gmax) || bad_ptr(g_stream) ||
+      bad_ptr(grad_in))
+    return XNOR_ERR_INVALID_ARG;
+  xnor::ConvGeom gb;
+  if (!backward_geom(d, &gb)) return XNOR_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  cudaError_t e = xnor::launch_grad_max(g, gb.N, (size_t)gb.C * gb.H * gb.W, gmax, st);
+  if (e == cudaSuccess) e = xnor::launch_bwn_prepare_grad(g, alpha, gmax, gb, g_stream, st);
+  if (e == cudaSuccess) e = xnor::launch_bwn_conv(g_stream, wT_packed, nullptr, nullptr, gb, grad_in, st);
+  if (e != cudaSuccess) (void)cudaGetLastError();
+  return from_cuda(e);
 }
 
 xnor_status xnor_shortcut_conv1x1(const float *x, const float *w, int N, int C_in, int H, int W,

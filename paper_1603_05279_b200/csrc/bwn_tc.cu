@@ -26,7 +26,7 @@
 
 #include <algorithm>
 
-#include "common.cuh"
+#include "bgrad.cuh"
 #include "umma_common.cuh"
 
 namespace xnor {
@@ -468,7 +468,8 @@ bwn_conv_kernel(const __grid_constant__ BwnParams P) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = tid; i < P.vec_len; i += kThreads)
-    reinterpret_cast<float *>(smem + P.off_vec)[i] = i < P.Co ? __ldg(P.alpha + i) : 0.0f;
+    reinterpret_cast<float *>(smem + P.off_vec)[i] =
+        i < P.Co ? (P.alpha != nullptr ? __ldg(P.alpha + i) : 1.0f) : 0.0f;   // no alpha: unit scale
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(S.tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
@@ -512,8 +513,9 @@ __device__ __forceinline__ uint32_t bf16_rne(float v) {
 
 __global__ void __launch_bounds__(256)
 bwn_prepare_kernel(const float *__restrict__ x, const float *__restrict__ scale,
-                   const float *__restrict__ shift, int N, int C, int H, int W, int s, int Hq, int Wq,
-                   int leadY, int leadX, long long L, int Cp, uint16_t *__restrict__ xs) {
+                   const float *__restrict__ shift, const float *__restrict__ gmax, int N, int C, int H,
+                   int W, int s, int Hq, int Wq, int leadY, int leadX, long long L, int Cp,
+                   uint16_t *__restrict__ xs) {
   __shared__ float tile[64][33];
   const int lane = threadIdx.x & 31, wy = threadIdx.x >> 5;      // 8 warps
   const long long nblk = (L + 31) / 32;
@@ -524,10 +526,12 @@ bwn_prepare_kernel(const float *__restrict__ x, const float *__restrict__ scale,
   const long long m = m0 + lane;
   bool real = m < L;
   size_t src = 0;
+  float gm = 0.0f;             // gradient mode: the scale of this position's image
   if (real) {
     const long long r = m / Wq;
     const int c = (int)(m - r * Wq);
     const long long n = r / Hq;
+    if (gmax != nullptr) gm = __ldg(gmax + n);
     const int ry = (int)(r - n * Hq);
     const int iy = (ry - leadY) * s + py, ix = (c - leadX) * s + px;
     real = ry >= leadY && c >= leadX && iy < H && ix < W;
@@ -546,7 +550,13 @@ bwn_prepare_kernel(const float *__restrict__ x, const float *__restrict__ scale,
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
       const int ch = c0 + wy + 8 * q;
-      if (scale != nullptr && real && ch < C) v[q] = __fmaf_rn(__ldg(scale + ch), v[q], __ldg(shift + ch));
+      if (gmax != nullptr) {
+        // binarised gradient (Section 3.2, "Binary Gradient"): sign(g) scaled by the image's
+        // max|g| and, here, by the filter's alpha (`scale`), the product formed in fp32
+        if (real && ch < C) v[q] = v[q] >= 0.0f ? __fmul_rn(gm, __ldg(scale + ch)) : -__fmul_rn(gm, __ldg(scale + ch));
+      } else if (scale != nullptr && real && ch < C) {
+        v[q] = __fmaf_rn(__ldg(scale + ch), v[q], __ldg(shift + ch));
+      }
       tile[wy + 8 * q][lane] = v[q];
     }
     __syncthreads();
@@ -714,8 +724,18 @@ cudaError_t launch_bwn_prepare(const float *x, const float *scale, const float *
   const StreamGeom q = stream_geom(g);
   const long long nblk = (q.L + 31) / 32 * q.phases;
   if (nblk >= (1ll << 31)) return cudaErrorInvalidValue;
-  bwn_prepare_kernel<<<(unsigned)nblk, 256, 0, st>>>(x, scale, shift, g.N, g.C, g.H, g.W, q.s, q.Hq,
-                                                    q.Wq, q.leadY, q.leadX, q.L, q.Cp, x_stream);
+  bwn_prepare_kernel<<<(unsigned)nblk, 256, 0, st>>>(x, scale, shift, nullptr, g.N, g.C, g.H, g.W, q.s,
+                                                    q.Hq, q.Wq, q.leadY, q.leadX, q.L, q.Cp, x_stream);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_bwn_prepare_grad(const float *g, const float *alpha, const float *gmax,
+                                    const ConvGeom &gb, uint16_t *g_stream, cudaStream_t st) {
+  const StreamGeom q = stream_geom(gb);
+  const long long nblk = (q.L + 31) / 32 * q.phases;
+  if (nblk >= (1ll << 31)) return cudaErrorInvalidValue;
+  bwn_prepare_kernel<<<(unsigned)nblk, 256, 0, st>>>(g, alpha, nullptr, gmax, gb.N, gb.C, gb.H, gb.W, q.s,
+                                                    q.Hq, q.Wq, q.leadY, q.leadX, q.L, q.Cp, g_stream);
   return cudaGetLastError();
 }
 
