@@ -252,7 +252,8 @@ class LayersJob:
         self.host_x, self.host_w, self.host_out = [], [], []
         for li, L in zip(layer_ids, self.layers):
             seed = du.rank_seed(wl.layer_seed(name, li), rank)
-            self.host_x.append(torch.from_numpy(wl.make_input(L.shape, seed)).pin_memory())
+            self.host_x.append(torch.from_numpy(wl.make_input(L.shape, seed) if variant != "bgrad" else
+                                                wl.normal(tuple(L.x.shape), seed)).pin_memory())
             self.host_w.append(torch.from_numpy(wl.make_weights(L.shape, seed)).pin_memory())
             self.host_out.append(torch.empty(L.out.shape, dtype=torch.float32).pin_memory())
             L.x.copy_(self.host_x[-1])
@@ -565,7 +566,7 @@ def run_ours(args):
     n_conv = len(job.conv_macs)
     sms = props.multi_processor_count
     clk_mhz = clocks["sm_mhz"] or 1965.0
-    if args.variant == "bwn":
+    if args.variant in ("bwn", "bgrad"):
         # bf16 x (+-1 as bf16) on kind::f16: the measured bf16 GEMM peak; the burst figure when the
         # sampled clock is the maximum one, else the sustained figure
         burst = clocks["sm_max_mhz"] is not None and clk_mhz >= 0.97 * (clocks["sm_max_mhz"] or clk_mhz)
@@ -659,6 +660,8 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": ("bf16 activations x 1-bit weights (as +-1 bf16), fp32 accumulation" if args.variant == "bwn"
+                  else "1-bit gradient scaled to bf16 x 1-bit weights (as +-1 bf16), fp32 accumulation"
+                  if args.variant == "bgrad"
                   else "u32 bit words (XOR+popcount), int32 sums, fp32 scaling" if engine == "popc"
                   else "e2m1 (fp4) tensor-core operands from 1-bit words, exact integer sums in "
                        "fp32, fp32 scaling"),
@@ -673,7 +676,9 @@ def run_ours(args):
                    "l2": "step working set %d MB of inputs+outputs (L2 is 126 MB); no flush"
                          % ((job.h2d + job.d2h + (job.act_bytes if args.workload == "chain" else 0))
                             // 1000000),
-                   "step": "weight binarisation + BN/BinActiv + BinConv for each layer",
+                   "step": ("weight binarisation (both packings) + max|g|, gradient stream, backward "
+                            "convolution for each layer" if args.variant == "bgrad" else
+                            "weight binarisation + BN/BinActiv + BinConv for each layer"),
                    "launch": (("one CUDA graph per step, independent work on parallel branches"
                                if branches else "one CUDA graph per step") if graph is not None
                               else "one library call per kernel group")},
@@ -709,9 +714,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true",
                     help="time call-by-call launches instead of a CUDA graph of the step")
     ap.add_argument("--engine", default="auto", choices=["auto", "popc", "umma", "umma_stream"])
-    ap.add_argument("--variant", default="xnor", choices=["xnor", "bwn", "kbit"],
+    ap.add_argument("--variant", default="xnor", choices=["xnor", "bwn", "kbit", "bgrad"],
                     help="layer workloads only: the XNOR block (default, the bench line), the "
-                         "Binary-Weight-Network convolution on real inputs, or k-bit activations")
+                         "Binary-Weight-Network convolution on real inputs, k-bit activations, or the "
+                         "backward convolution with a binarised gradient (stride-1 layers)")
     ap.add_argument("--kbits", type=int, default=2, help="bits of the k-bit variant")
     ap.add_argument("--workload", default="alexnet", choices=sorted(WORKLOAD_NAMES),
                     help="shape set (the bench line proper is the default, alexnet)")

@@ -13,8 +13,10 @@ class LayerBuffers:
     """All device tensors of one layer; inputs are filled by the caller."""
 
     def __init__(self, shape, device="cuda", with_acc=False, with_bn=True, variant="xnor", kbits=2):
-        """variant: "xnor" (the block of Eq. 11), "bwn" (real inputs, binary weights, Eq. 1) or
-        "kbit" (q_k activations with `kbits` bits in place of sign)."""
+        """variant: "xnor" (the block of Eq. 11), "bwn" (real inputs, binary weights, Eq. 1),
+        "kbit" (q_k activations with `kbits` bits in place of sign) or "bgrad" (the layer's backward
+        convolution with a binarised gradient: x is then the gradient at the layer's output,
+        [N][C_out][H_out][W_out], and out the gradient at its input, [N][C_in][H][W])."""
         s = shape
         self.variant, self.kbits = variant, kbits
         self.shape = s
@@ -33,11 +35,19 @@ class LayerBuffers:
         elif variant == "kbit":
             self.x_planes = torch.empty((kbits,) + tuple(self.x_packed.shape), dtype=torch.int32,
                                         device=device)
+        elif variant == "bgrad":
+            self.x = torch.empty(tuple(self.out.shape), dtype=torch.float32, device=device)
+            self.wT_packed = B.alloc_weights_transposed(s.C_out, s.C_in, s.k, s.k, device)
+            self.gmax, self.g_stream, self.out = B.alloc_bgrad(self.desc, device)
 
     def binarize_weights(self, stream=None):
         B.xnor_binarize_weights(self.w, self.w_packed, self.alpha, stream)
+        if self.variant == "bgrad":
+            B.xnor_binarize_weights_transposed(self.w, self.wT_packed, stream)
 
     def binactiv(self, stream=None):
+        if self.variant == "bgrad":
+            return                   # the gradient is scaled and laid out inside the backward call
         if self.variant == "bwn":
             B.xnor_bwn_prepare_input(self.x, self.bn_scale, self.bn_shift, self.desc, self.x_stream, stream)
         elif self.variant == "kbit":
@@ -48,7 +58,10 @@ class LayerBuffers:
                             self.K, stream)
 
     def conv(self, stream=None):
-        if self.variant == "bwn":
+        if self.variant == "bgrad":
+            B.xnor_binary_gradient_backward(self.x, self.wT_packed, self.alpha, self.desc, self.gmax,
+                                            self.g_stream, self.out, stream)
+        elif self.variant == "bwn":
             B.xnor_bwn_conv2d_forward(self.x_stream, self.w_packed, self.alpha, self.residual,
                                       self.desc, self.out, stream)
         elif self.variant == "kbit":
@@ -66,6 +79,8 @@ class LayerBuffers:
 
     # algorithmic bytes, as the roofline of each kernel counts them
     def binactiv_launches(self):
+        if self.variant == "bgrad":
+            return 0
         if self.variant == "bwn":
             return 1
         if self.variant == "kbit":
@@ -75,10 +90,14 @@ class LayerBuffers:
     def launches(self):
         """Kernels one forward() launches: binarize 1, BinActiv 1 or 2 (pack + A, box filter; one
         kernel where a block streams whole images), BinConv 1 (k-bit: one per plane)."""
+        if self.variant == "bgrad":
+            return 2 + 3             # two weight packings; maximum, gradient stream, convolution
         conv = self.kbits if self.variant == "kbit" else 1
         return 1 + self.binactiv_launches() + conv
 
     def binactiv_bytes(self):
+        if self.variant == "bgrad":
+            return 0
         s = self.shape
         ho, wo = wl.out_hw(s)
         cw = (s.C_in + 31) // 32
