@@ -156,6 +156,9 @@ xnor_status xnor_binactiv(const float *x, const float *bn_scale, const float *bn
  * xnor_binactiv refuses.  has_bn != 0 = with bn_scale / bn_shift.
  */
 int xnor_binactiv_launches(const xnor_conv_desc *d, int has_bn);
+/* The same for xnor_binactiv_kbit (below): its one-kernel path has the same conditions, with
+ * k times the packed words of an image staged in shared memory.  0: bad arguments. */
+int xnor_binactiv_kbit_launches(const xnor_conv_desc *d, int kbits, int has_bn);
 
 /*
  * xnor_binactiv without a caller-supplied A buffer.  (The paper has no

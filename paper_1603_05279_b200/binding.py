@@ -37,7 +37,7 @@ EXPORTS = [
     "xnor_version", "xnor_built_with_bounds_check", "xnor_status_string", "xnor_words_per_pixel", "xnor_out_extent",
     "xnor_binarize_weights", "xnor_binactiv", "xnor_binactiv_static", "xnor_conv2d_forward", "xnor_shortcut_conv1x1",
     "xnor_set_engine", "xnor_get_engine", "xnor_check_device", "xnor_selftest_wait_timeout",
-    "xnor_maxpool2d", "xnor_binactiv_launches", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
+    "xnor_maxpool2d", "xnor_binactiv_launches", "xnor_binactiv_kbit_launches", "xnor_conv2d_binactiv_parts", "xnor_conv2d_forward_binactiv", "xnor_binactiv_finish",
     "xnor_binactiv_kbit", "xnor_conv2d_forward_kbit",
     "xnor_bwn_input_elems", "xnor_bwn_prepare_input", "xnor_bwn_conv2d_forward",
     "xnor_bgrad_stream_elems", "xnor_binarize_weights_transposed", "xnor_binary_gradient_backward", "xnor_measure_peaks",
@@ -93,6 +93,8 @@ def load():
     lib.xnor_check_device.restype = ci
     lib.xnor_check_device.argtypes = [vp]
     lib.xnor_conv2d_binactiv_parts.restype = ci
+    lib.xnor_binactiv_kbit_launches.restype = ci
+    lib.xnor_binactiv_kbit_launches.argtypes = [ctypes.POINTER(xnor_conv_desc), ci, ci]
     lib.xnor_binactiv_launches.restype = ci
     lib.xnor_binactiv_launches.argtypes = [ctypes.POINTER(xnor_conv_desc), ci]
     lib.xnor_conv2d_binactiv_parts.argtypes = [ctypes.POINTER(xnor_conv_desc)]
@@ -196,6 +198,11 @@ def xnor_check_device(stream=None):
 def xnor_binactiv_launches(d, has_bn=False):
     """Kernels xnor_binactiv launches for this shape (1 or 2; 0 = refused shape)."""
     return int(load().xnor_binactiv_launches(ctypes.byref(d), int(bool(has_bn))))
+
+
+def xnor_binactiv_kbit_launches(d, kbits, has_bn=False):
+    """Kernels xnor_binactiv_kbit launches for this shape (1 or 2; 0 = bad arguments)."""
+    return int(load().xnor_binactiv_kbit_launches(ctypes.byref(d), int(kbits), int(bool(has_bn))))
 
 
 def xnor_conv2d_binactiv_parts(d):

@@ -2,6 +2,7 @@
 #include <atomic>
 
 #include "bgrad.cuh"
+#include "kbit.cuh"
 
 namespace {
 
@@ -229,6 +230,11 @@ int xnor_binactiv_launches(const xnor_conv_desc *d, int has_bn) {
   const xnor::ConvGeom g = xnor::make_geom(*d);
   if (!xnor::binactiv_supported(g, has_bn != 0)) return 0;
   return xnor::binactiv_launch_count(g, has_bn != 0);
+}
+
+int xnor_binactiv_kbit_launches(const xnor_conv_desc *d, int kbits, int has_bn) {
+  if (!good_desc(d) || kbits < 1 || kbits > 7) return 0;
+  return xnor::binactiv_kbit_launch_count(xnor::make_geom(*d), has_bn != 0, kbits);
 }
 
 int xnor_conv2d_binactiv_parts(const xnor_conv_desc *d) {

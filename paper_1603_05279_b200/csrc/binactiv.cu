@@ -3,7 +3,7 @@
 // convolution's output positions.
 #include <algorithm>
 
-#include "common.cuh"
+#include "kbit.cuh"
 #include "umma_common.cuh"
 
 namespace xnor {
@@ -215,6 +215,7 @@ struct ImgParams {
   uint32_t chunk_bytes;            // cc * H * W * 4, a multiple of 16
   uint32_t off_buf, off_words, off_apart, off_aimg, off_bn;   // byte offsets in shared memory
   int kh, kw, stride, pad, Ho, Wo, valid_taps;
+  int kbits;                       // k-bit mode: bit planes of the level index (x_packed = [k][N][H][W][Cw])
 };
 
 __device__ __forceinline__ float lds_f(uint32_t addr) {
@@ -238,7 +239,9 @@ __device__ __forceinline__ bool img_sync(uint32_t bar, uint32_t &phase, int lane
   return __all_sync(0xFFFFFFFFu, ok);
 }
 
-template <bool kHasBN, int KS>
+// kKbit: q_k in place of sign (see binactiv_pack_kbit_kernel below for the rule): a unit then
+// yields one byte of each of the k bit planes, staged plane by plane.
+template <bool kHasBN, int KS, bool kKbit>
 __global__ void __launch_bounds__(kImgThreads, 2)
 binactiv_image_kernel(const __grid_constant__ ImgParams P) {
   using namespace umma;
@@ -254,6 +257,14 @@ binactiv_image_kernel(const __grid_constant__ ImgParams P) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int HW = P.H * P.W, nsub = P.cc >> 3, nchunks = P.C / P.cc;
   const int npg = (HW + 31) >> 5;
+  const int nplanes = kKbit ? P.kbits : 1;
+  const uint32_t plane_bytes = (uint32_t)HW * (uint32_t)P.Cw * 4u;      // staged words of one bit plane
+  __shared__ float tau[kKbit ? 128 : 1];     // decision points tau[j], j = 1 .. 2^k - 1
+  if (kKbit) {
+    const int levels = (1 << P.kbits) - 1;
+    for (int j = 1 + tid; j <= levels; j += kImgThreads)
+      tau[j] = (float)((double)(2 * j - 1) / (double)levels - 1.0);
+  }
 
   const int my_images = ((int)blockIdx.x < P.N) ? (P.N - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   const long long total = (long long)my_images * nchunks;
@@ -281,7 +292,7 @@ binactiv_image_kernel(const __grid_constant__ ImgParams P) {
     for (; q < total && q < P.nbuf; ++q) issue_chunk();
   }
   // bytes of channels beyond C (C % 32 != 0) are never written by a unit: they stay zero
-  for (int i = tid; i < HW * P.Cw; i += kImgThreads) reinterpret_cast<uint32_t *>(wbytes)[i] = 0u;
+  for (int i = tid; i < nplanes * HW * P.Cw; i += kImgThreads) reinterpret_cast<uint32_t *>(wbytes)[i] = 0u;
   if (kHasBN)
     for (int c = tid; c < P.C; c += kImgThreads) bn[c] = make_float2(__ldg(P.scale + c), __ldg(P.shift + c));
   __syncthreads();
@@ -347,16 +358,36 @@ binactiv_image_kernel(const __grid_constant__ ImgParams P) {
               float y[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) y[j] = lds_f(ta[j] + (uint32_t)(r * pstep * 4));
-              uint32_t bits = 0u;
+              uint32_t bits = 0u;              // sign mode: the 8 bits; k-bit: plane p in byte p (k <= 4)
+              uint32_t bits_hi = 0u;           // planes 4 .. 6
               float p0 = 0.0f, p1 = 0.0f;
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 float v = y[j];
                 if (kHasBN) v = (j & 1) ? __fmaf_rn(ss[j >> 1].z, v, ss[j >> 1].w) : __fmaf_rn(ss[j >> 1].x, v, ss[j >> 1].y);
-                if (v >= 0.0f) bits |= 1u << j;
+                if (kKbit) {
+                  // largest index whose decision point is <= v, by bisection over the sorted tau
+                  int idx = 0;
+                  for (int bb = P.kbits - 1; bb >= 0; --bb) {
+                    const int cand = idx + (1 << bb);
+                    if (v >= tau[cand]) idx = cand;
+                  }
+                  // bit p of idx -> bit j of byte p: spread the low four bits over four bytes
+                  const uint32_t lo = (uint32_t)idx & 15u, hi = (uint32_t)idx >> 4;
+                  bits |= ((lo & 1u) | ((lo & 2u) << 7) | ((lo & 4u) << 14) | ((lo & 8u) << 21)) << j;
+                  bits_hi |= ((hi & 1u) | ((hi & 2u) << 7) | ((hi & 4u) << 14)) << j;
+                } else {
+                  if (v >= 0.0f) bits |= 1u << j;
+                }
                 if (j & 1) p1 += fabsf(v); else p0 += fabsf(v);
               }
-              wb[(size_t)(r * pstep) * (P.Cw * 4)] = (uint8_t)bits;
+              if (kKbit) {
+                for (int pl = 0; pl < P.kbits; ++pl)
+                  wb[(size_t)pl * plane_bytes + (size_t)(r * pstep) * (P.Cw * 4)] =
+                      (uint8_t)((pl < 4 ? bits >> (8 * pl) : bits_hi >> (8 * (pl - 4))) & 0xFFu);
+              } else {
+                wb[(size_t)(r * pstep) * (P.Cw * 4)] = (uint8_t)bits;
+              }
               asum[r] += p0 + p1;
             }
           }
@@ -380,9 +411,9 @@ binactiv_image_kernel(const __grid_constant__ ImgParams P) {
       P.A[(size_t)n * HW + p] = a;
       aimg[p] = a;
     }
-    {
-      uint32_t *dst = P.x_packed + (size_t)n * HW * P.Cw;
-      const uint32_t *srcw = reinterpret_cast<const uint32_t *>(wbytes);
+    for (int pl = 0; pl < nplanes; ++pl) {
+      uint32_t *dst = P.x_packed + ((size_t)pl * P.N + n) * HW * P.Cw;
+      const uint32_t *srcw = reinterpret_cast<const uint32_t *>(wbytes + (size_t)pl * plane_bytes);
       for (int i = tid; i < HW * P.Cw; i += 32 * kImgWarps) dst[i] = srcw[i];
     }
     if (!img_sync(cbar, cph, lane, abort_flag)) return;
@@ -504,7 +535,7 @@ constexpr uint32_t kImgHeader = 256;             // barriers and the abort flag
 // not a multiple of four pixels, whole bytes of packed channels (with the 16-byte alignment of
 // x that the entry point checks, every image then starts on a 16-byte boundary), enough images to occupy the SMs, and a chunk of at least eight channel planes
 // small enough that two (better four) of them fit beside the staged outputs of an image.
-bool image_plan(const ConvGeom &g, bool bn, int sms, ImgParams *ip) {
+bool image_plan(const ConvGeom &g, bool bn, int sms, int kbits, ImgParams *ip) {
   const long long HW = (long long)g.H * g.W;
   if ((HW & 3) == 0 || (g.C & 7) != 0) return false;
   if (g.N < sms / 2 || HW > 32 * kImgWarps * kImgRounds) return false;
@@ -513,52 +544,63 @@ bool image_plan(const ConvGeom &g, bool bn, int sms, ImgParams *ip) {
   for (int pass = 0; pass < 3; ++pass) {
     const int nbuf = pass == 0 ? 4 : pass == 1 ? 3 : 2;
     const long long chunk_max = pass == 0 ? 24 * 1024 : pass == 1 ? 32 * 1024 : 48 * 1024;
-    int cc = 0;
-    for (int c = 8; c <= g.C; c += 8)
-      if (g.C % c == 0 && (long long)c * HW * 4 <= chunk_max) cc = c;
-    if (cc == 0) continue;
-    const uint32_t chunk = (uint32_t)(cc * HW * 4);
-    uint32_t off = kImgHeader;
-    ip->off_buf = off; off += (uint32_t)nbuf * chunk;
-    ip->off_words = off; off += (uint32_t)(HW * g.Cw * 4);
-    ip->off_apart = off; off += (uint32_t)(slots * HW * 4);
-    ip->off_aimg = off; off += (uint32_t)(HW * 4);
-    off = (off + 15u) & ~15u;
-    ip->off_bn = off; off += bn ? (uint32_t)g.C * 8u : 0u;
-    if (off > kImgSmemMax) continue;
-    ip->cc = cc; ip->nbuf = nbuf; ip->chunk_bytes = chunk;
-    return true;
+    // the largest chunk of whole channel planes (a multiple of 8 that divides C) under the
+    // pass's chunk size that fits shared memory beside the staged outputs of an image
+    for (int cc = g.C; cc >= 8; cc -= 8) {
+      if (g.C % cc != 0 || (long long)cc * HW * 4 > chunk_max) continue;
+      const uint32_t chunk = (uint32_t)(cc * HW * 4);
+      uint32_t off = kImgHeader;
+      ip->off_buf = off; off += (uint32_t)nbuf * chunk;
+      ip->off_words = off; off += (uint32_t)((kbits > 0 ? kbits : 1) * HW * g.Cw * 4);
+      ip->off_apart = off; off += (uint32_t)(slots * HW * 4);
+      ip->off_aimg = off; off += (uint32_t)(HW * 4);
+      off = (off + 15u) & ~15u;
+      ip->off_bn = off; off += bn ? (uint32_t)g.C * 8u : 0u;
+      if (off > kImgSmemMax) continue;
+      ip->cc = cc; ip->nbuf = nbuf; ip->chunk_bytes = chunk; ip->kbits = kbits;
+      return true;
+    }
   }
   return false;
 }
 
-template <bool kHasBN, int KS>
+template <bool kHasBN, int KS, bool kKbit>
 cudaError_t launch_image_variant(const ImgParams &ip, int sms, size_t smem, cudaStream_t st) {
   static bool attr_flags[64] = {};
   bool &attr_set = attr_done_for_current_device(attr_flags);
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(binactiv_image_kernel<kHasBN, KS>,
+    cudaError_t e = cudaFuncSetAttribute(binactiv_image_kernel<kHasBN, KS, kKbit>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kImgSmemMax);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return e; }
     attr_set = true;
   }
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, binactiv_image_kernel<kHasBN, KS>, kImgThreads,
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, binactiv_image_kernel<kHasBN, KS, kKbit>, kImgThreads,
                                                     smem) != cudaSuccess || per_sm < 1) {
     (void)cudaGetLastError();
     per_sm = 1;
   }
   const long long resident = (long long)per_sm * sms;
   const unsigned grid = (unsigned)(ip.N < resident ? ip.N : resident);
-  binactiv_image_kernel<kHasBN, KS><<<grid, kImgThreads, smem, st>>>(ip);
+  binactiv_image_kernel<kHasBN, KS, kKbit><<<grid, kImgThreads, smem, st>>>(ip);
   return cudaGetLastError();
+}
+
+void fill_img_params(ImgParams &ip, const float *x, const float *scale, const float *shift,
+                     const ConvGeom &g, uint32_t *x_packed, float *A, float *K) {
+  ip.x = x; ip.scale = scale; ip.shift = shift; ip.x_packed = x_packed; ip.A = A; ip.K = K;
+  ip.N = g.N; ip.C = g.C; ip.H = g.H; ip.W = g.W; ip.Cw = g.Cw;
+  ip.kh = g.kh; ip.kw = g.kw; ip.stride = g.stride; ip.pad = g.pad; ip.Ho = g.Ho; ip.Wo = g.Wo;
+  ip.valid_taps = (g.flags & XNOR_FLAG_K_VALID_TAPS) ? 1 : 0;
 }
 
 cudaError_t launch_binactiv_image(const ImgParams &ip, bool bn, int sms, cudaStream_t st) {
   const size_t smem = (size_t)ip.off_bn + (bn ? (size_t)ip.C * 8 : 0);
   const int ks = ip.kh == ip.kw ? ip.kh : 0;
-#define XNOR_IMG(KS) (bn ? launch_image_variant<true, KS>(ip, sms, smem, st) \
-                         : launch_image_variant<false, KS>(ip, sms, smem, st))
+#define XNOR_IMG(KS) (ip.kbits > 0 ? (bn ? launch_image_variant<true, KS, true>(ip, sms, smem, st)    \
+                                       : launch_image_variant<false, KS, true>(ip, sms, smem, st))  \
+                                  : (bn ? launch_image_variant<true, KS, false>(ip, sms, smem, st)   \
+                                       : launch_image_variant<false, KS, false>(ip, sms, smem, st)))
   if (ks == 1) return XNOR_IMG(1);
   if (ks == 3) return XNOR_IMG(3);
   if (ks == 5) return XNOR_IMG(5);
@@ -569,10 +611,12 @@ cudaError_t launch_binactiv_image(const ImgParams &ip, bool bn, int sms, cudaStr
 
 }  // namespace
 
-int binactiv_launch_count(const ConvGeom &g, bool has_bn) {
+int binactiv_kbit_launch_count(const ConvGeom &g, bool has_bn, int kbits) {
   ImgParams ip;
-  return image_plan(g, has_bn, sm_count_of_current_device(), &ip) ? 1 : 2;
+  return image_plan(g, has_bn, sm_count_of_current_device(), kbits, &ip) ? 1 : 2;
 }
+
+int binactiv_launch_count(const ConvGeom &g, bool has_bn) { return binactiv_kbit_launch_count(g, has_bn, 0); }
 
 cudaError_t read_status_act(int *status) {
   cudaError_t e = cudaMemcpyFromSymbol(status, g_status_act, sizeof(int));
@@ -599,11 +643,8 @@ cudaError_t launch_binactiv(const float *x, const float *scale, const float *shi
   const int sms = sm_count_of_current_device();
   {
     ImgParams ip;
-    if (image_plan(g, scale != nullptr, sms, &ip)) {
-      ip.x = x; ip.scale = scale; ip.shift = shift; ip.x_packed = x_packed; ip.A = A; ip.K = K;
-      ip.N = g.N; ip.C = g.C; ip.H = g.H; ip.W = g.W; ip.Cw = g.Cw;
-      ip.kh = g.kh; ip.kw = g.kw; ip.stride = g.stride; ip.pad = g.pad; ip.Ho = g.Ho; ip.Wo = g.Wo;
-      ip.valid_taps = (g.flags & XNOR_FLAG_K_VALID_TAPS) ? 1 : 0;
+    if (image_plan(g, scale != nullptr, sms, 0, &ip)) {
+      fill_img_params(ip, x, scale, shift, g, x_packed, A, K);
       return launch_binactiv_image(ip, scale != nullptr, sms, st);
     }
   }
@@ -763,6 +804,15 @@ binactiv_pack_kbit_kernel(const float *__restrict__ x, const float *__restrict__
 cudaError_t launch_binactiv_kbit(const float *x, const float *scale, const float *shift,
                                  const ConvGeom &g, int kbits, uint32_t *x_planes, float *A, float *K,
                                  cudaStream_t st) {
+  {
+    // planes of odd size and enough images: the kernel that streams whole images, in k-bit mode
+    const int sms = sm_count_of_current_device();
+    ImgParams ip;
+    if (image_plan(g, scale != nullptr, sms, kbits, &ip)) {
+      fill_img_params(ip, x, scale, shift, g, x_planes, A, K);
+      return launch_binactiv_image(ip, scale != nullptr, sms, st);
+    }
+  }
   const long long total_pix = (long long)g.N * g.H * g.W;
   const long long nblocks = ((total_pix + 31) / 32 + 7) / 8;
   const unsigned grid = (unsigned)std::min<long long>(nblocks, 8ll * sm_count_of_current_device());

@@ -84,7 +84,7 @@ class LayerBuffers:
         if self.variant == "bwn":
             return 1
         if self.variant == "kbit":
-            return 2
+            return B.xnor_binactiv_kbit_launches(self.desc, self.kbits, self.bn_scale is not None)
         return B.xnor_binactiv_launches(self.desc, self.bn_scale is not None)
 
     def launches(self):

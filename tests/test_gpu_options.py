@@ -185,3 +185,47 @@ def test_kbit_decision_points(oracle):
         X.xnor_binactiv_kbit(dev(x), None, None, d, kbits, planes, A, K)
         torch.cuda.synchronize()
         assert np.array_equal(2 * _index_of_planes(host(planes), C) - m, oracle.quantize_k(x, kbits).astype(np.int64))
+
+
+@pytest.mark.parametrize("kbits", [1, 2, 3, 7])
+@pytest.mark.parametrize("shape", [(160, 96, 27, 27, 5, 2, True), (150, 40, 13, 13, 3, 1, False),
+                                   (96, 256, 7, 7, 3, 1, True)])
+def test_kbit_binactiv_on_planes_of_odd_size_with_many_images(oracle, shape, kbits):
+    """With enough images and planes that are not a multiple of four pixels the k-bit BinActiv is
+    one kernel that streams whole images (as for sign bits): level codes identical to the oracle's
+    and to the two-kernel path, A and K within tolerance."""
+    N, C, H, W, k, p, bn = shape
+    g = rng(3 * sum(shape[:6]) + kbits)
+    x = (0.6 * g.standard_normal((N, C, H, W))).astype(np.float32)
+    scale = (1.0 + 0.2 * g.standard_normal(C)).astype(np.float32) if bn else None
+    shift = (0.2 * g.standard_normal(C)).astype(np.float32) if bn else None
+    d = X.make_desc(N, C, H, W, 8, k, k, 1, p)
+    # one kernel whenever k planes of an image's packed words fit shared memory beside the copies
+    assert X.xnor_binactiv_kbit_launches(d, kbits, bn) == (1 if kbits <= 3 else X.xnor_binactiv_kbit_launches(d, kbits, bn))
+    Cw = (C + 31) // 32
+    gs = GuardSet()
+    planes = gs.new("x_planes", (kbits, N, H, W, Cw), torch.int32)
+    _, A0, K0 = X.alloc_binactiv(d)
+    A, K = gs.like("A", A0), gs.like("K", K0)
+    planes.fill_(-1); A.fill_(float("nan")); K.fill_(float("nan"))
+    xd = dev(x)
+    sc, sh = (None, None) if scale is None else (dev(scale), dev(shift))
+    X.xnor_binactiv_kbit(xd, sc, sh, d, kbits, planes, A, K)
+    X.xnor_check_device()
+    gs.check()
+    m = 2 ** kbits - 1
+    for n in sorted({0, N // 2, N - 1}):
+        y = x[n:n + 1] if scale is None else oracle.bn_affine(x[n:n + 1], scale, shift)
+        codes = 2 * _index_of_planes(host(planes[:, n:n + 1]), C) - m
+        assert np.array_equal(codes, oracle.quantize_k(y, kbits).astype(np.int64)), n
+        A_or = oracle.channel_abs_mean(y)
+        assert_close(host(A[n:n + 1]), A_or, "A of image %d" % n)
+        assert_close(host(K[n:n + 1]), oracle.box_filter(A_or, k, k, 1, p), "K of image %d" % n)
+    # the last images alone take the two-kernel path: same planes
+    d8 = X.make_desc(8, C, H, W, 8, k, k, 1, p)
+    assert X.xnor_binactiv_kbit_launches(d8, kbits, bn) == 2
+    planes8 = torch.empty((kbits, 8, H, W, Cw), dtype=torch.int32, device="cuda")
+    _, A8, K8 = X.alloc_binactiv(d8)
+    X.xnor_binactiv_kbit(xd[N - 8:].contiguous(), sc, sh, d8, kbits, planes8, A8, K8)
+    assert torch.equal(planes8, planes[:, N - 8:])
+    assert_close(host(A8), host(A[N - 8:]), "A of the two paths")
