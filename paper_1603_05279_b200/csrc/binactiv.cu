@@ -327,6 +327,10 @@ binactiv_image_kernel(const __grid_constant__ ImgParams P) {
   const int pg0 = npg >= kImgWarps ? warp : warp % npg;
   const int slot = npg >= kImgWarps ? 0 : warp / npg;
   const bool has_work = slot < slots;
+  // k <= 2: tau_1 .. tau_3 (k = 1 has tau_1 = 0 alone: the other two never compare true)
+  const float kInf = __int_as_float(0x7f800000);
+  const float t1 = kKbit ? tau[1] : 0.0f;
+  const float t2 = kKbit && P.kbits == 2 ? tau[2] : kInf, t3 = kKbit && P.kbits == 2 ? tau[3] : kInf;
   const int pstep = 32 * kImgWarps;
   const uint32_t plane4 = (uint32_t)HW * 4u;
   const uint32_t bn_addr = base + P.off_bn;
@@ -368,14 +372,22 @@ binactiv_image_kernel(const __grid_constant__ ImgParams P) {
                 if (kKbit) {
                   // largest index whose decision point is <= v, by bisection over the sorted tau
                   int idx = 0;
-                  for (int bb = P.kbits - 1; bb >= 0; --bb) {
-                    const int cand = idx + (1 << bb);
-                    if (v >= tau[cand]) idx = cand;
+                  if (P.kbits <= 2) {           // up to three decision points, held in registers
+                    idx = (v >= t1 ? 1 : 0) + (v >= t2 ? 1 : 0) + (v >= t3 ? 1 : 0);
+                  } else {
+                    for (int bb = P.kbits - 1; bb >= 0; --bb) {
+                      const int cand = idx + (1 << bb);
+                      if (v >= tau[cand]) idx = cand;
+                    }
                   }
                   // bit p of idx -> bit j of byte p: spread the low four bits over four bytes
                   const uint32_t lo = (uint32_t)idx & 15u, hi = (uint32_t)idx >> 4;
-                  bits |= ((lo & 1u) | ((lo & 2u) << 7) | ((lo & 4u) << 14) | ((lo & 8u) << 21)) << j;
-                  bits_hi |= ((hi & 1u) | ((hi & 2u) << 7) | ((hi & 4u) << 14)) << j;
+                  if (P.kbits <= 2) {
+                    bits |= ((lo & 1u) | ((lo & 2u) << 7)) << j;
+                  } else {
+                    bits |= ((lo & 1u) | ((lo & 2u) << 7) | ((lo & 4u) << 14) | ((lo & 8u) << 21)) << j;
+                    if (P.kbits > 4) bits_hi |= ((hi & 1u) | ((hi & 2u) << 7) | ((hi & 4u) << 14)) << j;
+                  }
                 } else {
                   if (v >= 0.0f) bits |= 1u << j;
                 }
