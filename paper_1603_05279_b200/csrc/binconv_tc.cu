@@ -144,7 +144,7 @@ struct TcParams {
   int vec_len;                 // the next layer's scale and shift; vec_len floats each
   uint32_t raw_bytes;          // size of a raw buffer: the packed input rows a patch can touch
   int nraw;                    // raw buffers per subgroup of patch warps (1 or 2)
-  int pat_group;               // warps that build patches: 3, or 7 with four of the weight warps
+  int pat_group;               // warps that build patches
   int pat_sub;                 // subgroups they form (each builds whole patches): 3 or 1
   int wgt_warps;               // warps that expand weights: 8, or 4
   uint32_t idesc;
@@ -647,9 +647,8 @@ __device__ __forceinline__ bool weight_dispatch(const TcParams &P, const Smem &S
 }
 
 // ------------------------------------------------------------------ patch producers
-// A group of P.pat_group warps (the three patch warps, in the resident schedule also four of
-// the weight warps) builds the CTA's patches one after the other, all warps on the same
-// patch: units of (32 stream positions, phase plane, up to 4 channel words) are dealt round
+// A group of P.pat_group warps (the three patch warps) builds the CTA's patches one after the
+// other, all warps on the same patch: units of (32 stream positions, phase plane, up to 4 channel words) are dealt round
 // robin.  The packed pixels a patch touches are ONE contiguous range of x_packed: input rows
 // g0 .. g1 - 1 of the N*H rows (images follow one another in memory, the zero rows and
 // columns of the stream exist only in the patch).  Every patch buffer has a raw buffer; the
@@ -1183,8 +1182,6 @@ binconv_tc_kernel(const __grid_constant__ TcParams P) {
     const int wt = tid - 32 * kWgtWarp0;
     if (warp == kMmaWarp) { if (S.rank == 0) mma_role<kRes, kPair>(P, S, i0, i1, tmem_base); }
     else if (warp >= kPatWarp0) patch_role<kRes>(P, S, i0, i1, warp - kPatWarp0, lane);
-    else if (kRes && P.pat_group > kPatWarps && warp >= kWgtWarp0 + 4)
-      patch_role<kRes>(P, S, i0, i1, kPatWarps + warp - (kWgtWarp0 + 4), lane);   // helpers
     else if (!kRes) {
       if (warp < kEpiWarps)
         epilogue_role<false, kFuse>(P, S, i0, 0, 0, 0, (uint32_t)(i1 - i0), 0, tmem_base, warp, 0, lane);
@@ -1317,12 +1314,11 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
       P.NT = slab_width(g.Co, ns, pair || fuse);
       P.NTh = pair ? P.NT / 2 : P.NT;
       if (P.NT < 128 && ns > 1) break;
-      // The slab is expanded once per visit, so four weight warps are enough when a thread
-      // per row fits them; with many channel words per pixel (measured: from 12 on) the other
-      // four then build patches instead of draining accumulators.
-      const bool helpers = g.Cw >= 12 && P.NTh <= 128;
-      P.wgt_warps = helpers ? kWgtWarps / 2 : kWgtWarps;
-      P.pat_group = helpers ? kPatWarps + kWgtWarps / 2 : kPatWarps;
+      // (Lending four of the weight warps to the patch builders where a pixel has many channel
+      // words was the better split while the drain loop was longer; since its trimming twelve
+      // draining warps win on every layer measured: conv4 50.4 -> 48.1 us, conv5 39.4 -> 37.3.)
+      P.wgt_warps = kWgtWarps;
+      P.pat_group = kPatWarps;
       plan_stage(P);
       const int nst = (P.nsteps + P.mps - 1) / P.mps;
       if (nst <= kMaxBarStages && fits(nst, 2, 1)) {
@@ -1351,8 +1347,8 @@ Plan make_plan(const ConvGeom &g, int schedule, bool pair, bool fuse = false) {
   P.nraw = fits(stages, npb, 2) ? 2 : 1;
   P.nacc = std::max(1, std::min(kMaxAcc, kMaxAccCols / P.NT));
   // worker warps per quarter of the lanes in the resident schedule: the four epilogue warps
-  // and the weight warps (all eight, or the four that are not patch helpers)
-  P.epi_split = std::min(P.pat_group > kPatWarps ? 2 : kEpiSplitMax, P.NT / (fuse ? 32 : 16));
+  // and the eight weight warps
+  P.epi_split = std::min(kEpiSplitMax, P.NT / (fuse ? 32 : 16));
   if (fuse && (g.Co & 31) != 0) return pl;          // whole words of the next layer's input
   P.stages = stages; P.npb = npb;
   // small patches: every patch warp builds whole patches on its own, three at a time
