@@ -924,14 +924,22 @@ __device__ bool epilogue_role(const TcParams &P, const Smem &S, long long i0, in
       next_new = false;
       if (++nslab == P.nslabs) { nslab = 0; ++ntile; next_new = true; }
     }
-    if (P.residual != nullptr && valid && e == 0) {
+    if (P.residual != nullptr && e == 0) {
       // The residual tile of this item is pulled into L2 while its MMAs run: the loads in the
       // drain loop then see L2 latency only, and the bytes in flight are not bounded by registers.
-      const float *rp = P.residual + obase + (size_t)(slab * P.NT) * HoWo;
-      const int nf = min(P.NT, P.Co - slab * P.NT);
-      for (int j = 0; j < nf; ++j) {
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(rp));
-        rp += HoWo;
+      // The warp's pixels are one run of a filter's plane (at most 128 bytes: two lines), so a
+      // lane takes a filter and touches the two ends of its run: a handful of instructions per
+      // item instead of one prefetch per filter and lane.
+      const unsigned vm = __ballot_sync(0xffffffffu, valid);
+      if (vm != 0u) {
+        const unsigned long long o0 = __shfl_sync(0xffffffffu, (unsigned long long)obase, __ffs(vm) - 1);
+        const unsigned long long o1 = __shfl_sync(0xffffffffu, (unsigned long long)obase, 31 - __clz(vm));
+        const int nf = min(P.NT, P.Co - slab * P.NT);
+        const float *rp = P.residual + (size_t)(slab * P.NT) * HoWo;
+        for (int j = lane; j < nf; j += 32) {
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(rp + o0 + (size_t)j * HoWo));
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(rp + o1 + (size_t)j * HoWo));
+        }
       }
     }
     ok = mbar_wait_relaxed(S.afull + 8u * ab, fph, S.abort_flag, &g_status_tc, XNOR_SLEEP_EPI);
